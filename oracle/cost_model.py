@@ -1,0 +1,112 @@
+"""CPU restatement of the paper's scheduling cost model.  TEST INFRASTRUCTURE ONLY.
+
+Follows Section 3 equation by equation, in the paper's notation, in IEEE fp32
+(numpy float32 scalars: every operation is one correctly rounded fp32 operation,
+no fused multiply-add), so that a device implementation that uses the same
+operation order and round-to-nearest intrinsics must return the same plan.
+
+Single-GPU reading of the workload terms (the paper counts only remote tokens,
+which would be zero without peers): every token-expert pair moves through HBM,
+so with P pairs, T tokens and B = 2H bytes per row
+    W_comp     = P * 6*H*I              (Eq. 1, X_local + X_in = P)
+    W_dispatch = (T + P) * B            (Eq. 2: each token read once, P rows written)
+    W_combine  = (P + T) * B            (Eq. 3: P rows read, T rows written)
+    W_comm     = W_dispatch + W_combine (Eq. 11's undefined symbol, as in Eq. 5)
+
+Units: work in FLOPs / bytes, rates in FLOP/us and byte/us, times in us.
+Parity: pinned by closed forms in tests/test_oracle_cost_model.py.  The values
+the paper prints for its own runs (c*=40, K*=4 at 1.365 ms; 8.2 % gap; 0.54 us)
+depend on calibration curves that exist only as figures: parity unpinned for
+those, they are context only.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Sequence
+
+import numpy as np
+
+f32 = np.float32
+K_CANDIDATES = (1, 2, 4, 8)
+
+
+@dataclass
+class CostTables:
+    """Hardware input of the cost model (Figure 7: bandwidth / throughput curves)."""
+    n_sm: int
+    bw: np.ndarray        # [n_sm+1] float32, byte/us moved by c movement SMs (bw[0] unused)
+    tflops: np.ndarray    # [n_sm+1] float32, FLOP/us delivered by n GEMM SMs (tflops[0] unused)
+    eff_chunk: np.ndarray  # [4] float32, eff_chunk(K) for K = 1,2,4,8 (Eq. 9), eff_chunk[0] = 1
+    alpha: float          # tile-level overlap ratio in [0,1) (Section 3.1)
+    c_min: int = 2
+    c_max: int = 74
+    c_step: int = 2
+
+
+@dataclass
+class Plan:
+    c: int
+    K: int
+    n_steal: int
+    t_total: float
+
+
+def workloads(T: int, P: int, H: int, I: int):
+    """Eq. 1-3 under the single-GPU reading; fp32 like the device."""
+    B = f32(2 * H)
+    w_comp = f32(P) * f32(6.0) * f32(H) * f32(I)
+    w_disp = f32(T + P) * B
+    w_comb = f32(P + T) * B
+    return w_comp, w_disp, w_comb
+
+
+def t_total(tab: CostTables, c: int, ki: int, w_comp, w_disp, w_comb) -> np.float32:
+    """Eq. 15 with Eq. 9 (T_comp), Eq. 5 (T_comm) and Eq. 10 (T_tail)."""
+    K = f32(K_CANDIDATES[ki])
+    bw = f32(tab.bw[c])
+    tf = f32(tab.tflops[tab.n_sm - c])
+    t_comp = w_comp / (tf * f32(tab.eff_chunk[ki]))
+    t_comm = (w_disp + w_comb) / bw
+    t_tail = (f32(1.0) - f32(tab.alpha)) * (w_comb / (bw * K))
+    return np.maximum(t_comp + t_tail, t_comm)
+
+
+def candidates(tab: CostTables):
+    c = tab.c_min
+    while c <= tab.c_max and c <= tab.n_sm - 1:
+        yield c
+        c += tab.c_step
+
+
+def n_steal(tab: CostTables, c: int, w_comp, w_disp, w_comb, n_tiles: int) -> int:
+    """Eq. 11-14.  W_tile is the mean FLOPs of the n_tiles GEMM tiles of this layer,
+    so n_steal = W_steal / (N * W_tile); rounded to nearest (half away from zero is
+    impossible to hit exactly with these magnitudes; floor(x+0.5) is used), clamped
+    to [0, n_tiles]."""
+    if n_tiles <= 0:
+        return 0
+    t_comm = (w_disp + w_comb) / f32(tab.bw[c])                     # Eq. 11
+    w_partial = t_comm * f32(tab.tflops[tab.n_sm - c])              # Eq. 12
+    w_steal = np.maximum(f32(0.0), w_comp - w_partial)              # Eq. 13
+    w_tile = w_comp / f32(n_tiles)
+    if not (w_tile > 0):
+        return 0
+    ns = w_steal / (f32(tab.n_sm) * w_tile)                         # Eq. 14
+    ns = int(np.floor(ns + f32(0.5)))
+    return max(0, min(ns, n_tiles))
+
+
+def plan(tab: CostTables, T: int, P: int, H: int, I: int, n_tiles_of_K: Sequence[int]) -> Plan:
+    """Eq. 16: argmin over the (c,K) grid, ties to the smaller c and then the smaller K;
+    then the steal count at (c*,K*).  n_tiles_of_K[ki] = number of GEMM tiles of the
+    layer when it is cut into K_CANDIDATES[ki] chunks."""
+    w_comp, w_disp, w_comb = workloads(T, P, H, I)
+    best = None
+    for c in candidates(tab):
+        for ki in range(len(K_CANDIDATES)):
+            t = t_total(tab, c, ki, w_comp, w_disp, w_comb)
+            if best is None or t < best[0]:
+                best = (t, c, ki)
+    t, c, ki = best
+    return Plan(c, K_CANDIDATES[ki], n_steal(tab, c, w_comp, w_disp, w_comb, n_tiles_of_K[ki]),
+                float(t))
