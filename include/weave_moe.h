@@ -1,0 +1,153 @@
+/*
+ * weave_moe.h - C ABI of a single-GPU Mixture-of-Experts layer that runs as ONE persistent
+ * sm_100a kernel: top-k routing, dispatch (token-major -> expert-major rows), grouped expert
+ * SwiGLU GEMMs, combine (gate-weighted reduction back to token order), with an in-kernel cost
+ * model that splits the SMs between data-movement workers and GEMM workers and a tile-level
+ * ready-flag scheduler (chunk pipeline, bubble stealing).
+ *
+ * Conventions for every entry point
+ *   - Plain C, no exceptions, no global state.  Return value: 0 = WEAVE_OK, negative = error
+ *     (weave_moe_strerror() names it).
+ *   - "device pointer" = address in the memory of the CUDA device that is current when
+ *     weave_moe_create() is called; "host pointer" = ordinary (ideally pinned) host memory.
+ *   - The caller owns every buffer (weights, workspace, inputs, outputs) and keeps the weights
+ *     and the workspace alive and untouched until weave_moe_destroy().  The handle owns only
+ *     host state.  The library never allocates or frees device memory.
+ *   - One forward call per handle may be in flight at a time; calls are asynchronous on the
+ *     given stream unless stated otherwise.
+ *   - bf16 = IEEE-like bfloat16 bit patterns (upper 16 bits of an fp32).  All matrices are
+ *     row-major and dense.
+ */
+#ifndef WEAVE_MOE_H
+#define WEAVE_MOE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct weave_moe *weave_moe_t;
+
+enum {
+    WEAVE_OK = 0,
+    WEAVE_ERR_INVALID_ARG = -1,        /* null / misaligned pointer, bad shape, T > max_tokens, ...   */
+    WEAVE_ERR_UNSUPPORTED_DEVICE = -2, /* not an sm_100 device, or cooperative launch unavailable     */
+    WEAVE_ERR_CUDA = -3,               /* a CUDA runtime/driver call failed (see weave_moe_last_cuda_error) */
+    WEAVE_ERR_WORKSPACE = -4,          /* workspace_bytes smaller than weave_moe_workspace_bytes()    */
+    WEAVE_ERR_NONFINITE_LOGITS = -5,   /* device status: a router logit was NaN or +-inf               */
+    WEAVE_ERR_TIMEOUT = -6             /* device status: a bounded in-kernel wait expired              */
+};
+
+/* Scheduling modes (the paper's ablation, Section 5.5):
+ *   AUTO   - full method: the cost model of Section 3.3 (Eq. 15-16) picks the number of movement
+ *            SMs c and the chunk count K from the routing result, Eq. 11-14 give the steal count.
+ *   FIXED  - the given c, K and steal count are used as they are ("w/o T" when K = 1, steal = 0).
+ *   SERIAL - dispatch, GEMMs and combine run one after the other on all SMs ("w/o S+T").       */
+enum { WEAVE_SCHED_AUTO = 0, WEAVE_SCHED_FIXED = 1, WEAVE_SCHED_SERIAL = 2 };
+
+typedef struct weave_moe_config {
+    int hidden;       /* H: model width, multiple of 128                                          */
+    int ffn;          /* I: per-expert intermediate width, multiple of 128                         */
+    int num_experts;  /* E: routed experts, >= 1                                                  */
+    int top_k;        /* k: experts per token, 1 <= k <= min(E, 16)                               */
+    int num_shared;   /* S: always-on experts applied to every token with weight 1; E + S <= 256  */
+    int max_tokens;   /* largest T a forward call may pass (sizes the workspace)                  */
+    const void *gate_up; /* device, bf16 [E+S][2I][H]: rows [0,I) gate projection (gets SiLU),
+                            rows [I,2I) up projection; 16-byte aligned                            */
+    const void *down;    /* device, bf16 [E+S][H][I]; 16-byte aligned                             */
+    void *workspace;     /* device scratch of at least weave_moe_workspace_bytes(); 1024-byte aligned */
+    size_t workspace_bytes;
+} weave_moe_config;
+
+/* Bytes of device scratch a handle with this config needs.  Pure host arithmetic (reads only the
+ * six integer fields).  Returns 0 if the shape is invalid. */
+size_t weave_moe_workspace_bytes(const weave_moe_config *cfg);
+
+/* Validates the config, encodes the TMA descriptors of the weight and scratch matrices, zeroes
+ * the control words in the workspace (synchronous), installs default cost-model tables.
+ * The layer computed is the five-stage MoE forward of the paper's Section 2.1 / Figure 3, with the
+ * router added in front:  idx[t,0..k) = the k largest fp32 logits of token t (ties to the lowest
+ * expert index, listed by descending logit);  gate[t,j] = softmax over those k logits;
+ *   out[t] = sum_j gate[t,j] * Wd[e_j] ( silu(Wg[e_j] x[t]) (.) Wu[e_j] x[t] )  +  sum_s (same, shared
+ * expert s, weight 1).  Intermediates h and y are rounded to bf16; accumulation is fp32. */
+int weave_moe_create(const weave_moe_config *cfg, weave_moe_t *out_handle);
+
+/* One layer.  x: device bf16 [T][H];  router_logits: device fp32 [T][E];  out: device bf16 [T][H]
+ * (fully overwritten).  All three 16-byte aligned, not aliasing each other or the workspace.
+ * 0 <= T <= max_tokens (T = 0 is a no-op).  cuda_stream: a cudaStream_t (NULL = default stream).
+ * Launches exactly one kernel; returns once it is enqueued.  Device-side failures
+ * (WEAVE_ERR_NONFINITE_LOGITS, WEAVE_ERR_TIMEOUT) are reported by weave_moe_status(). */
+int weave_moe_forward(weave_moe_t h, const void *x, const float *router_logits, void *out, int T,
+                      void *cuda_stream);
+
+/* Same layer with HOST buffers: copies x and router_logits into staging areas of the workspace,
+ * runs weave_moe_forward, copies out back; all enqueued on the stream (asynchronous only if the
+ * host buffers are pinned). */
+int weave_moe_forward_host(weave_moe_t h, const void *x_host, const float *router_logits_host,
+                           void *out_host, int T, void *cuda_stream);
+
+/* Releases host state.  Does not touch device memory. */
+int weave_moe_destroy(weave_moe_t h);
+
+/* ---- scheduling surface (Section 3; ablation of Section 5.5) -------------------------------- */
+
+/* mode: WEAVE_SCHED_*.  For FIXED: c = number of movement SMs (clamped to [1, n_sm-1]), K = chunk
+ * count in {1,2,4,8}, steal = GEMM tiles each movement SM takes after dispatch (Section 3.2.2).
+ * Takes effect at the next forward. */
+int weave_moe_set_schedule(weave_moe_t h, int mode, int c, int K, int steal);
+
+/* Hardware input of the cost model (Figure 7): bw[i] = bytes/us moved by i movement SMs,
+ * tflops[i] = FLOP/us of i GEMM SMs, i in [0, n_sm] (host arrays of n_sm+1 floats, entry 0
+ * ignored); eff_chunk[4] = Eq. 9's correction factor for K = 1,2,4,8; alpha = Section 3.1's
+ * overlap ratio in [0,1); candidate grid c = c_min, c_min+c_step, ... <= c_max (at most 64
+ * values).  Synchronous copy to the device. */
+int weave_moe_set_cost_tables(weave_moe_t h, const float *bw, const float *tflops,
+                              const float *eff_chunk, float alpha, int c_min, int c_max, int c_step);
+
+/* Plan of the most recent forward (Section 3.3: SM split, chunk count, steal count) and the
+ * model's predicted layer time in us.  Synchronises the handle's last stream. */
+int weave_moe_get_plan(weave_moe_t h, int *c, int *K, int *n_steal, float *t_total_us);
+
+/* Geometry the scheduler works with: number of SMs (= persistent CTAs), rows per GEMM m-block,
+ * h-columns per gemm0 tile, out-columns per gemm1 tile, tokens per routing block, tokens per
+ * combine tile.  Any pointer may be NULL. */
+int weave_moe_get_geometry(weave_moe_t h, int *n_sm, int *block_m, int *tile_n0, int *tile_n1,
+                           int *route_block, int *combine_tile);
+
+/* ---- verification surface ------------------------------------------------------------------- */
+
+/* Device pointers INTO THE WORKSPACE holding the routing result of the most recent forward:
+ * topk_idx int32 [T][k], gates fp32 [T][k], counts int32 [E+S], offsets int32 [E+S+1],
+ * row_of int32 [T][k] (routed slots; the row of shared expert s is offsets[E+s] + t),
+ * token_of int32 [T*(k+S)].  Valid until the next forward.  Any pointer may be NULL. */
+int weave_moe_get_routing(weave_moe_t h, const int32_t **topk_idx, const float **gates,
+                          const int32_t **counts, const int32_t **offsets, const int32_t **row_of,
+                          const int32_t **token_of);
+
+/* Device pointers into the workspace of the expert-major intermediates of the most recent
+ * forward: xe bf16 [P][H] (dispatched rows), h bf16 [P][I], y bf16 [P][H], P = T*(k+S). */
+int weave_moe_get_intermediates(weave_moe_t h, const void **xe, const void **hbuf, const void **y);
+
+/* Synchronises the last stream, returns the device status word of the last forward
+ * (WEAVE_OK, WEAVE_ERR_NONFINITE_LOGITS, WEAVE_ERR_TIMEOUT) and clears it; after a failure it
+ * also re-zeroes the control words so that the handle is usable again. */
+int weave_moe_status(weave_moe_t h);
+
+/* Upper bound, in milliseconds, for any single in-kernel wait (grid barrier, ready flag,
+ * mbarrier); after it the kernel records WEAVE_ERR_TIMEOUT and every CTA returns.  Default 4000. */
+int weave_moe_set_timeout_ms(weave_moe_t h, int ms);
+
+/* Test hook for the give-up path: the m-block with this index never publishes its
+ * "dispatched" flag (-1 = off), so its consumer's bounded wait expires.  Host-side injection
+ * only; nothing faults or traps. */
+int weave_moe_debug_withhold_flag(weave_moe_t h, int m_block);
+
+int weave_moe_last_cuda_error(weave_moe_t h);
+const char *weave_moe_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WEAVE_MOE_H */

@@ -1,0 +1,933 @@
+// The persistent MoE-layer megakernel: one CTA per SM, one launch per layer.
+//
+//   phase R  (all CTAs)   warp-level top-k routing, per-block expert bitmasks -> in-block ranks and
+//                         a [block][expert] histogram; grid barrier (bounded)
+//   set-up   (every CTA, redundantly) counts, offsets, candidate tile counts, cost model -> plan
+//                         (c, K, n_steal), segment tables of the chosen K; permutation fix-up
+//   phase A  (movement CTAs: blockIdx < c)  dispatch tiles: gather x rows into expert-major Xe
+//   phase B  (GEMM CTAs until the queue is empty; movement CTAs for n_steal tiles)
+//                         warp-specialised TMA -> smem ring -> tcgen05.mma -> TMEM -> epilogue
+//   phase C  (every CTA once it has nothing else)  combine tiles, chunk by chunk as the chunk's
+//                         gemm1 tiles complete
+//
+// Stage list, roles, queue order, steal placement and the all-SM final combine follow the paper's
+// Sections 3 and 4; the cost model is Section 3's Eq. 1-16.
+#pragma once
+#include <cuda.h>
+
+#include "weave_ptx.cuh"
+
+namespace weave {
+
+constexpr int kThreads = 256;
+constexpr int kBM = 128;        // rows per GEMM m-block (UMMA M)
+constexpr int kBK = 64;         // K elements per pipeline stage: 128 bytes of bf16 = one swizzle row
+constexpr int kTN0 = 128;       // h columns per gemm0 tile; the MMA is N = 256 (gate | up)
+constexpr int kStages = 4;
+constexpr int kStageA = kBM * kBK * 2;                  // 16 KB
+constexpr int kStageB = 256 * kBK * 2;                  // 32 KB
+constexpr int kStageBytes = kStageA + kStageB;          // 48 KB
+constexpr int kRouteBlock = 64;  // tokens per routing block (one 64-bit mask per expert)
+constexpr int kCombTile = 16;    // tokens per combine tile
+constexpr int kMaxEE = 256;      // routed + shared experts
+constexpr int kMaxTopK = 16;
+constexpr int kFine = 8;         // fine chunks = largest chunk count K
+constexpr int kMaxSeg = kFine * kMaxEE;
+constexpr int kTinfo = 4;        // tile-descriptor ring between the producer and its consumers
+constexpr int kTmemCols = 512;
+constexpr int kEpiWarps = 4;     // warps 4..7
+
+constexpr int kErrNonFinite = -5;
+constexpr int kErrTimeout = -6;
+
+enum { kModeAuto = 0, kModeFixed = 1, kModeSerial = 2 };
+
+// Control words in global memory.  The first kCtlZeroWords words are zero at kernel entry and are
+// re-zeroed by the last CTA to leave, so no memset precedes a launch.
+struct Ctl {
+    unsigned bar_count;   // grid-barrier arrivals
+    unsigned q_disp;      // next dispatch tile
+    unsigned q_gemm;      // next GEMM tile (chunk-pipeline DAG order)
+    unsigned q_comb;      // next combine tile
+    unsigned fix_done;    // routing blocks whose rows are final
+    unsigned exit_count;
+    unsigned abort;       // set by the first wait that gives up; every wait polls it
+    unsigned pad0;
+    unsigned y_done[kFine];  // per chunk: epilogue-warp arrivals of finished gemm1 tiles
+    // ---- not re-zeroed: results for the host
+    int status;
+    int timeout_where;
+    int plan_c, plan_K, plan_steal;
+    float plan_t;
+    int plan_nmb, plan_ngemm;
+};
+constexpr int kCtlZeroWords = 16;
+
+struct KParams {
+    int T, H, I, E, S, k, EE;
+    int nblk;             // routing blocks = ceil(T / 64)
+    int mode, fixed_c, fixed_K, fixed_steal;
+    int bn1;              // out columns per gemm1 tile: 256, or 128 when H % 256 != 0
+    int nt0, nt1;         // n-tiles per m-block: I / 128, H / bn1
+    int nmb_max;          // allocated length of the per-m-block flag arrays
+    int withhold_mb;      // test hook: this m-block's "dispatched" flag is never published (-1 = off)
+    int c_min, c_max, c_step;
+    float alpha;
+    float eff[4];
+    unsigned long long timeout_ns;
+    const __nv_bfloat16 *x;
+    const float *logits;
+    __nv_bfloat16 *out;
+    Ctl *ctl;
+    unsigned *fcnt;       // [8][256] rows per (fine chunk, expert); zero at entry
+    int *hist;            // [nblk][256]
+    int *topk_idx;        // [T][k]
+    float *gates;         // [T][k]
+    int *row_of;          // [T][k]
+    int *token_of;        // [P]
+    int *counts;          // [EE]
+    int *offsets;         // [EE+1]
+    __nv_bfloat16 *xe;    // [P][H]
+    __nv_bfloat16 *hbuf;  // [P][I]
+    __nv_bfloat16 *y;     // [P][H]
+    unsigned *xe_ready;   // [nmb_max] 1 when the m-block's rows are dispatched; zero at entry
+    unsigned *h_ready;    // [nmb_max] epilogue-warp arrivals of the m-block's gemm0 tiles; zero at entry
+    const float *bw;      // [n_sm+1] byte/us
+    const float *tf;      // [n_sm+1] FLOP/us
+};
+
+struct TileInfo {
+    int type;   // 0 gemm0 (+SwiGLU), 1 gemm1, 2 no more tiles
+    int mb, row0, nrows, e, n, chunk, nkb;
+};
+
+struct SmemTail {
+    uint64_t full[kStages], empty[kStages];
+    uint64_t tmem_full[2], tmem_empty[2];
+    uint64_t ti_full[kTinfo], ti_empty[kTinfo];
+    TileInfo ti[kTinfo];
+    uint32_t tmem_base;
+    int bcast[3];
+    int red_i[8][4];
+    float red_f[8];
+    int scan_w[8];
+    int scan_total;
+    int c, K, steal, nmb, n_gemm, n_comb;
+    int chunk_mb0[kFine + 1];
+    int chunk_tile0[kFine + 1];
+    int offsets[kMaxEE + 1];
+    int tok[kBM];
+    int crow[8][kMaxTopK + 8];
+    float cgate[8][kMaxTopK + 8];
+    int seg_mb0[kMaxSeg + 1];
+    int seg_row0[kMaxSeg];
+    int seg_rows[kMaxSeg];
+};
+
+constexpr int kSmemBytes = kStages * kStageBytes + (int)sizeof(SmemTail) + 1024;
+static_assert(kSmemBytes <= 232448, "exceeds the 227 KB a CTA may opt into");
+
+// ------------------------------------------------------------------------------------ waits
+
+__device__ __noinline__ void give_up(Ctl *ctl, int where)
+{
+    if (atomicCAS(&ctl->status, 0, kErrTimeout) == 0) ctl->timeout_where = where;
+    atomicExch(&ctl->abort, 1u);
+}
+
+// Every wait is bounded: it polls the global abort word and a wall-clock limit, and returns false
+// instead of spinning forever.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, const KParams &p, int where)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    unsigned it = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++it & 31u) == 0u) {
+            if (ld_relaxed_u32(&p.ctl->abort)) return false;
+            if (globaltimer_ns() - t0 > p.timeout_ns) {
+                give_up(p.ctl, where);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ bool flag_wait_ge(const unsigned *flag, unsigned target, const KParams &p, int where)
+{
+    if (ld_acquire_u32(flag) >= target) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    unsigned it = 0;
+    while (ld_acquire_u32(flag) < target) {
+        __nanosleep(40);
+        if ((++it & 31u) == 0u) {
+            if (ld_relaxed_u32(&p.ctl->abort)) return false;
+            if (globaltimer_ns() - t0 > p.timeout_ns) {
+                give_up(p.ctl, where);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+// All CTAs are co-resident (cooperative launch); arrivals accumulate over the barriers of a launch.
+__device__ __forceinline__ bool grid_barrier(const KParams &p, SmemTail &S, unsigned target, int where)
+{
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        red_release_add_u32(&p.ctl->bar_count, 1u);
+        S.bcast[2] = flag_wait_ge(&p.ctl->bar_count, target, p, where) ? 1 : 0;
+    }
+    __syncthreads();
+    return S.bcast[2] != 0;
+}
+
+// ------------------------------------------------------------------------------------ block helpers
+
+__device__ __forceinline__ int block_excl_scan(int v, SmemTail &S, int &total)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        int n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
+    }
+    __syncthreads();
+    if (lane == 31) S.scan_w[warp] = inc;
+    __syncthreads();
+    int wbase = 0, tot = 0;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) {
+        int s = S.scan_w[w];
+        if (w < warp) wbase += s;
+        tot += s;
+    }
+    total = tot;
+    return wbase + inc - v;
+}
+
+// ------------------------------------------------------------------------------------ phase R
+
+// One warp routes one token: the k largest logits (ties to the lowest expert index) in descending
+// order, gates = softmax over those k.  Lane l holds the logits of experts l, l+32, ...
+__device__ __forceinline__ void route_token(const KParams &p, int t, int tl, unsigned long long *r_mask, int *r_idx)
+{
+    const int lane = threadIdx.x & 31;
+    const float NEG_INF = __int_as_float(0xff800000);
+    float v[kMaxEE / 32];
+    bool bad = false;
+#pragma unroll
+    for (int m = 0; m < kMaxEE / 32; ++m) {
+        int e = lane + 32 * m;
+        float x = NEG_INF;
+        if (e < p.E) {
+            x = __ldg(p.logits + (size_t)t * p.E + e);
+            if (!(fabsf(x) <= 3.402823466e38f)) {   // NaN or +-inf: flag it, keep indices in range
+                bad = true;
+                x = -3.402823466e38f;
+            }
+        }
+        v[m] = x;
+    }
+    if (__any_sync(0xffffffffu, bad) && lane == 0) atomicCAS(&p.ctl->status, 0, kErrNonFinite);
+
+    int my_e = 0;
+    float my_v = 0.f;
+    for (int j = 0; j < p.k; ++j) {
+        float bv = NEG_INF;
+        int be = 0x7fffffff;
+#pragma unroll
+        for (int m = 0; m < kMaxEE / 32; ++m)
+            if (v[m] > bv) { bv = v[m]; be = lane + 32 * m; }   // strict '>' keeps the lower index
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            float ov = __shfl_xor_sync(0xffffffffu, bv, o);
+            int oe = __shfl_xor_sync(0xffffffffu, be, o);
+            if (ov > bv || (ov == bv && oe < be)) { bv = ov; be = oe; }
+        }
+        if ((be & 31) == lane) {
+#pragma unroll
+            for (int m = 0; m < kMaxEE / 32; ++m)
+                if (m == (be >> 5)) v[m] = NEG_INF;             // taken
+        }
+        if (lane == j) { my_e = be; my_v = bv; }
+    }
+    const float vmax = __shfl_sync(0xffffffffu, my_v, 0);
+    const float pj = lane < p.k ? expf(my_v - vmax) : 0.f;
+    float sum = 0.f;
+    for (int j = 0; j < p.k; ++j) sum += __shfl_sync(0xffffffffu, pj, j);   // slot order
+    if (lane < p.k) {
+        p.topk_idx[(size_t)t * p.k + lane] = my_e;
+        p.gates[(size_t)t * p.k + lane] = __fdiv_rn(pj, sum);
+        r_idx[tl * kMaxTopK + lane] = my_e;
+        atomicOr(&r_mask[my_e], 1ull << tl);
+    }
+}
+
+// ------------------------------------------------------------------------------------ cost model
+
+// Eq. 15 for one candidate, in the same fp32 operation order as the CPU restatement:
+// T_comp = W_comp / (TFLOPS(N-c) * eff_chunk(K))  (Eq. 9),  T_comm = (W_disp + W_comb) / BW(c)  (Eq. 5),
+// T_tail = (1 - alpha) * W_comb / (BW(c) * K)  (Eq. 10),  T_total = max(T_comp + T_tail, T_comm).
+__device__ __forceinline__ float model_t_total(const KParams &p, int n_sm, int c, int ki, float w_comp, float w_disp,
+                                               float w_comb)
+{
+    const float Kf = (float)(1 << ki);
+    const float bw = p.bw[c];
+    const float tf = p.tf[n_sm - c];
+    const float t_comp = __fdiv_rn(w_comp, __fmul_rn(tf, p.eff[ki]));
+    const float t_comm = __fdiv_rn(__fadd_rn(w_disp, w_comb), bw);
+    const float t_tail = __fmul_rn(__fsub_rn(1.0f, p.alpha), __fdiv_rn(w_comb, __fmul_rn(bw, Kf)));
+    return fmaxf(__fadd_rn(t_comp, t_tail), t_comm);
+}
+
+// Eq. 11-14 with W_tile = W_comp / n_tiles (the mean GEMM tile of this layer).
+__device__ __forceinline__ int model_n_steal(const KParams &p, int n_sm, int c, float w_comp, float w_disp,
+                                             float w_comb, int n_tiles)
+{
+    if (n_tiles <= 0) return 0;
+    const float t_comm = __fdiv_rn(__fadd_rn(w_disp, w_comb), p.bw[c]);
+    const float w_partial = __fmul_rn(t_comm, p.tf[n_sm - c]);
+    const float w_steal = fmaxf(0.0f, __fsub_rn(w_comp, w_partial));
+    const float w_tile = __fdiv_rn(w_comp, (float)n_tiles);
+    if (!(w_tile > 0.0f)) return 0;
+    const float ns = __fdiv_rn(w_steal, __fmul_rn((float)n_sm, w_tile));
+    int r = (int)floorf(__fadd_rn(ns, 0.5f));
+    return max(0, min(r, n_tiles));
+}
+
+// ------------------------------------------------------------------------------------ tile decoding
+
+// largest s in [lo, hi) with (seg_mb0[s] - base) * mul <= key   (empty segments share a start)
+__device__ __forceinline__ int seg_search(const SmemTail &S, int lo, int hi, int base, int mul, int key)
+{
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if ((S.seg_mb0[mid] - base) * mul <= key) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+__device__ __forceinline__ void decode_mblock(const SmemTail &S, int EE, int mb, int &row0, int &nrows)
+{
+    const int s = seg_search(S, 0, S.K * EE, 0, 1, mb);
+    const int m = mb - S.seg_mb0[s];
+    row0 = S.seg_row0[s] + m * kBM;
+    nrows = min(kBM, S.seg_rows[s] - m * kBM);
+}
+
+// GEMM queue order (the chunk-pipeline DAG order): chunk by chunk; inside a chunk all gemm0 tiles,
+// then all gemm1 tiles; inside those expert-major, n-tile, m-block fastest (so consecutive tiles
+// share a weight panel in L2).
+__device__ __forceinline__ void decode_gemm_tile(const SmemTail &S, const KParams &p, int g, TileInfo &ti)
+{
+    int j = 0;
+    while (j + 1 < S.K && g >= S.chunk_tile0[j + 1]) ++j;
+    int local = g - S.chunk_tile0[j];
+    const int cmb0 = S.chunk_mb0[j];
+    const int nmbj = S.chunk_mb0[j + 1] - cmb0;
+    int type = 0, nt = p.nt0;
+    if (local >= nmbj * p.nt0) { type = 1; local -= nmbj * p.nt0; nt = p.nt1; }
+    const int s = seg_search(S, j * p.EE, (j + 1) * p.EE, cmb0, nt, local);
+    const int mbs = S.seg_mb0[s + 1] - S.seg_mb0[s];
+    const int within = local - (S.seg_mb0[s] - cmb0) * nt;
+    const int n = within / mbs, m = within - n * mbs;
+    ti.type = type;
+    ti.mb = S.seg_mb0[s] + m;
+    ti.row0 = S.seg_row0[s] + m * kBM;
+    ti.nrows = min(kBM, S.seg_rows[s] - m * kBM);
+    ti.e = s - j * p.EE;
+    ti.n = n;
+    ti.chunk = j;
+    ti.nkb = (type == 0 ? p.H : p.I) / kBK;
+}
+
+// ------------------------------------------------------------------------------------ phase A: dispatch
+
+// Tile = one m-block: Xe[row0 + r] = x[token_of[row0 + r]].  16-byte vectors, 8 loads in flight
+// per thread; the m-block's ready flag is released when its rows are written.
+__device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S)
+{
+    const int tid = threadIdx.x;
+    if (tid == 0) S.bcast[1] = flag_wait_ge(&p.ctl->fix_done, (unsigned)p.nblk, p, 10) ? 1 : 0;
+    __syncthreads();
+    if (!S.bcast[1]) return;
+    const int n16 = p.H >> 3;
+    for (;;) {
+        if (tid == 0) S.bcast[0] = (int)atomicAdd(&p.ctl->q_disp, 1u);
+        __syncthreads();
+        const int mb = S.bcast[0];
+        if (mb >= S.nmb) break;
+        int row0, nrows;
+        decode_mblock(S, p.EE, mb, row0, nrows);
+        for (int i = tid; i < nrows; i += kThreads) S.tok[i] = __ldcg(p.token_of + row0 + i);
+        __syncthreads();
+        const int total = nrows * n16;
+        constexpr int U = 8;
+        for (int base = tid; base < total; base += kThreads * U) {
+            uint4 v[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int i = base + u * kThreads;
+                if (i < total) {
+                    const int r = i / n16, c = i - r * n16;
+                    v[u] = ld_nc_v4(p.x + (size_t)S.tok[r] * p.H + (size_t)c * 8);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int i = base + u * kThreads;
+                if (i < total) {
+                    const int r = i / n16, c = i - r * n16;
+                    st_v4(p.xe + (size_t)(row0 + r) * p.H + (size_t)c * 8, v[u]);
+                }
+            }
+        }
+        fence_proxy_async();      // these rows are read by TMA (async proxy) on another SM
+        __syncthreads();
+        if (tid == 0 && mb != p.withhold_mb) {
+            __threadfence();
+            st_release_u32(&p.xe_ready[mb], 1u);
+        }
+    }
+    __syncthreads();
+}
+
+// ------------------------------------------------------------------------------------ phase C: combine
+
+// Tile = 16 tokens; a warp owns two of them.  out[t] = sum_j gate[t,j] * y[row_of[t,j]] in slot
+// order, then the shared experts with weight 1; fp32 accumulate, bf16 store.
+__device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S)
+{
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n16 = p.H >> 3;
+    const int kk = p.k + p.S;
+    const int g = kFine / S.K;
+    int ready_upto = -1;     // chunks [0, ready_upto] are known complete
+    for (;;) {
+        if (tid == 0) S.bcast[0] = (int)atomicAdd(&p.ctl->q_comb, 1u);
+        __syncthreads();
+        const int q = S.bcast[0];
+        if (q >= S.n_comb) break;
+        const int t0 = q * kCombTile;
+        const int chunk = (((t0 / kRouteBlock) * kFine) / p.nblk) / g;
+        if (chunk > ready_upto) {
+            if (tid == 0) {
+                bool ok = flag_wait_ge(&p.ctl->fix_done, (unsigned)p.nblk, p, 20);
+                for (int j = ready_upto + 1; ok && j <= chunk; ++j) {
+                    const unsigned target = (unsigned)((S.chunk_mb0[j + 1] - S.chunk_mb0[j]) * p.nt1 * kEpiWarps);
+                    ok = flag_wait_ge(&p.ctl->y_done[j], target, p, 21);
+                }
+                S.bcast[1] = ok ? 1 : 0;
+            }
+            __syncthreads();
+            if (!S.bcast[1]) break;
+            ready_upto = chunk;
+        }
+        for (int tt = 0; tt < kCombTile / 8; ++tt) {
+            const int t = t0 + warp * (kCombTile / 8) + tt;
+            if (t >= p.T) break;                                   // warp-uniform
+            if (lane < p.k) {
+                S.crow[warp][lane] = __ldcg(p.row_of + (size_t)t * p.k + lane);
+                S.cgate[warp][lane] = __ldcg(p.gates + (size_t)t * p.k + lane);
+            } else if (lane < kk) {
+                S.crow[warp][lane] = S.offsets[p.E + (lane - p.k)] + t;
+                S.cgate[warp][lane] = 1.0f;
+            }
+            __syncwarp();
+            for (int v = lane; v < n16; v += 64) {
+                const bool has1 = (v + 32) < n16;
+                float a0[8], a1[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) { a0[i] = 0.f; a1[i] = 0.f; }
+                for (int j0 = 0; j0 < kk; j0 += 4) {
+                    uint4 q0[4], q1[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (j0 + u < kk) {
+                            const __nv_bfloat16 *src = p.y + (size_t)S.crow[warp][j0 + u] * p.H + (size_t)v * 8;
+                            q0[u] = ld_cg_v4(src);
+                            if (has1) q1[u] = ld_cg_v4(src + 256);
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (j0 + u < kk) {
+                            const float gw = S.cgate[warp][j0 + u];
+                            a0[0] = fmaf(gw, bf16lo_to_f32(q0[u].x), a0[0]); a0[1] = fmaf(gw, bf16hi_to_f32(q0[u].x), a0[1]);
+                            a0[2] = fmaf(gw, bf16lo_to_f32(q0[u].y), a0[2]); a0[3] = fmaf(gw, bf16hi_to_f32(q0[u].y), a0[3]);
+                            a0[4] = fmaf(gw, bf16lo_to_f32(q0[u].z), a0[4]); a0[5] = fmaf(gw, bf16hi_to_f32(q0[u].z), a0[5]);
+                            a0[6] = fmaf(gw, bf16lo_to_f32(q0[u].w), a0[6]); a0[7] = fmaf(gw, bf16hi_to_f32(q0[u].w), a0[7]);
+                            if (has1) {
+                                a1[0] = fmaf(gw, bf16lo_to_f32(q1[u].x), a1[0]); a1[1] = fmaf(gw, bf16hi_to_f32(q1[u].x), a1[1]);
+                                a1[2] = fmaf(gw, bf16lo_to_f32(q1[u].y), a1[2]); a1[3] = fmaf(gw, bf16hi_to_f32(q1[u].y), a1[3]);
+                                a1[4] = fmaf(gw, bf16lo_to_f32(q1[u].z), a1[4]); a1[5] = fmaf(gw, bf16hi_to_f32(q1[u].z), a1[5]);
+                                a1[6] = fmaf(gw, bf16lo_to_f32(q1[u].w), a1[6]); a1[7] = fmaf(gw, bf16hi_to_f32(q1[u].w), a1[7]);
+                            }
+                        }
+                    }
+                }
+                __nv_bfloat16 *dst = p.out + (size_t)t * p.H + (size_t)v * 8;
+                st_cs_v4(dst, make_uint4(pack_bf16x2(a0[0], a0[1]), pack_bf16x2(a0[2], a0[3]),
+                                         pack_bf16x2(a0[4], a0[5]), pack_bf16x2(a0[6], a0[7])));
+                if (has1)
+                    st_cs_v4(dst + 256, make_uint4(pack_bf16x2(a1[0], a1[1]), pack_bf16x2(a1[2], a1[3]),
+                                                   pack_bf16x2(a1[4], a1[5]), pack_bf16x2(a1[6], a1[7])));
+            }
+            __syncwarp();
+        }
+        __syncthreads();
+    }
+    __syncthreads();
+}
+
+// ------------------------------------------------------------------------------------ phase B: GEMM
+
+struct PipeState {     // per-role ring positions; they persist across the tiles of a phase
+    int stage = 0;  uint32_t stage_phase = 0;
+    int acc = 0;    uint32_t acc_phase = 0;
+    int slot = 0;   uint32_t slot_phase = 0;
+    __device__ __forceinline__ void next_stage() { if (++stage == kStages) { stage = 0; stage_phase ^= 1u; } }
+    __device__ __forceinline__ void next_acc() { if (++acc == 2) { acc = 0; acc_phase ^= 1u; } }
+    __device__ __forceinline__ void next_slot() { if (++slot == kTinfo) { slot = 0; slot_phase ^= 1u; } }
+};
+
+__device__ __forceinline__ float silu_mul(float g, float u)
+{
+    return __fdividef(g, 1.0f + __expf(-g)) * u;
+}
+
+// budget = how many tiles this CTA may claim (the steal count for a movement CTA).
+__device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_t *stages, uint32_t tmem_base,
+                                           const CUtensorMap *tm_xe, const CUtensorMap *tm_wgu,
+                                           const CUtensorMap *tm_h, const CUtensorMap *tm_wd, int budget,
+                                           PipeState &ps)
+{
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    fence_proxy_async();     // the stage buffers were last touched by ordinary stores (routing scratch)
+    __syncthreads();
+
+    if (warp == 0) {
+        // ---------------- producer: claims tiles, waits for their inputs, feeds the smem ring by TMA
+        if (lane == 0) {
+            int taken = 0;
+            bool dead = false;
+            while (!dead) {
+                TileInfo ti;
+                const int g = taken < budget ? (int)atomicAdd(&p.ctl->q_gemm, 1u) : 0x7fffffff;
+                if (g >= S.n_gemm) ti.type = 2; else decode_gemm_tile(S, p, g, ti);
+                if (!mbar_wait(&S.ti_empty[ps.slot], ps.slot_phase ^ 1u, p, 30)) { dead = true; break; }
+                S.ti[ps.slot] = ti;
+                mbar_arrive(&S.ti_full[ps.slot]);
+                ps.next_slot();
+                if (ti.type == 2) break;
+                ++taken;
+                const CUtensorMap *tma_a, *tma_b;
+                int brow0, brow1;
+                bool ok;
+                if (ti.type == 0) {
+                    ok = flag_wait_ge(&p.xe_ready[ti.mb], 1u, p, 31);
+                    tma_a = tm_xe; tma_b = tm_wgu;
+                    brow0 = ti.e * 2 * p.I + ti.n * kTN0;     // gate rows
+                    brow1 = brow0 + p.I;                       // up rows
+                } else {
+                    ok = flag_wait_ge(&p.h_ready[ti.mb], (unsigned)(p.nt0 * kEpiWarps), p, 32);
+                    tma_a = tm_h; tma_b = tm_wd;
+                    brow0 = ti.e * p.H + ti.n * p.bn1;
+                    brow1 = brow0 + 128;
+                }
+                if (!ok) { dead = true; break; }
+                fence_proxy_async();     // rows written with ordinary stores elsewhere, read by TMA here
+                const bool two_b = (ti.type == 0) || (p.bn1 == 256);
+                const uint32_t tx = kStageA + (two_b ? kStageB : kStageB / 2);
+                for (int kb = 0; kb < ti.nkb; ++kb) {
+                    if (!mbar_wait(&S.empty[ps.stage], ps.stage_phase ^ 1u, p, 33)) { dead = true; break; }
+                    uint8_t *sa = stages + ps.stage * kStageBytes;
+                    uint8_t *sb = sa + kStageA;
+                    mbar_arrive_expect_tx(&S.full[ps.stage], tx);
+                    tma_load_2d(sa, tma_a, kb * kBK, ti.row0, &S.full[ps.stage]);
+                    tma_load_2d(sb, tma_b, kb * kBK, brow0, &S.full[ps.stage]);
+                    if (two_b) tma_load_2d(sb + kStageB / 2, tma_b, kb * kBK, brow1, &S.full[ps.stage]);
+                    ps.next_stage();
+                }
+            }
+            if (dead) {     // let loads already issued land before this CTA can leave
+                const unsigned long long t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 50000ull) __nanosleep(1000);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---------------- MMA issuer: one thread drives the tensor core, accumulators live in TMEM
+        if (lane == 0) {
+            bool dead = false;
+            while (!dead) {
+                if (!mbar_wait(&S.ti_full[ps.slot], ps.slot_phase, p, 40)) { dead = true; break; }
+                const TileInfo ti = S.ti[ps.slot];
+                mbar_arrive(&S.ti_empty[ps.slot]);
+                ps.next_slot();
+                if (ti.type == 2) break;
+                const uint32_t idesc = umma_idesc_bf16(kBM, ti.type == 0 ? 256u : (uint32_t)p.bn1);
+                if (!mbar_wait(&S.tmem_empty[ps.acc], ps.acc_phase ^ 1u, p, 41)) { dead = true; break; }
+                tc_fence_after();
+                const uint32_t d = tmem_base + (uint32_t)ps.acc * 256u;
+                for (int kb = 0; kb < ti.nkb; ++kb) {
+                    if (!mbar_wait(&S.full[ps.stage], ps.stage_phase, p, 42)) { dead = true; break; }
+                    tc_fence_after();
+                    const uint32_t a0 = smem_u32(stages + ps.stage * kStageBytes);
+                    const uint32_t b0 = a0 + kStageA;
+#pragma unroll
+                    for (int kk = 0; kk < kBK / 16; ++kk)
+                        tc_mma_bf16(d, umma_desc_sw128(a0 + kk * 32), umma_desc_sw128(b0 + kk * 32), idesc,
+                                    (uint32_t)((kb | kk) != 0));
+                    tc_commit(&S.empty[ps.stage]);       // frees the stage when these MMAs have read it
+                    ps.next_stage();
+                }
+                if (dead) break;
+                tc_commit(&S.tmem_full[ps.acc]);         // accumulator complete
+                ps.next_acc();
+            }
+            if (dead) {
+                const unsigned long long t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 50000ull) __nanosleep(1000);
+            }
+        }
+        __syncwarp();
+    } else if (warp >= 4) {
+        // ---------------- epilogue: TMEM -> registers -> (SwiGLU) -> bf16 -> global, row-masked
+        const int q = warp & 3;                      // TMEM lane quadrant this warp may read
+        bool dead = false;
+        while (!dead) {
+            if (!mbar_wait(&S.ti_full[ps.slot], ps.slot_phase, p, 50)) { dead = true; }
+            dead = __any_sync(0xffffffffu, dead);
+            if (dead) break;
+            const TileInfo ti = S.ti[ps.slot];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&S.ti_empty[ps.slot]);
+            ps.next_slot();
+            if (ti.type == 2) break;
+            if (!mbar_wait(&S.tmem_full[ps.acc], ps.acc_phase, p, 51)) { dead = true; }
+            dead = __any_sync(0xffffffffu, dead);
+            if (dead) break;
+            tc_fence_after();
+            const int r = q * 32 + lane;
+            const bool valid = r < ti.nrows;
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)ps.acc * 256u;
+            if (ti.type == 0) {
+                __nv_bfloat16 *dst = p.hbuf + (size_t)(ti.row0 + r) * p.I + (size_t)ti.n * kTN0;
+#pragma unroll 1
+                for (int c = 0; c < kTN0 / 32; ++c) {
+                    uint32_t gr[32], ur[32];
+                    tmem_ld_32x32(taddr + c * 32, gr);
+                    tmem_ld_32x32(taddr + 128 + c * 32, ur);
+                    tmem_ld_wait();
+                    uint32_t o[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        o[i] = pack_bf16x2(silu_mul(__uint_as_float(gr[2 * i]), __uint_as_float(ur[2 * i])),
+                                           silu_mul(__uint_as_float(gr[2 * i + 1]), __uint_as_float(ur[2 * i + 1])));
+                    if (valid) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            st_v4(dst + c * 32 + i * 8, make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]));
+                    }
+                }
+            } else {
+                __nv_bfloat16 *dst = p.y + (size_t)(ti.row0 + r) * p.H + (size_t)ti.n * p.bn1;
+                const int nc = p.bn1 / 32;
+#pragma unroll 1
+                for (int c = 0; c < nc; ++c) {
+                    uint32_t ar[32];
+                    tmem_ld_32x32(taddr + c * 32, ar);
+                    tmem_ld_wait();
+                    if (valid) {
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            st_v4(dst + c * 32 + i * 8,
+                                  make_uint4(pack_bf16x2(__uint_as_float(ar[8 * i]), __uint_as_float(ar[8 * i + 1])),
+                                             pack_bf16x2(__uint_as_float(ar[8 * i + 2]), __uint_as_float(ar[8 * i + 3])),
+                                             pack_bf16x2(__uint_as_float(ar[8 * i + 4]), __uint_as_float(ar[8 * i + 5])),
+                                             pack_bf16x2(__uint_as_float(ar[8 * i + 6]), __uint_as_float(ar[8 * i + 7]))));
+                    }
+                }
+            }
+            // accumulator may be overwritten by the next-but-one tile
+            tc_fence_before();
+            fence_proxy_async();     // h rows are read by TMA on another SM
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(&S.tmem_empty[ps.acc]);
+                __threadfence();
+                red_release_add_u32(ti.type == 0 ? &p.h_ready[ti.mb] : &p.ctl->y_done[ti.chunk], 1u);
+            }
+            ps.next_acc();
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+}
+
+// ------------------------------------------------------------------------------------ the kernel
+
+__global__ void __launch_bounds__(kThreads, 1)
+weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUtensorMap tm_xe,
+                 const __grid_constant__ CUtensorMap tm_wgu, const __grid_constant__ CUtensorMap tm_h,
+                 const __grid_constant__ CUtensorMap tm_wd)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *stages = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    SmemTail &S = *reinterpret_cast<SmemTail *>(stages + kStages * kStageBytes);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_sm = (int)gridDim.x;
+    const int EE = p.EE;
+
+    if (tid == 0) {
+        for (int i = 0; i < kStages; ++i) { mbar_init(&S.full[i], 1); mbar_init(&S.empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&S.tmem_full[i], 1); mbar_init(&S.tmem_empty[i], kEpiWarps); }
+        for (int i = 0; i < kTinfo; ++i) { mbar_init(&S.ti_full[i], 1); mbar_init(&S.ti_empty[i], 1 + kEpiWarps); }
+        fence_mbar_init();
+        tma_prefetch_desc(&tm_xe); tma_prefetch_desc(&tm_wgu); tma_prefetch_desc(&tm_h); tma_prefetch_desc(&tm_wd);
+    }
+    if (warp == 1) { tmem_alloc(&S.tmem_base, kTmemCols); tmem_relinquish(); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = S.tmem_base;
+
+    // routing scratch lives in the (not yet used) stage buffers
+    unsigned long long *r_mask = reinterpret_cast<unsigned long long *>(stages);          // [256]
+    int *r_idx = reinterpret_cast<int *>(stages + 2048);                                   // [64][16]
+    int *r_base = reinterpret_cast<int *>(stages + 2048 + kRouteBlock * kMaxTopK * 4);     // [256]
+
+    // ================= phase R: routing
+    for (int b = blockIdx.x; b < p.nblk; b += n_sm) {
+        for (int e = tid; e < EE; e += kThreads) r_mask[e] = 0ull;
+        __syncthreads();
+        for (int tl = warp; tl < kRouteBlock; tl += kThreads / 32) {
+            const int t = b * kRouteBlock + tl;
+            if (t < p.T) route_token(p, t, tl, r_mask, r_idx);
+        }
+        __syncthreads();
+        // in-block rank of each (token, slot): tokens before it in the block that chose the same expert
+        for (int pi = tid; pi < kRouteBlock * p.k; pi += kThreads) {
+            const int tl = pi / p.k, j = pi - tl * p.k;
+            const int t = b * kRouteBlock + tl;
+            if (t < p.T) {
+                const int e = r_idx[tl * kMaxTopK + j];
+                p.row_of[(size_t)t * p.k + j] = __popcll(r_mask[e] & ((1ull << tl) - 1ull));
+            }
+        }
+        const int ntok = min(kRouteBlock, p.T - b * kRouteBlock);
+        const int f = (b * kFine) / p.nblk;
+        for (int e = tid; e < EE; e += kThreads) {
+            const int cnt = e < p.E ? __popcll(r_mask[e]) : ntok;
+            p.hist[(size_t)b * kMaxEE + e] = cnt;
+            if (cnt) atomicAdd(&p.fcnt[f * kMaxEE + e], (unsigned)cnt);
+        }
+        __syncthreads();
+    }
+    bool alive = grid_barrier(p, S, (unsigned)n_sm, 1);
+
+    // ================= set-up: counts, offsets, plan, segment tables (identical on every CTA)
+    int cf[kFine];
+    int cnt = 0;
+#pragma unroll
+    for (int f = 0; f < kFine; ++f) {
+        cf[f] = (alive && tid < EE) ? (int)__ldcg(p.fcnt + f * kMaxEE + tid) : 0;
+        cnt += cf[f];
+    }
+    int total_rows;
+    const int off = block_excl_scan(cnt, S, total_rows);
+    if (tid < EE) S.offsets[tid] = off;
+    if (tid == 0) S.offsets[EE] = total_rows;
+    if (blockIdx.x == 0 && tid < EE) {
+        p.counts[tid] = cnt;
+        p.offsets[tid] = off;
+        if (tid == 0) p.offsets[EE] = total_rows;
+    }
+    // m-blocks of the layer for each candidate K (a segment = one expert's rows inside one chunk)
+    int mbk[4];
+#pragma unroll
+    for (int ki = 0; ki < 4; ++ki) {
+        const int K = 1 << ki, g = kFine / K;
+        int acc = 0;
+        for (int j = 0; j < K; ++j) {
+            int rows = 0;
+#pragma unroll
+            for (int f = 0; f < kFine; ++f) if (f / g == j) rows += cf[f];
+            acc += (rows + kBM - 1) / kBM;
+        }
+        mbk[ki] = acc;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mbk[ki] += __shfl_xor_sync(0xffffffffu, mbk[ki], o);
+    }
+    if (lane == 0) { S.red_i[warp][0] = mbk[0]; S.red_i[warp][1] = mbk[1]; S.red_i[warp][2] = mbk[2]; S.red_i[warp][3] = mbk[3]; }
+    __syncthreads();
+    int n_tiles_k[4];
+#pragma unroll
+    for (int ki = 0; ki < 4; ++ki) {
+        int s = 0;
+        for (int w = 0; w < kThreads / 32; ++w) s += S.red_i[w][ki];
+        n_tiles_k[ki] = s * (p.nt0 + p.nt1);
+    }
+    __syncthreads();     // red_i is reused by the arg-min below
+
+    const int P = p.T * (p.k + p.S);
+    int plan_c, plan_ki, plan_steal;
+    float plan_t = 0.f;
+    if (p.mode == kModeAuto) {
+        // Eq. 1-3 (single-GPU reading: every pair moves through HBM), then Eq. 16 over the grid
+        const float B = (float)(2 * p.H);
+        const float w_comp = __fmul_rn(__fmul_rn(__fmul_rn((float)P, 6.0f), (float)p.H), (float)p.I);
+        const float w_disp = __fmul_rn((float)(p.T + P), B);
+        const float w_comb = __fmul_rn((float)(P + p.T), B);
+        const int ci = tid >> 2, ki = tid & 3;
+        const int cc = p.c_min + ci * p.c_step;
+        float t = __int_as_float(0x7f800000);
+        if (cc >= 1 && cc <= p.c_max && cc <= n_sm - 1) t = model_t_total(p, n_sm, cc, ki, w_comp, w_disp, w_comb);
+        int bi = tid;       // candidate order = (c ascending, K ascending): ties go to the smaller index
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ot = __shfl_xor_sync(0xffffffffu, t, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+            if (ot < t || (ot == t && oi < bi)) { t = ot; bi = oi; }
+        }
+        if (lane == 0) { S.red_f[warp] = t; S.red_i[warp][0] = bi; }
+        __syncthreads();
+        t = S.red_f[0]; bi = S.red_i[0][0];
+        for (int w = 1; w < kThreads / 32; ++w) {
+            const float ot = S.red_f[w];
+            const int oi = S.red_i[w][0];
+            if (ot < t || (ot == t && oi < bi)) { t = ot; bi = oi; }
+        }
+        plan_c = p.c_min + (bi >> 2) * p.c_step;
+        plan_ki = bi & 3;
+        plan_t = t;
+        plan_steal = model_n_steal(p, n_sm, plan_c, w_comp, w_disp, w_comb, n_tiles_k[plan_ki]);
+        __syncthreads();
+    } else if (p.mode == kModeFixed) {
+        plan_c = max(1, min(p.fixed_c, n_sm - 1));
+        plan_ki = p.fixed_K >= 8 ? 3 : p.fixed_K >= 4 ? 2 : p.fixed_K >= 2 ? 1 : 0;
+        plan_steal = max(0, p.fixed_steal);
+    } else {
+        plan_c = n_sm;
+        plan_ki = 0;
+        plan_steal = 0;
+    }
+    const int K = 1 << plan_ki;
+    {
+        const int g = kFine / K;
+        int run_row = tid < EE ? off : 0;
+        int mb_base = 0;
+        for (int j = 0; j < K; ++j) {
+            int rows = 0;
+#pragma unroll
+            for (int f = 0; f < kFine; ++f) if (f / g == j) rows += cf[f];
+            const int mbs = (rows + kBM - 1) / kBM;
+            int tot;
+            const int ex = block_excl_scan(mbs, S, tot);
+            if (tid < EE) {
+                S.seg_mb0[j * EE + tid] = mb_base + ex;
+                S.seg_row0[j * EE + tid] = run_row;
+                S.seg_rows[j * EE + tid] = rows;
+            }
+            if (tid == 0) { S.chunk_mb0[j] = mb_base; S.chunk_tile0[j] = mb_base * (p.nt0 + p.nt1); }
+            run_row += rows;
+            mb_base += tot;
+        }
+        if (tid == 0) {
+            S.seg_mb0[K * EE] = mb_base;
+            S.chunk_mb0[K] = mb_base;
+            S.chunk_tile0[K] = mb_base * (p.nt0 + p.nt1);
+            S.c = plan_c; S.K = K; S.steal = plan_steal;
+            S.nmb = mb_base;
+            S.n_gemm = mb_base * (p.nt0 + p.nt1);
+            S.n_comb = (p.T + kCombTile - 1) / kCombTile;
+            if (blockIdx.x == 0) {
+                p.ctl->plan_c = plan_c; p.ctl->plan_K = K; p.ctl->plan_steal = plan_steal; p.ctl->plan_t = plan_t;
+                p.ctl->plan_nmb = mb_base; p.ctl->plan_ngemm = mb_base * (p.nt0 + p.nt1);
+            }
+        }
+    }
+    __syncthreads();
+
+    // ================= permutation fix-up: in-block rank + rows of earlier blocks + expert offset
+    if (alive) {
+        int fixed = 0;
+        for (int b = blockIdx.x; b < p.nblk; b += n_sm) {
+            const int f = (b * kFine) / p.nblk;
+            const int bstart = (f * p.nblk + kFine - 1) / kFine;
+            if (tid < EE) {
+                int base = off;
+#pragma unroll
+                for (int ff = 0; ff < kFine; ++ff) if (ff < f) base += cf[ff];
+                for (int bb = bstart; bb < b; ++bb) base += __ldcg(p.hist + (size_t)bb * kMaxEE + tid);
+                r_base[tid] = base;
+            }
+            __syncthreads();
+            for (int pi = tid; pi < kRouteBlock * p.k; pi += kThreads) {
+                const int tl = pi / p.k, j = pi - tl * p.k;
+                const int t = b * kRouteBlock + tl;
+                if (t < p.T) {
+                    const int e = __ldcg(p.topk_idx + (size_t)t * p.k + j);
+                    const int r = __ldcg(p.row_of + (size_t)t * p.k + j) + r_base[e];
+                    p.row_of[(size_t)t * p.k + j] = r;
+                    p.token_of[r] = t;
+                }
+            }
+            for (int pi = tid; pi < kRouteBlock * p.S; pi += kThreads) {
+                const int tl = pi / p.S, s = pi - tl * p.S;
+                const int t = b * kRouteBlock + tl;
+                if (t < p.T) p.token_of[S.offsets[p.E + s] + t] = t;
+            }
+            __syncthreads();
+            ++fixed;
+        }
+        if (tid == 0 && fixed) {
+            __threadfence();
+            red_release_add_u32(&p.ctl->fix_done, (unsigned)fixed);
+        }
+    }
+
+    // ================= main phases
+    PipeState ps;
+    if (alive) {
+        if (p.mode == kModeSerial) {
+            dispatch_phase(p, S);
+            alive = grid_barrier(p, S, 2u * n_sm, 2);
+            if (alive) gemm_phase(p, S, stages, tmem_base, &tm_xe, &tm_wgu, &tm_h, &tm_wd, 0x7fffffff, ps);
+            alive = alive && grid_barrier(p, S, 3u * n_sm, 3);
+            if (alive) combine_phase(p, S);
+        } else {
+            const bool mover = (int)blockIdx.x < plan_c;      // role from c* and the block index
+            if (mover) dispatch_phase(p, S);
+            const int budget = mover ? plan_steal : 0x7fffffff;
+            if (budget > 0) gemm_phase(p, S, stages, tmem_base, &tm_xe, &tm_wgu, &tm_h, &tm_wd, budget, ps);
+            combine_phase(p, S);
+        }
+    }
+
+    // ================= leave: free TMEM; the last CTA out re-zeroes the control words
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+    if (tid == 0) {
+        __threadfence();
+        S.bcast[0] = atom_acqrel_add_u32(&p.ctl->exit_count, 1u) == (unsigned)(n_sm - 1) ? 1 : 0;
+    }
+    __syncthreads();
+    if (S.bcast[0]) {
+        for (int i = tid; i < kFine * kMaxEE; i += kThreads) p.fcnt[i] = 0u;
+        for (int i = tid; i < p.nmb_max; i += kThreads) { p.xe_ready[i] = 0u; p.h_ready[i] = 0u; }
+        unsigned *z = reinterpret_cast<unsigned *>(p.ctl);
+        if (tid < kCtlZeroWords) z[tid] = 0u;
+    }
+}
+
+}  // namespace weave

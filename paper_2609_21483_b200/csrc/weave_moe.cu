@@ -1,0 +1,448 @@
+// Host side of the C ABI declared in include/weave_moe.h: argument checks, workspace layout,
+// TMA descriptor encoding, the single cooperative launch per layer, and the small query calls.
+// No device memory is allocated here; everything lives in the caller's workspace.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/weave_moe.h"
+#include "weave_kernel.cuh"
+
+using namespace weave;
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Layout {
+    size_t ctl, fcnt, xe_ready, h_ready, zero_end;       // [0, zero_end) is zeroed at create / recovery
+    size_t hist, topk, gates, row_of, token_of, counts, offsets, bw, tf;
+    size_t xe, hbuf, y, st_x, st_logits, st_out, total;
+    int nmb_max, nblk_max, p_max;
+};
+
+bool shape_ok(const weave_moe_config *c)
+{
+    if (!c) return false;
+    if (c->hidden < 128 || c->hidden % 128 || c->ffn < 128 || c->ffn % 128) return false;
+    if (c->num_experts < 1 || c->num_shared < 0 || c->num_experts + c->num_shared > kMaxEE) return false;
+    if (c->top_k < 1 || c->top_k > c->num_experts || c->top_k > kMaxTopK || c->num_shared > 8) return false;
+    if (c->max_tokens < 1 || c->max_tokens > (1 << 20)) return false;
+    // row and weight-row coordinates of the TMA descriptors are 32-bit
+    const long long rows_w = (long long)(c->num_experts + c->num_shared) * 2 * c->ffn;
+    const long long rows_d = (long long)(c->num_experts + c->num_shared) * c->hidden;
+    const long long p_max = (long long)c->max_tokens * (c->top_k + c->num_shared);
+    if (rows_w >= (1ll << 31) || rows_d >= (1ll << 31) || p_max >= (1ll << 30)) return false;
+    return true;
+}
+
+Layout make_layout(const weave_moe_config *c)
+{
+    Layout L{};
+    const int EE = c->num_experts + c->num_shared;
+    const int ks = c->top_k + c->num_shared;
+    const size_t T = (size_t)c->max_tokens;
+    L.p_max = (int)(T * ks);
+    L.nblk_max = (int)((T + kRouteBlock - 1) / kRouteBlock);
+    L.nmb_max = (L.p_max + kBM - 1) / kBM + EE * kFine;
+    size_t o = 0;
+    auto take = [&](size_t bytes, size_t al) { o = align_up(o, al); size_t r = o; o += bytes; return r; };
+    L.ctl = take(sizeof(Ctl), 256);
+    L.fcnt = take(sizeof(unsigned) * kFine * kMaxEE, 256);
+    L.xe_ready = take(sizeof(unsigned) * L.nmb_max, 256);
+    L.h_ready = take(sizeof(unsigned) * L.nmb_max, 256);
+    L.zero_end = align_up(o, 256);
+    L.hist = take(sizeof(int) * (size_t)L.nblk_max * kMaxEE, 256);
+    L.topk = take(sizeof(int) * T * c->top_k, 256);
+    L.gates = take(sizeof(float) * T * c->top_k, 256);
+    L.row_of = take(sizeof(int) * T * c->top_k, 256);
+    L.token_of = take(sizeof(int) * (size_t)L.p_max, 256);
+    L.counts = take(sizeof(int) * EE, 256);
+    L.offsets = take(sizeof(int) * (EE + 1), 256);
+    L.bw = take(sizeof(float) * 1024, 256);
+    L.tf = take(sizeof(float) * 1024, 256);
+    L.xe = take((size_t)L.p_max * c->hidden * 2, 1024);
+    L.hbuf = take((size_t)L.p_max * c->ffn * 2, 1024);
+    L.y = take((size_t)L.p_max * c->hidden * 2, 1024);
+    L.st_x = take(T * c->hidden * 2, 1024);
+    L.st_logits = take(T * c->num_experts * 4, 1024);
+    L.st_out = take(T * c->hidden * 2, 1024);
+    L.total = align_up(o, 1024);
+    return L;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+}  // namespace
+
+struct weave_moe {
+    weave_moe_config cfg;
+    Layout L;
+    uint8_t *ws;
+    int n_sm;
+    int device;
+    int mode, fixed_c, fixed_K, fixed_steal;
+    int c_min, c_max, c_step;
+    float alpha, eff[4];
+    int timeout_ms;
+    int withhold_mb;
+    int last_T;
+    cudaStream_t last_stream;
+    int last_cuda_error;
+    CUtensorMap tm_xe, tm_wgu, tm_h, tm_wd;
+};
+
+namespace {
+
+int cuda_fail(weave_moe *h, cudaError_t e)
+{
+    if (h) h->last_cuda_error = (int)e;
+    return WEAVE_ERR_CUDA;
+}
+
+// bf16 matrix [rows][cols] row-major, box = 64 columns (128 bytes) x 128 rows, 128-byte swizzle
+int encode_map(EncodeTiledFn fn, CUtensorMap *m, const void *base, uint64_t rows, uint64_t cols, bool weights)
+{
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {cols * 2};
+    cuuint32_t box[2] = {kBK, kBM};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    weights ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? 0 : (int)r;
+}
+
+void default_tables(int n_sm, std::vector<float> &bw, std::vector<float> &tf)
+{
+    // Placeholder curves of the shape the paper's Figure 4 describes (bandwidth near-linear then
+    // saturating, GEMM throughput sub-linear); replaced by measured ones through
+    // weave_moe_set_cost_tables().  Units: byte/us and FLOP/us.
+    bw.assign(n_sm + 1, 0.f);
+    tf.assign(n_sm + 1, 0.f);
+    for (int i = 1; i <= n_sm; ++i) {
+        float lin = 45.0e3f * i;                       // ~45 GB/s per movement SM
+        bw[i] = lin < 5.5e6f ? lin : 5.5e6f;           // saturates near 5.5 TB/s
+        float x = (float)i / (float)n_sm;
+        tf[i] = 1.30e9f * x * (1.15f - 0.15f * x);     // ~1.3 PFLOP/s with all SMs, mildly sub-linear
+    }
+    bw[0] = bw[1];
+    tf[0] = tf[1];
+}
+
+int upload_tables(weave_moe *h, const float *bw, const float *tf)
+{
+    cudaError_t e = cudaMemcpy(h->ws + h->L.bw, bw, sizeof(float) * (h->n_sm + 1), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    e = cudaMemcpy(h->ws + h->L.tf, tf, sizeof(float) * (h->n_sm + 1), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    return WEAVE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t weave_moe_workspace_bytes(const weave_moe_config *cfg)
+{
+    if (!shape_ok(cfg)) return 0;
+    return make_layout(cfg).total;
+}
+
+int weave_moe_create(const weave_moe_config *cfg, weave_moe_t *out)
+{
+    if (!out) return WEAVE_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!shape_ok(cfg)) return WEAVE_ERR_INVALID_ARG;
+    if (!cfg->gate_up || !cfg->down || !cfg->workspace) return WEAVE_ERR_INVALID_ARG;
+    if (((uintptr_t)cfg->gate_up & 15) || ((uintptr_t)cfg->down & 15) || ((uintptr_t)cfg->workspace & 1023))
+        return WEAVE_ERR_INVALID_ARG;
+    Layout L = make_layout(cfg);
+    if (cfg->workspace_bytes < L.total) return WEAVE_ERR_WORKSPACE;
+
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return WEAVE_ERR_CUDA;
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, dev);
+    if (e != cudaSuccess) return WEAVE_ERR_CUDA;
+    if (prop.major != 10 || !prop.cooperativeLaunch) return WEAVE_ERR_UNSUPPORTED_DEVICE;
+    if ((int)prop.sharedMemPerBlockOptin < kSmemBytes) return WEAVE_ERR_UNSUPPORTED_DEVICE;
+    if (prop.multiProcessorCount + 1 > 1024) return WEAVE_ERR_UNSUPPORTED_DEVICE;
+
+    weave_moe *h = new (std::nothrow) weave_moe();
+    if (!h) return WEAVE_ERR_INVALID_ARG;
+    h->cfg = *cfg;
+    h->L = L;
+    h->ws = static_cast<uint8_t *>(cfg->workspace);
+    h->n_sm = prop.multiProcessorCount;
+    h->device = dev;
+    h->mode = WEAVE_SCHED_AUTO;
+    h->fixed_c = h->n_sm * 15 / 100;
+    h->fixed_K = 1;
+    h->fixed_steal = 0;
+    h->c_min = 2;
+    h->c_max = h->n_sm / 2;
+    h->c_step = 2;
+    h->alpha = 0.5f;
+    h->eff[0] = 1.0f; h->eff[1] = 0.93f; h->eff[2] = 0.85f; h->eff[3] = 0.73f;
+    h->timeout_ms = 4000;
+    h->withhold_mb = -1;
+    h->last_T = 0;
+    h->last_stream = nullptr;
+    h->last_cuda_error = 0;
+
+    e = cudaFuncSetAttribute(weave_moe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    if (e != cudaSuccess) { int rc = cuda_fail(h, e); delete h; return rc; }
+    int occ = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, weave_moe_kernel, kThreads, kSmemBytes);
+    if (e != cudaSuccess || occ < 1) { delete h; return WEAVE_ERR_UNSUPPORTED_DEVICE; }
+
+    void *fnp = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fnp, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || !fnp || qres != cudaDriverEntryPointSuccess) { delete h; return WEAVE_ERR_UNSUPPORTED_DEVICE; }
+    EncodeTiledFn enc = reinterpret_cast<EncodeTiledFn>(fnp);
+    const int EE = cfg->num_experts + cfg->num_shared;
+    int r = 0;
+    r |= encode_map(enc, &h->tm_xe, h->ws + L.xe, (uint64_t)L.p_max, (uint64_t)cfg->hidden, false);
+    r |= encode_map(enc, &h->tm_wgu, cfg->gate_up, (uint64_t)EE * 2 * cfg->ffn, (uint64_t)cfg->hidden, true);
+    r |= encode_map(enc, &h->tm_h, h->ws + L.hbuf, (uint64_t)L.p_max, (uint64_t)cfg->ffn, false);
+    r |= encode_map(enc, &h->tm_wd, cfg->down, (uint64_t)EE * cfg->hidden, (uint64_t)cfg->ffn, true);
+    if (r) { h->last_cuda_error = r; delete h; return WEAVE_ERR_CUDA; }
+
+    e = cudaMemset(h->ws, 0, L.zero_end);
+    if (e != cudaSuccess) { int rc = cuda_fail(h, e); delete h; return rc; }
+    std::vector<float> bw, tf;
+    default_tables(h->n_sm, bw, tf);
+    int rc = upload_tables(h, bw.data(), tf.data());
+    if (rc) { delete h; return rc; }
+    e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) { rc = cuda_fail(h, e); delete h; return rc; }
+    *out = h;
+    return WEAVE_OK;
+}
+
+int weave_moe_forward(weave_moe_t h, const void *x, const float *logits, void *out, int T, void *stream)
+{
+    if (!h) return WEAVE_ERR_INVALID_ARG;
+    if (T < 0 || T > h->cfg.max_tokens) return WEAVE_ERR_INVALID_ARG;
+    if (T == 0) return WEAVE_OK;
+    if (!x || !logits || !out) return WEAVE_ERR_INVALID_ARG;
+    if (((uintptr_t)x & 15) || ((uintptr_t)logits & 15) || ((uintptr_t)out & 15)) return WEAVE_ERR_INVALID_ARG;
+
+    const weave_moe_config &c = h->cfg;
+    const Layout &L = h->L;
+    KParams p;
+    memset(&p, 0, sizeof(p));
+    p.T = T; p.H = c.hidden; p.I = c.ffn; p.E = c.num_experts; p.S = c.num_shared; p.k = c.top_k;
+    p.EE = c.num_experts + c.num_shared;
+    p.nblk = (T + kRouteBlock - 1) / kRouteBlock;
+    p.mode = h->mode; p.fixed_c = h->fixed_c; p.fixed_K = h->fixed_K; p.fixed_steal = h->fixed_steal;
+    p.bn1 = (c.hidden % 256 == 0) ? 256 : 128;
+    p.nt0 = c.ffn / kTN0;
+    p.nt1 = c.hidden / p.bn1;
+    p.nmb_max = L.nmb_max;
+    p.withhold_mb = h->withhold_mb;
+    p.c_min = h->c_min; p.c_max = h->c_max; p.c_step = h->c_step;
+    p.alpha = h->alpha;
+    for (int i = 0; i < 4; ++i) p.eff[i] = h->eff[i];
+    p.timeout_ns = (unsigned long long)h->timeout_ms * 1000000ull;
+    p.x = static_cast<const __nv_bfloat16 *>(x);
+    p.logits = logits;
+    p.out = static_cast<__nv_bfloat16 *>(out);
+    uint8_t *ws = h->ws;
+    p.ctl = reinterpret_cast<Ctl *>(ws + L.ctl);
+    p.fcnt = reinterpret_cast<unsigned *>(ws + L.fcnt);
+    p.hist = reinterpret_cast<int *>(ws + L.hist);
+    p.topk_idx = reinterpret_cast<int *>(ws + L.topk);
+    p.gates = reinterpret_cast<float *>(ws + L.gates);
+    p.row_of = reinterpret_cast<int *>(ws + L.row_of);
+    p.token_of = reinterpret_cast<int *>(ws + L.token_of);
+    p.counts = reinterpret_cast<int *>(ws + L.counts);
+    p.offsets = reinterpret_cast<int *>(ws + L.offsets);
+    p.xe = reinterpret_cast<__nv_bfloat16 *>(ws + L.xe);
+    p.hbuf = reinterpret_cast<__nv_bfloat16 *>(ws + L.hbuf);
+    p.y = reinterpret_cast<__nv_bfloat16 *>(ws + L.y);
+    p.xe_ready = reinterpret_cast<unsigned *>(ws + L.xe_ready);
+    p.h_ready = reinterpret_cast<unsigned *>(ws + L.h_ready);
+    p.bw = reinterpret_cast<const float *>(ws + L.bw);
+    p.tf = reinterpret_cast<const float *>(ws + L.tf);
+
+    void *args[] = {&p, &h->tm_xe, &h->tm_wgu, &h->tm_h, &h->tm_wd};
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaLaunchCooperativeKernel((const void *)weave_moe_kernel, dim3(h->n_sm), dim3(kThreads), args,
+                                                (size_t)kSmemBytes, st);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    h->last_T = T;
+    h->last_stream = st;
+    return WEAVE_OK;
+}
+
+int weave_moe_forward_host(weave_moe_t h, const void *x_host, const float *logits_host, void *out_host, int T,
+                           void *stream)
+{
+    if (!h) return WEAVE_ERR_INVALID_ARG;
+    if (T < 0 || T > h->cfg.max_tokens) return WEAVE_ERR_INVALID_ARG;
+    if (T == 0) return WEAVE_OK;
+    if (!x_host || !logits_host || !out_host) return WEAVE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const weave_moe_config &c = h->cfg;
+    uint8_t *ws = h->ws;
+    const size_t xb = (size_t)T * c.hidden * 2, lb = (size_t)T * c.num_experts * 4;
+    cudaError_t e = cudaMemcpyAsync(ws + h->L.st_x, x_host, xb, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    e = cudaMemcpyAsync(ws + h->L.st_logits, logits_host, lb, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    int rc = weave_moe_forward(h, ws + h->L.st_x, reinterpret_cast<const float *>(ws + h->L.st_logits),
+                               ws + h->L.st_out, T, stream);
+    if (rc) return rc;
+    e = cudaMemcpyAsync(out_host, ws + h->L.st_out, xb, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    return WEAVE_OK;
+}
+
+int weave_moe_destroy(weave_moe_t h)
+{
+    delete h;
+    return WEAVE_OK;
+}
+
+int weave_moe_set_schedule(weave_moe_t h, int mode, int c, int K, int steal)
+{
+    if (!h || mode < WEAVE_SCHED_AUTO || mode > WEAVE_SCHED_SERIAL) return WEAVE_ERR_INVALID_ARG;
+    if (mode == WEAVE_SCHED_FIXED) {
+        if (c < 1 || (K != 1 && K != 2 && K != 4 && K != 8) || steal < 0) return WEAVE_ERR_INVALID_ARG;
+        h->fixed_c = c; h->fixed_K = K; h->fixed_steal = steal;
+    }
+    h->mode = mode;
+    return WEAVE_OK;
+}
+
+int weave_moe_set_cost_tables(weave_moe_t h, const float *bw, const float *tflops, const float *eff_chunk,
+                              float alpha, int c_min, int c_max, int c_step)
+{
+    if (!h || !bw || !tflops || !eff_chunk) return WEAVE_ERR_INVALID_ARG;
+    if (!(alpha >= 0.f && alpha < 1.f) || c_min < 1 || c_step < 1 || c_max < c_min) return WEAVE_ERR_INVALID_ARG;
+    if ((c_max - c_min) / c_step + 1 > 64) return WEAVE_ERR_INVALID_ARG;
+    for (int i = 1; i <= h->n_sm; ++i)
+        if (!(bw[i] > 0.f) || !(tflops[i] > 0.f)) return WEAVE_ERR_INVALID_ARG;
+    for (int i = 0; i < 4; ++i)
+        if (!(eff_chunk[i] > 0.f && eff_chunk[i] <= 1.f)) return WEAVE_ERR_INVALID_ARG;
+    if (h->last_stream || h->last_T) cudaStreamSynchronize(h->last_stream);
+    int rc = upload_tables(h, bw, tflops);
+    if (rc) return rc;
+    for (int i = 0; i < 4; ++i) h->eff[i] = eff_chunk[i];
+    h->alpha = alpha; h->c_min = c_min; h->c_max = c_max; h->c_step = c_step;
+    return WEAVE_OK;
+}
+
+int weave_moe_get_plan(weave_moe_t h, int *c, int *K, int *n_steal, float *t_total_us)
+{
+    if (!h) return WEAVE_ERR_INVALID_ARG;
+    cudaError_t e = cudaStreamSynchronize(h->last_stream);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    Ctl ctl;
+    e = cudaMemcpy(&ctl, h->ws + h->L.ctl, sizeof(Ctl), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    if (c) *c = ctl.plan_c;
+    if (K) *K = ctl.plan_K;
+    if (n_steal) *n_steal = ctl.plan_steal;
+    if (t_total_us) *t_total_us = ctl.plan_t;
+    return WEAVE_OK;
+}
+
+int weave_moe_get_geometry(weave_moe_t h, int *n_sm, int *block_m, int *tile_n0, int *tile_n1, int *route_block,
+                           int *combine_tile)
+{
+    if (!h) return WEAVE_ERR_INVALID_ARG;
+    if (n_sm) *n_sm = h->n_sm;
+    if (block_m) *block_m = kBM;
+    if (tile_n0) *tile_n0 = kTN0;
+    if (tile_n1) *tile_n1 = (h->cfg.hidden % 256 == 0) ? 256 : 128;
+    if (route_block) *route_block = kRouteBlock;
+    if (combine_tile) *combine_tile = kCombTile;
+    return WEAVE_OK;
+}
+
+int weave_moe_get_routing(weave_moe_t h, const int32_t **topk_idx, const float **gates, const int32_t **counts,
+                          const int32_t **offsets, const int32_t **row_of, const int32_t **token_of)
+{
+    if (!h) return WEAVE_ERR_INVALID_ARG;
+    const Layout &L = h->L;
+    if (topk_idx) *topk_idx = reinterpret_cast<const int32_t *>(h->ws + L.topk);
+    if (gates) *gates = reinterpret_cast<const float *>(h->ws + L.gates);
+    if (counts) *counts = reinterpret_cast<const int32_t *>(h->ws + L.counts);
+    if (offsets) *offsets = reinterpret_cast<const int32_t *>(h->ws + L.offsets);
+    if (row_of) *row_of = reinterpret_cast<const int32_t *>(h->ws + L.row_of);
+    if (token_of) *token_of = reinterpret_cast<const int32_t *>(h->ws + L.token_of);
+    return WEAVE_OK;
+}
+
+int weave_moe_get_intermediates(weave_moe_t h, const void **xe, const void **hbuf, const void **y)
+{
+    if (!h) return WEAVE_ERR_INVALID_ARG;
+    if (xe) *xe = h->ws + h->L.xe;
+    if (hbuf) *hbuf = h->ws + h->L.hbuf;
+    if (y) *y = h->ws + h->L.y;
+    return WEAVE_OK;
+}
+
+int weave_moe_status(weave_moe_t h)
+{
+    if (!h) return WEAVE_ERR_INVALID_ARG;
+    cudaError_t e = cudaStreamSynchronize(h->last_stream);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    Ctl ctl;
+    e = cudaMemcpy(&ctl, h->ws + h->L.ctl, sizeof(Ctl), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    int st = ctl.status;
+    if (st != 0) {
+        // a failed launch may have left flags behind: start from a clean slate
+        e = cudaMemset(h->ws, 0, h->L.zero_end);
+        if (e != cudaSuccess) return cuda_fail(h, e);
+        e = cudaDeviceSynchronize();
+        if (e != cudaSuccess) return cuda_fail(h, e);
+        h->last_cuda_error = ctl.timeout_where;   // where the first wait gave up (diagnostic)
+    }
+    return st;
+}
+
+int weave_moe_set_timeout_ms(weave_moe_t h, int ms)
+{
+    if (!h || ms < 1) return WEAVE_ERR_INVALID_ARG;
+    h->timeout_ms = ms;
+    return WEAVE_OK;
+}
+
+int weave_moe_debug_withhold_flag(weave_moe_t h, int m_block)
+{
+    if (!h) return WEAVE_ERR_INVALID_ARG;
+    h->withhold_mb = m_block;
+    return WEAVE_OK;
+}
+
+int weave_moe_last_cuda_error(weave_moe_t h) { return h ? h->last_cuda_error : 0; }
+
+const char *weave_moe_strerror(int code)
+{
+    switch (code) {
+        case WEAVE_OK: return "ok";
+        case WEAVE_ERR_INVALID_ARG: return "invalid argument";
+        case WEAVE_ERR_UNSUPPORTED_DEVICE: return "unsupported device (needs sm_100 with cooperative launch)";
+        case WEAVE_ERR_CUDA: return "CUDA call failed";
+        case WEAVE_ERR_WORKSPACE: return "workspace too small";
+        case WEAVE_ERR_NONFINITE_LOGITS: return "non-finite router logit";
+        case WEAVE_ERR_TIMEOUT: return "a bounded in-kernel wait expired";
+        default: return "unknown error";
+    }
+}
+
+}  // extern "C"
