@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Benchmark of the MoE-layer megakernel: layer latency, tokens/s, fraction of the layer roofline.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+A step is one pass of the whole hot path (routing, dispatch, grouped SwiGLU GEMMs, combine: one
+kernel launch per layer) over one batch of seeded synthetic input.  The default workload is the
+Mixtral-8x7B-shaped prefill layer (T=4096, H=4096, I=14336, E=8, top-2).  One JSON line is
+printed by rank 0.  With --gpus N > 1 (launched by torch.distributed.run) every rank runs an
+independent replica of the layer on its own GPU (the path has no cross-GPU exchange step on one
+node: "replicas only"); the value is the number of tokens all ranks processed divided by the
+slowest rank's device time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "moe_layer_tokens_per_s"
+UNIT = "tokens/s"
+DEFAULT_CONFIG = "c2_mixtral"
+
+
+def load_peaks():
+    """Measured roofline denominators of this machine's B200s, else the documented fallback."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    except Exception:
+        return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def layer_work(cfg, active_experts=None):
+    """Algorithmic FLOPs and bytes of one layer (per launch).
+    FLOPs = P * 6*H*I (Eq. 1).  Bytes = what the method itself moves, each intermediate written
+    once and read once: logits, routing, dispatch (T rows read, P written), gemm0 reads P rows and
+    the weights, h written and read, y written and read, out written."""
+    T, H, I, E, k, S = cfg.T, cfg.H, cfg.I, cfg.E, cfg.k, cfg.S
+    P = T * (k + S)
+    ea = (E + S) if active_experts is None else active_experts
+    flops = P * 6.0 * H * I
+    weights = ea * 3.0 * H * I * 2
+    act = (4.0 * T * E + 8.0 * T * k + (T + P) * 2.0 * H + P * 2.0 * H + 2 * P * 2.0 * I + 2 * P * 2.0 * H
+           + T * 2.0 * H)
+    return {"flops": flops, "bytes": weights + act, "weights_bytes": weights, "act_bytes": act,
+            "movement_bytes": (T + P) * 2.0 * H + (P + T) * 2.0 * H}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.idx}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons, pw = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            f = [s.strip() for s in r.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = [s for s, p in zip(sm, pw) if p > 0.5 * max(pw)] or sm
+        return {"sm_mhz": float(np.median(busy)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "power_w_max": float(max(pw)), "samples": len(sm)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def aggregate_max(value: float, world: int, use_cuda: bool) -> float:
+    """Max over ranks of a per-rank time (all-reduce MAX); identity for one process."""
+    if world <= 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device="cuda" if use_cuda else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_throughput(tokens_per_rank_step: int, steps: int, world: int, max_seconds: float) -> float:
+    return tokens_per_rank_step * steps * world / max_seconds
+
+
+# --------------------------------------------------------------------------------------- reference arm
+
+def run_reference(args):
+    """The reference arm of this tier is the CPU oracle as it stands, timed on the host cores on
+    a bounded token sample of the same workload (rank 0 only)."""
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    import oracle
+    import workloads as wl
+    cfg = wl.CONFIGS[args.config]
+    oracle.build(); wl.build()
+    inp = wl.make_inputs(cfg)
+    n = args.ref_tokens
+    toks = wl.stratified_token_sample(cfg.T, n, seed=cfg.cfg_id)
+    for _ in range(max(args.warmup, 0) and 1):
+        oracle.moe_tokens(inp.x, inp.logits, inp.gate_up, inp.down, cfg.k, toks[:1], cfg.S)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.routing(inp.logits, cfg.k, cfg.S)
+        oracle.moe_tokens(inp.x, inp.logits, inp.gate_up, inp.down, cfg.k, toks, cfg.S)
+    dt = time.perf_counter() - t0
+    val = len(toks) * args.steps / dt
+    cores = oracle.num_threads()
+    sample = (f"{len(toks)} stratified tokens of T={cfg.T} per step (full-T routing + per-token FFN/combine), "
+              f"{args.steps} steps, {dt:.1f} s")
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "I": cfg.I, "E": cfg.E, "top_k": cfg.k,
+                       "shared": cfg.S},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------- our arm
+
+def run_ours(args):
+    import torch
+    import workloads as wl
+    import paper_2609_21483_b200 as pk
+
+    rank, world, local = dist_env()
+    if args.gpus > 1 and world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} needs torch.distributed.run with {args.gpus} ranks (WORLD_SIZE={world})")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path (use --impl reference for the oracle)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    pk.load()
+
+    cfg = wl.CONFIGS[args.config]
+    wl.build()
+    as_bf16 = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)
+    gu_h, dn_h = wl.make_weights(cfg)
+    gu, dn = as_bf16(gu_h).cuda(), as_bf16(dn_h).cuda()
+    x_h = as_bf16(wl.make_x(cfg)).pin_memory()
+    x = x_h.cuda()
+    L = cfg.layers
+    logits_h = [torch.from_numpy(wl.make_logits(cfg, l)).pin_memory() for l in range(L)]
+    logits = [t.cuda() for t in logits_h]
+    out = torch.empty_like(x)
+    out_h = torch.empty_like(x_h).pin_memory()
+    moe = pk.WeaveMoE(gu, dn, cfg.E, cfg.k, cfg.S, max_tokens=cfg.T)
+    stream = torch.cuda.current_stream()
+    sched = {"auto": (pk.SCHED_AUTO, 0, 1, 0), "serial": (pk.SCHED_SERIAL, 0, 1, 0)}
+    geo = moe.geometry()
+    fixed_c = max(1, int(round(0.15 * geo["n_sm"])))
+    sched["fixed"] = (pk.SCHED_FIXED, fixed_c, 1, 0)
+
+    def step_dev():
+        for l in range(L):
+            moe.forward(x, logits[l], out)
+
+    def step_host():
+        for l in range(L):
+            moe.forward_host(x_h, logits_h[l], out_h)
+
+    def timed(fn, steps, warmup):
+        for _ in range(warmup):
+            fn()
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(stream)
+        for _ in range(steps):
+            fn()
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+        return ev0.elapsed_time(ev1) * 1e-3
+
+    moe.set_schedule(*sched[args.sched])
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    sec = timed(step_dev, args.steps, args.warmup)
+    moe.check()
+    plans = []
+    if rank == 0:
+        plans.append(moe.plan())
+    sec_max = aggregate_max(sec, world, True)
+    clocks = sampler.stop() if rank == 0 else None
+    sec_e2e = aggregate_max(timed(step_host, max(1, min(args.steps, 10)), 3), world, True)
+    e2e_steps = max(1, min(args.steps, 10))
+    moe.check()
+
+    ablation = {}
+    if rank == 0 and not args.no_ablation:
+        for name in ("auto", "fixed", "serial"):
+            moe.set_schedule(*sched[name])
+            s = timed(step_dev, max(3, min(args.steps, 10)), 3) if world == 1 else None
+            if s is not None:
+                ablation[name + "_us_per_layer"] = s / max(3, min(args.steps, 10)) / L * 1e6
+        moe.set_schedule(*sched[args.sched])
+        moe.check()
+
+    if rank != 0:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return
+
+    peaks = load_peaks()
+    work = layer_work(cfg)
+    layer_s = sec_max / args.steps / L
+    t_flops = work["flops"] / (peaks["bf16_tflops"] * 1e12)
+    t_bytes = work["bytes"] / (peaks["hbm_gbs"] * 1e9)
+    bound = "tensor" if t_flops >= t_bytes else "hbm"
+    if bound == "tensor":
+        achieved, peak, runit = work["flops"] / layer_s / 1e12, peaks["bf16_tflops"], "TFLOP/s"
+    else:
+        achieved, peak, runit = work["bytes"] / layer_s / 1e9, peaks["hbm_gbs"], "GB/s"
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(tpath):
+        try:
+            traffic = json.load(open(tpath)).get(cfg.name)
+        except Exception:
+            traffic = None
+
+    cpu_base = None
+    if not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        inp = wl.LayerInputs(cfg, wl.make_x(cfg), logits_h[0].numpy(), gu_h, dn_h)
+        n = args.ref_tokens
+        toks = wl.stratified_token_sample(cfg.T, n, seed=cfg.cfg_id)
+        t0 = time.perf_counter()
+        oracle.routing(inp.logits, cfg.k, cfg.S)
+        oracle.moe_tokens(inp.x, inp.logits, inp.gate_up, inp.down, cfg.k, toks, cfg.S)
+        dt = time.perf_counter() - t0
+        cpu_base = {"value": len(toks) / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                    "sample": f"{len(toks)} stratified tokens of T={cfg.T} (full-T routing + per-token FFN/combine) "
+                              f"in {dt:.1f} s"}
+
+    xb = cfg.T * cfg.H * 2
+    line = {
+        "metric": METRIC, "value": whole_job_throughput(cfg.T * L, args.steps, world, sec_max), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec_max / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "I": cfg.I, "E": cfg.E, "top_k": cfg.k,
+                   "shared": cfg.S, "layers": L, "sched": args.sched, "parallelism": f"replicas x{world}",
+                   "l2_policy": "inputs larger than L2 (weights %.2f GB streamed every step)" % (work["weights_bytes"] / 1e9)},
+        "layer_us": layer_s * 1e6,
+        "layer_roofline_us": max(t_flops, t_bytes) * 1e6,
+        "roofline": {"bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
+                     "traffic": traffic, "peak_source": peaks["source"] + " (burst)",
+                     "flops_per_launch": work["flops"], "bytes_per_launch": work["bytes"],
+                     "frac_of_sustained": (achieved / peaks["bf16_tflops_sustained"]) if bound == "tensor" else None},
+        "e2e": {"value": whole_job_throughput(cfg.T * L, e2e_steps, world, sec_e2e), "unit": UNIT,
+                "h2d_bytes_per_step": (xb + cfg.T * cfg.E * 4) * L, "d2h_bytes_per_step": xb * L},
+        "gpu_launches": args.steps * L,
+        "clocks": clocks,
+        "plan": plans[0] if plans else None,
+        "ablation": ablation,
+        "cpu_baseline": cpu_base,
+        "paper_context": "paper reports 2.89x geomean MoE-layer speedup over 5 systems on 4xH100 (EP=4); no 1-GPU or B200 number",
+    }
+    print(json.dumps(line), flush=True)
+    moe.close()
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default=DEFAULT_CONFIG)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--sched", default="auto", choices=["auto", "fixed", "serial"])
+    ap.add_argument("--ref-tokens", type=int, default=16, help="tokens in the CPU oracle's timed sample")
+    ap.add_argument("--no-ablation", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,332 @@
+"""GPU parity: the CUDA layer, called through its C ABI, against the CPU oracle on the same seeded
+inputs.  Routing, counts, offsets and permutation bit-exact; values within
+|gpu - ref| <= 2e-2 + 2e-2*|ref| and relative L2 <= 5e-3 (see tests/parity.py)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads as wl
+import paper_2609_21483_b200 as pk
+from parity import bf16_to_np, check_routing, check_values, oracle_rows, run_case, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _small(name, T, H, I, E, k, S=0, zipf=None, cfg_id=90):
+    return wl.MoEConfig(name, cfg_id, T=T, H=H, I=I, E=E, k=k, S=S, zipf_s=zipf)
+
+
+# ------------------------------------------------------------------ the configs of record
+
+def test_c1_tiny_every_schedule_matches_oracle_and_each_other():
+    """Config 1 in full under AUTO, SERIAL and forced (c, K, steal): the output must not depend on
+    the schedule (bitwise) and must match the oracle."""
+    cfg = wl.CONFIGS["c1_tiny"]
+    inp = wl.make_inputs(cfg)
+    dev = to_dev(inp)
+    moe, out0, l2 = run_case(cfg, inp=inp, dev_tensors=dev)
+    ref_bits = out0.view(torch.int16).clone()
+    scheds = [(pk.SCHED_SERIAL, 0, 1, 0)]
+    for c in (1, 20, 147):
+        for K in (1, 2, 4, 8):
+            for steal in (0, 2, 1 << 20):
+                scheds.append((pk.SCHED_FIXED, c, K, steal))
+    for s in scheds:
+        _, out, _ = run_case(cfg, sched=s, inp=inp, dev_tensors=dev, moe=moe)
+        assert torch.equal(out.view(torch.int16), ref_bits), f"schedule {s} changed the output bits"
+        if s[0] == pk.SCHED_FIXED:
+            p = moe.plan()
+            assert (p["c"], p["K"], p["n_steal"]) == (s[1], s[2], s[3])
+    moe.close()
+
+
+@pytest.mark.parametrize("name,n_sample", [("c4_dsv2lite_T64", None), ("c4_dsv2lite_T256", 48),
+                                           ("c4_dsv2lite_T1024", 32)])
+def test_c4_decode_like_with_shared_experts(name, n_sample):
+    cfg = wl.CONFIGS[name]
+    moe, _, _ = run_case(cfg, n_sample=n_sample)
+    moe.close()
+
+
+def test_c3_skewed_routing_sampled():
+    """Qwen3-30B-shaped, Zipf-biased: a few huge experts, many with < 128 rows, some empty."""
+    cfg = wl.CONFIGS["c3_qwen3_30b"]
+    inp = wl.make_inputs(cfg)
+    dev = to_dev(inp)
+    moe, out0, _ = run_case(cfg, n_sample=24, inp=inp, dev_tensors=dev)
+    bits = out0.view(torch.int16).clone()
+    for s in [(pk.SCHED_SERIAL, 0, 1, 0), (pk.SCHED_FIXED, 22, 1, 0), (pk.SCHED_FIXED, 30, 4, 5)]:
+        moe.set_schedule(*s)
+        out = moe.forward(dev[0], dev[1])
+        moe.check()
+        assert torch.equal(out.view(torch.int16), bits), f"schedule {s} changed the output bits"
+    moe.close()
+
+
+def test_c2_mixtral_shaped_sampled():
+    cfg = wl.CONFIGS["c2_mixtral"]
+    moe, _, _ = run_case(cfg, n_sample=12)
+    moe.close()
+
+
+def test_c5_qwen3_235b_shaped_two_layers_sampled():
+    """Two layers of the 24-layer stack (same weights, fresh skew per layer) on one handle."""
+    cfg = wl.CONFIGS["c5_qwen3_235b"]
+    weights = wl.make_weights(cfg)
+    moe = None
+    dev_w = None
+    plans = []
+    for layer in (0, 7):
+        inp = wl.make_inputs(cfg, layer, weights)
+        if dev_w is None:
+            dev = to_dev(inp)
+            dev_w = dev[2:]
+        else:
+            x = torch.from_numpy(inp.x.view(np.int16)).view(torch.bfloat16).cuda()
+            dev = (x, torch.from_numpy(inp.logits).cuda()) + dev_w
+        moe, _, _ = run_case(cfg, n_sample=6, inp=inp, dev_tensors=dev, moe=moe)
+        plans.append(moe.plan())
+    moe.close()
+
+
+# ------------------------------------------------------------------ edge cases
+
+@pytest.mark.parametrize("T", [1, 2, 63, 64, 65, 130, 257])
+def test_ragged_token_counts(T):
+    cfg = _small(f"ragged_T{T}", T, 256, 384, 8, 2)
+    moe, _, _ = run_case(cfg, max_tokens=300)
+    moe.close()
+
+
+@pytest.mark.parametrize("H,I,E,k,S", [
+    (128, 128, 1, 1, 0),      # one expert: a dense SwiGLU MLP, gate 1
+    (384, 256, 4, 4, 0),      # k = E, and H % 256 != 0 (128-wide gemm1 tiles)
+    (256, 128, 16, 16, 0),    # the largest k
+    (256, 256, 248, 8, 8),    # E + S = 256, the largest expert count; most experts empty or tiny
+    (512, 640, 5, 3, 1),      # odd expert count, one shared expert
+])
+def test_shape_edges(H, I, E, k, S):
+    cfg = _small(f"edge_{H}_{I}_{E}_{k}_{S}", 200, H, I, E, k, S)
+    moe, _, _ = run_case(cfg)
+    moe.close()
+
+
+def test_all_tokens_to_one_expert_and_ties():
+    """Degenerate routing: (a) every token picks experts 3 and 5 (two huge segments, the rest
+    empty); (b) all logits equal, so ties decide everything (indices 0..k-1)."""
+    cfg = _small("degenerate", 700, 256, 256, 8, 2)
+    inp = wl.make_inputs(cfg)
+    inp.logits[:] = -1.0
+    inp.logits[:, 3] = 2.0
+    inp.logits[:, 5] = 1.0
+    moe, _, _ = run_case(cfg, inp=inp)
+    r = moe.routing(cfg.T)
+    assert r["counts"].tolist() == [0, 0, 0, 700, 0, 700, 0, 0]
+    inp.logits[:] = 0.25
+    moe2, _, _ = run_case(cfg, inp=inp)
+    assert (moe2.routing(cfg.T)["topk_idx"].cpu().numpy() == np.array([0, 1])).all()
+    moe.close(); moe2.close()
+
+
+def test_signed_zero_logits_tie_to_lowest_index():
+    cfg = _small("zeros", 64, 128, 128, 4, 2)
+    inp = wl.make_inputs(cfg)
+    inp.logits[:] = -3.0
+    inp.logits[:, 2] = 0.0
+    inp.logits[:, 1] = -0.0
+    moe, _, _ = run_case(cfg, inp=inp)
+    assert (moe.routing(cfg.T)["topk_idx"].cpu().numpy() == np.array([1, 2])).all()
+    moe.close()
+
+
+def test_identity_like_experts_closed_form_on_gpu():
+    """Combine equals the gate-weighted sum: with up = identity, gate projection = beta on column
+    0, x[:,0] = 1 and down[e] = d_e * identity, out[t] = x[t] * silu(beta) * sum_j g[t,j] d_{e_j}."""
+    T, H, E, k = 300, 256, 8, 2
+    I = H
+    cfg = _small("identity", T, H, I, E, k)
+    inp = wl.make_inputs(cfg)
+    one = wl.f32_to_bf16_bits(np.array([1.0], np.float32))[0]
+    inp.x[:, 0] = one
+    gu = np.zeros((E, 2 * I, H), np.uint16)
+    gu[:, :I, 0] = one
+    gu[:, I + np.arange(I), np.arange(H)] = one
+    d = wl.f32_to_bf16_bits(np.linspace(0.5, 2.25, E).astype(np.float32))
+    dn = np.zeros((E, H, I), np.uint16)
+    for e in range(E):
+        dn[e, np.arange(H), np.arange(I)] = d[e]
+    inp.gate_up, inp.down = gu, dn
+    moe, out, _ = run_case(cfg, inp=inp)
+    r = moe.routing(T)
+    g = r["gates"].cpu().numpy().astype(np.float64)
+    idx = r["topk_idx"].cpu().numpy()
+    s = 1.0 / (1.0 + np.exp(-1.0))
+    w = (g * wl.bf16_bits_to_f32(d).astype(np.float64)[idx]).sum(1)
+    ref = wl.bf16_bits_to_f32(inp.x).astype(np.float64) * s * w[:, None]
+    check_values(bf16_to_np(out), ref.astype(np.float32), "identity closed form")
+    moe.close()
+
+
+def test_dispatch_is_inverse_permutation():
+    """Xe[row] == x[token_of[row]] bit for bit, and un-permuting Xe through row_of gives x back."""
+    cfg = wl.CONFIGS["c1_tiny"]
+    inp = wl.make_inputs(cfg)
+    dev = to_dev(inp)
+    moe, _, _ = run_case(cfg, inp=inp, dev_tensors=dev)
+    r, im = moe.routing(cfg.T), moe.intermediates(cfg.T)
+    xe = im["xe"].view(torch.int16)
+    x = dev[0].view(torch.int16)
+    assert torch.equal(xe, x[r["token_of"].long()])
+    for j in range(cfg.k):
+        assert torch.equal(xe[r["row_of"][:, j].long()], x)
+    moe.close()
+
+
+def test_handle_reuse_smaller_batches_and_run_to_run_bits():
+    cfg = _small("reuse", 512, 256, 384, 16, 4, zipf=1.0)
+    inp = wl.make_inputs(cfg)
+    x, lg, gu, dn = to_dev(inp)
+    moe = pk.WeaveMoE(gu, dn, cfg.E, cfg.k, cfg.S, max_tokens=512)
+    outs = []
+    for T in (512, 100, 512, 7, 512):
+        sub = wl.LayerInputs(wl.MoEConfig(cfg.name, cfg.cfg_id, T, cfg.H, cfg.I, cfg.E, cfg.k), inp.x[:T],
+                             inp.logits[:T], inp.gate_up, inp.down)
+        out = moe.forward(x[:T].contiguous(), lg[:T].contiguous())
+        moe.check()
+        check_routing(moe, sub)
+        check_values(bf16_to_np(out), oracle_rows(sub), f"T={T}")
+        if T == 512:
+            outs.append(out.view(torch.int16).clone())
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[1], outs[2])
+    moe.close()
+
+
+def test_forward_host_equals_forward():
+    cfg = wl.CONFIGS["c1_tiny"]
+    inp = wl.make_inputs(cfg)
+    x, lg, gu, dn = to_dev(inp)
+    moe = pk.WeaveMoE(gu, dn, cfg.E, cfg.k, cfg.S, max_tokens=cfg.T)
+    out = moe.forward(x, lg)
+    moe.check()
+    xh, lh = x.cpu().pin_memory(), lg.cpu().pin_memory()
+    oh = torch.empty_like(xh).pin_memory()
+    moe.forward_host(xh, lh, oh)
+    moe.check()
+    assert torch.equal(oh.view(torch.int16), out.cpu().view(torch.int16))
+    moe.close()
+
+
+# ------------------------------------------------------------------ cost model and scheduler
+
+def _n_tiles_of_K(counts_fine, geo, H, I):
+    """GEMM tiles of the layer for K = 1,2,4,8 from per-(fine chunk, expert) row counts."""
+    nt = I // geo["tile_n0"] + H // geo["tile_n1"]
+    res = []
+    for K in (1, 2, 4, 8):
+        g = 8 // K
+        mb = 0
+        for j in range(K):
+            rows = counts_fine[j * g:(j + 1) * g].sum(axis=0)
+            mb += int(((rows + geo["block_m"] - 1) // geo["block_m"]).sum())
+        res.append(mb * nt)
+    return res
+
+
+def _fine_counts(ref, cfg, geo):
+    nblk = (cfg.T + geo["route_block"] - 1) // geo["route_block"]
+    fine = np.zeros((8, cfg.E + cfg.S), np.int64)
+    for t in range(cfg.T):
+        f = ((t // geo["route_block"]) * 8) // nblk
+        for e in ref.idx[t]:
+            fine[f, e] += 1
+        for s in range(cfg.S):
+            fine[f, cfg.E + s] += 1
+    return fine
+
+
+@pytest.mark.parametrize("name", ["c1_tiny", "c4_dsv2lite_T256"])
+def test_device_plan_equals_cpu_cost_model(name):
+    """AUTO's (c*, K*, n_steal) must equal the CPU restatement of Eq. 1-16 fed the same tables."""
+    from oracle import cost_model as cm
+    cfg = wl.CONFIGS[name]
+    inp = wl.make_inputs(cfg)
+    x, lg, gu, dn = to_dev(inp)
+    moe = pk.WeaveMoE(gu, dn, cfg.E, cfg.k, cfg.S, max_tokens=cfg.T)
+    geo = moe.geometry()
+    N = geo["n_sm"]
+    ref = oracle.routing(inp.logits, cfg.k, cfg.S)
+    fine = _fine_counts(ref, cfg, geo)
+    nt = _n_tiles_of_K(fine, geo, cfg.H, cfg.I)
+    rng = np.random.default_rng(5)
+    for trial in range(6):
+        idx = np.arange(N + 1, dtype=np.float64)
+        b, f = 10 ** rng.uniform(3.5, 5.5), 10 ** rng.uniform(6, 7.5)
+        bw = (b * np.minimum(idx, rng.uniform(20, 148))).astype(np.float32)
+        tf = (f * idx ** rng.uniform(0.7, 1.0)).astype(np.float32)
+        bw[0], tf[0] = bw[1], tf[1]
+        eff = np.array([1.0, rng.uniform(.8, 1), rng.uniform(.6, .9), rng.uniform(.4, .8)], np.float32)
+        alpha = float(rng.uniform(0, 0.95))
+        tab = cm.CostTables(N, bw, tf, eff, alpha, c_min=2, c_max=N // 2, c_step=2)
+        want = cm.plan(tab, cfg.T, cfg.P, cfg.H, cfg.I, nt)
+        moe.set_cost_tables(bw, tf, eff, alpha, 2, N // 2, 2)
+        moe.set_schedule(pk.SCHED_AUTO)
+        moe.forward(x, lg)
+        moe.check()
+        got = moe.plan()
+        assert (got["c"], got["K"], got["n_steal"]) == (want.c, want.K, want.n_steal), (trial, got, want)
+        assert abs(got["t_total_us"] - want.t_total) <= 1e-6 * want.t_total
+    moe.close()
+
+
+# ------------------------------------------------------------------ failure reporting (no GPU fault)
+
+def test_nonfinite_logits_are_reported():
+    cfg = _small("nonfinite", 128, 128, 128, 8, 2)
+    inp = wl.make_inputs(cfg)
+    x, lg, gu, dn = to_dev(inp)
+    moe = pk.WeaveMoE(gu, dn, cfg.E, cfg.k, cfg.S, max_tokens=cfg.T)
+    bad = lg.clone()
+    bad[17, 3] = float("nan")
+    moe.forward(x, bad)
+    assert moe.status() == pk.ERR_NONFINITE_LOGITS
+    bad[17, 3] = float("-inf")
+    moe.forward(x, bad)
+    assert moe.status() == pk.ERR_NONFINITE_LOGITS
+    # the handle still works afterwards
+    run_case(cfg, inp=inp, dev_tensors=(x, lg, gu, dn), moe=moe)
+    moe.close()
+
+
+def test_bounded_wait_gives_up_and_handle_recovers():
+    """A producer that never publishes one ready flag: the consumer's wait runs out after the
+    configured limit, the kernel returns, the host reads WEAVE_ERR_TIMEOUT, and the next forward
+    on the same handle is correct again."""
+    cfg = wl.CONFIGS["c1_tiny"]
+    inp = wl.make_inputs(cfg)
+    dev = to_dev(inp)
+    moe = pk.WeaveMoE(dev[2], dev[3], cfg.E, cfg.k, cfg.S, max_tokens=cfg.T)
+    moe.set_timeout_ms(20)
+    moe.debug_withhold_flag(1)
+    moe.forward(dev[0], dev[1])
+    assert moe.status() == pk.ERR_TIMEOUT
+    moe.debug_withhold_flag(-1)
+    moe.set_timeout_ms(4000)
+    run_case(cfg, inp=inp, dev_tensors=dev, moe=moe)
+    moe.close()
+
+
+def test_argument_errors_at_the_boundary():
+    cfg = wl.CONFIGS["c1_tiny"]
+    inp = wl.make_inputs(cfg)
+    x, lg, gu, dn = to_dev(inp)
+    moe = pk.WeaveMoE(gu, dn, cfg.E, cfg.k, cfg.S, max_tokens=128)
+    with pytest.raises(pk.WeaveError):          # T > max_tokens
+        moe.forward(x, lg)
+    lib = pk.load()
+    assert lib.weave_moe_forward(moe._h, None, lg.data_ptr(), x.data_ptr(), 16, None) == -1
+    assert lib.weave_moe_forward(moe._h, x.data_ptr() + 2, lg.data_ptr(), x.data_ptr(), 16, None) == -1
+    assert lib.weave_moe_forward(moe._h, x.data_ptr(), lg.data_ptr(), x.data_ptr(), 0, None) == 0  # T=0 no-op
+    with pytest.raises(pk.WeaveError):
+        moe.set_schedule(pk.SCHED_FIXED, 10, 3, 0)   # K not in {1,2,4,8}
+    moe.close()
