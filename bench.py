@@ -76,7 +76,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.idx}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except Exception:
@@ -136,6 +136,16 @@ def whole_job_throughput(tokens_per_rank_step: int, steps: int, world: int, max_
     return tokens_per_rank_step * steps * world / max_seconds
 
 
+def cpu_sample_size(oracle, wl, inp, cfg, seconds: float) -> int:
+    """How many tokens the oracle gets through in about `seconds` on this host: time a probe of
+    8 tokens, scale, clamp to [8, T]."""
+    probe = wl.stratified_token_sample(cfg.T, 8, seed=99)
+    t0 = time.perf_counter()
+    oracle.moe_tokens(inp.x, inp.logits, inp.gate_up, inp.down, cfg.k, probe, cfg.S)
+    per_tok = max((time.perf_counter() - t0) / len(probe), 1e-6)
+    return int(min(cfg.T, max(8, seconds / per_tok)))
+
+
 # --------------------------------------------------------------------------------------- reference arm
 
 def run_reference(args):
@@ -149,7 +159,8 @@ def run_reference(args):
     cfg = wl.CONFIGS[args.config]
     oracle.build(); wl.build()
     inp = wl.make_inputs(cfg)
-    n = args.ref_tokens
+    n = args.ref_tokens if args.ref_tokens > 0 else cpu_sample_size(
+        oracle, wl, inp, cfg, max(2.0, min(args.cpu_seconds, 120.0 / max(args.steps + 1, 1))))
     toks = wl.stratified_token_sample(cfg.T, n, seed=cfg.cfg_id)
     for _ in range(max(args.warmup, 0) and 1):
         oracle.moe_tokens(inp.x, inp.logits, inp.gate_up, inp.down, cfg.k, toks[:1], cfg.S)
@@ -287,7 +298,7 @@ def run_ours(args):
         import oracle
         oracle.build()
         inp = wl.LayerInputs(cfg, wl.make_x(cfg), logits_h[0].numpy(), gu_h, dn_h)
-        n = args.ref_tokens
+        n = args.ref_tokens if args.ref_tokens > 0 else cpu_sample_size(oracle, wl, inp, cfg, args.cpu_seconds)
         toks = wl.stratified_token_sample(cfg.T, n, seed=cfg.cfg_id)
         t0 = time.perf_counter()
         oracle.routing(inp.logits, cfg.k, cfg.S)
@@ -334,7 +345,9 @@ def main():
     ap.add_argument("--config", default=DEFAULT_CONFIG)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--sched", default="auto", choices=["auto", "fixed", "serial"])
-    ap.add_argument("--ref-tokens", type=int, default=16, help="tokens in the CPU oracle's timed sample")
+    ap.add_argument("--ref-tokens", type=int, default=0,
+                    help="tokens in the CPU oracle's timed sample (0 = sized for --cpu-seconds of work)")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--no-ablation", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

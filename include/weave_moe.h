@@ -144,6 +144,15 @@ int weave_moe_set_timeout_ms(weave_moe_t h, int ms);
  * only; nothing faults or traps. */
 int weave_moe_debug_withhold_flag(weave_moe_t h, int m_block);
 
+/* Optional in-kernel timeline (our analogue of the utilisation profile of the paper's Section 5.4).
+ * buf: device memory of at least n_sm * events_per_cta * 16 bytes, caller-owned, or NULL to switch
+ * tracing off.  Each CTA writes up to events_per_cta - 1 records {start ns, end ns (low 32 bits of
+ * the global nanosecond timer), kind << 24 | id, extra} into its slice; the slice's last record
+ * holds the number written.  Kinds: 1 routing, 2 set-up, 3 permutation fix-up, 4 dispatch tile,
+ * 5 GEMM tile loads (extra = ns until its inputs were ready), 6 GEMM tile epilogue (id = m-block,
+ * extra = type << 16 | n-tile), 7 combine tile, 8 wait for a chunk's gemm1, 9 grid barrier. */
+int weave_moe_set_trace(weave_moe_t h, void *buf, int events_per_cta);
+
 int weave_moe_last_cuda_error(weave_moe_t h);
 const char *weave_moe_strerror(int code);
 

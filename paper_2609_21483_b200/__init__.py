@@ -58,7 +58,7 @@ EXPORTS = [
     "weave_moe_destroy", "weave_moe_set_schedule", "weave_moe_set_cost_tables", "weave_moe_get_plan",
     "weave_moe_get_geometry", "weave_moe_get_routing", "weave_moe_get_intermediates",
     "weave_moe_status", "weave_moe_set_timeout_ms", "weave_moe_debug_withhold_flag",
-    "weave_moe_last_cuda_error", "weave_moe_strerror",
+    "weave_moe_last_cuda_error", "weave_moe_strerror", "weave_moe_set_trace",
 ]
 
 
@@ -101,6 +101,8 @@ def load():
     lib.weave_moe_set_timeout_ms.argtypes = [vp, ci]
     lib.weave_moe_debug_withhold_flag.restype = ci
     lib.weave_moe_debug_withhold_flag.argtypes = [vp, ci]
+    lib.weave_moe_set_trace.restype = ci
+    lib.weave_moe_set_trace.argtypes = [vp, vp, ci]
     lib.weave_moe_last_cuda_error.restype = ci
     lib.weave_moe_last_cuda_error.argtypes = [vp]
     lib.weave_moe_strerror.restype = ctypes.c_char_p
@@ -272,3 +274,22 @@ class WeaveMoE:
 
     def debug_withhold_flag(self, m_block: int):
         _check(self._lib.weave_moe_debug_withhold_flag(self._h, m_block), "weave_moe_debug_withhold_flag")
+
+    # ---- timeline
+    def enable_trace(self, events_per_cta: int = 2048):
+        """Allocates the event buffer and switches the in-kernel timeline on (0 = off)."""
+        torch = self._torch
+        if events_per_cta <= 0:
+            _check(self._lib.weave_moe_set_trace(self._h, None, 0), "weave_moe_set_trace")
+            self._trace = None
+            return
+        n_sm = self.geometry()["n_sm"]
+        self._trace = torch.zeros(n_sm, events_per_cta, 4, dtype=torch.int32, device=self.gate_up.device)
+        _check(self._lib.weave_moe_set_trace(self._h, self._trace.data_ptr(), events_per_cta), "weave_moe_set_trace")
+
+    def read_trace(self):
+        """Events of the last forward: list (one per CTA) of arrays [n,4] = start, end, kind<<24|id, extra."""
+        import numpy as np
+        self._torch.cuda.synchronize()
+        raw = self._trace.cpu().numpy().view(np.uint32)
+        return [raw[c, :int(raw[c, -1, 0])] for c in range(raw.shape[0])]

@@ -36,6 +36,7 @@ constexpr int kMaxSeg = kFine * kMaxEE;
 constexpr int kTinfo = 4;        // tile-descriptor ring between the producer and its consumers
 constexpr int kTmemCols = 512;
 constexpr int kEpiWarps = 4;     // warps 4..7
+constexpr int kMGroup = 16;      // m-blocks whose A rows are kept L2-resident while all n-tiles pass
 
 constexpr int kErrNonFinite = -5;
 constexpr int kErrTimeout = -6;
@@ -94,6 +95,8 @@ struct KParams {
     unsigned *h_ready;    // [nmb_max] epilogue-warp arrivals of the m-block's gemm0 tiles; zero at entry
     const float *bw;      // [n_sm+1] byte/us
     const float *tf;      // [n_sm+1] FLOP/us
+    uint4 *trace;         // optional [n_sm][trace_cap] event records (nullptr = off)
+    int trace_cap;
 };
 
 struct TileInfo {
@@ -113,6 +116,7 @@ struct SmemTail {
     int scan_w[8];
     int scan_total;
     int c, K, steal, nmb, n_gemm, n_comb;
+    unsigned trace_n;
     int chunk_mb0[kFine + 1];
     int chunk_tile0[kFine + 1];
     int offsets[kMaxEE + 1];
@@ -133,6 +137,23 @@ __device__ __noinline__ void give_up(Ctl *ctl, int where)
 {
     if (atomicCAS(&ctl->status, 0, kErrTimeout) == 0) ctl->timeout_where = where;
     atomicExch(&ctl->abort, 1u);
+}
+
+// Optional timeline: one 16-byte record {start ns, end ns, kind<<24 | id, extra} per event, per CTA.
+enum { kEvRoute = 1, kEvSetup = 2, kEvFixup = 3, kEvDispatch = 4, kEvGemmLoad = 5, kEvGemmEpi = 6,
+       kEvCombine = 7, kEvWaitChunk = 8, kEvBarrier = 9, kEvDepWait = 10 };
+__device__ __forceinline__ void trace_ev(const KParams &p, SmemTail &S, int kind, unsigned id,
+                                         unsigned long long t0, unsigned long long t1, unsigned extra)
+{
+    if (p.trace == nullptr) return;
+    const unsigned i = atomicAdd(&S.trace_n, 1u);
+    if (i + 1u < (unsigned)p.trace_cap)
+        p.trace[(size_t)blockIdx.x * p.trace_cap + i] =
+            make_uint4((unsigned)t0, (unsigned)t1, ((unsigned)kind << 24) | (id & 0xFFFFFFu), extra);
+}
+__device__ __forceinline__ unsigned long long trace_now(const KParams &p)
+{
+    return p.trace ? globaltimer_ns() : 0ull;
 }
 
 // Every wait is bounded: it polls the global abort word and a wall-clock limit, and returns false
@@ -321,8 +342,8 @@ __device__ __forceinline__ void decode_mblock(const SmemTail &S, int EE, int mb,
 }
 
 // GEMM queue order (the chunk-pipeline DAG order): chunk by chunk; inside a chunk all gemm0 tiles,
-// then all gemm1 tiles; inside those expert-major, n-tile, m-block fastest (so consecutive tiles
-// share a weight panel in L2).
+// then all gemm1 tiles; inside those expert-major, then m-group, n-tile, m-block fastest (so
+// consecutive tiles share a weight panel, and a group's rows stay in L2 across the n-tiles).
 __device__ __forceinline__ void decode_gemm_tile(const SmemTail &S, const KParams &p, int g, TileInfo &ti)
 {
     int j = 0;
@@ -335,7 +356,12 @@ __device__ __forceinline__ void decode_gemm_tile(const SmemTail &S, const KParam
     const int s = seg_search(S, j * p.EE, (j + 1) * p.EE, cmb0, nt, local);
     const int mbs = S.seg_mb0[s + 1] - S.seg_mb0[s];
     const int within = local - (S.seg_mb0[s] - cmb0) * nt;
-    const int n = within / mbs, m = within - n * mbs;
+    // inside a segment: groups of kMGroup m-blocks; per group every n-tile, m-block fastest, so the
+    // group's A rows and the expert's weight panels are re-read from L2, not from HBM
+    const int gi = within / (kMGroup * nt);
+    const int wg = within - gi * kMGroup * nt;
+    const int gsize = min(kMGroup, mbs - gi * kMGroup);
+    const int n = wg / gsize, m = gi * kMGroup + (wg - n * gsize);
     ti.type = type;
     ti.mb = S.seg_mb0[s] + m;
     ti.row0 = S.seg_row0[s] + m * kBM;
@@ -364,6 +390,7 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S)
         if (mb >= S.nmb) break;
         int row0, nrows;
         decode_mblock(S, p.EE, mb, row0, nrows);
+        const unsigned long long tr0 = trace_now(p);
         for (int i = tid; i < nrows; i += kThreads) S.tok[i] = __ldcg(p.token_of + row0 + i);
         __syncthreads();
         const int total = nrows * n16;
@@ -393,6 +420,7 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S)
             __threadfence();
             st_release_u32(&p.xe_ready[mb], 1u);
         }
+        if (tid == 0) trace_ev(p, S, kEvDispatch, (unsigned)mb, tr0, trace_now(p), (unsigned)nrows);
     }
     __syncthreads();
 }
@@ -417,17 +445,20 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S)
         const int chunk = (((t0 / kRouteBlock) * kFine) / p.nblk) / g;
         if (chunk > ready_upto) {
             if (tid == 0) {
+                const unsigned long long tw0 = trace_now(p);
                 bool ok = flag_wait_ge(&p.ctl->fix_done, (unsigned)p.nblk, p, 20);
                 for (int j = ready_upto + 1; ok && j <= chunk; ++j) {
                     const unsigned target = (unsigned)((S.chunk_mb0[j + 1] - S.chunk_mb0[j]) * p.nt1 * kEpiWarps);
                     ok = flag_wait_ge(&p.ctl->y_done[j], target, p, 21);
                 }
                 S.bcast[1] = ok ? 1 : 0;
+                trace_ev(p, S, kEvWaitChunk, (unsigned)chunk, tw0, trace_now(p), 0u);
             }
             __syncthreads();
             if (!S.bcast[1]) break;
             ready_upto = chunk;
         }
+        const unsigned long long tc0 = trace_now(p);
         for (int tt = 0; tt < kCombTile / 8; ++tt) {
             const int t = t0 + warp * (kCombTile / 8) + tt;
             if (t >= p.T) break;                                   // warp-uniform
@@ -481,6 +512,7 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S)
             __syncwarp();
         }
         __syncthreads();
+        if (tid == 0) trace_ev(p, S, kEvCombine, (unsigned)q, tc0, trace_now(p), 0u);
     }
     __syncthreads();
 }
@@ -516,9 +548,13 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
         if (lane == 0) {
             int taken = 0;
             bool dead = false;
+            // the claim for the next tile is issued before this tile's loads, so the atomic's round
+            // trip to L2 is hidden behind them
+            int g_next = budget > 0 ? (int)atomicAdd(&p.ctl->q_gemm, 1u) : 0x7fffffff;
             while (!dead) {
                 TileInfo ti;
-                const int g = taken < budget ? (int)atomicAdd(&p.ctl->q_gemm, 1u) : 0x7fffffff;
+                const int g = g_next;
+                const unsigned long long tp0 = trace_now(p);
                 if (g >= S.n_gemm) ti.type = 2; else decode_gemm_tile(S, p, g, ti);
                 if (!mbar_wait(&S.ti_empty[ps.slot], ps.slot_phase ^ 1u, p, 30)) { dead = true; break; }
                 S.ti[ps.slot] = ti;
@@ -526,6 +562,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                 ps.next_slot();
                 if (ti.type == 2) break;
                 ++taken;
+                g_next = taken < budget ? (int)atomicAdd(&p.ctl->q_gemm, 1u) : 0x7fffffff;
                 const CUtensorMap *tma_a, *tma_b;
                 int brow0, brow1;
                 bool ok;
@@ -541,6 +578,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                     brow1 = brow0 + 128;
                 }
                 if (!ok) { dead = true; break; }
+                const unsigned long long tp1 = trace_now(p);
                 fence_proxy_async();     // rows written with ordinary stores elsewhere, read by TMA here
                 const bool two_b = (ti.type == 0) || (p.bn1 == 256);
                 const uint32_t tx = kStageA + (two_b ? kStageB : kStageB / 2);
@@ -554,6 +592,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                     if (two_b) tma_load_2d(sb + kStageB / 2, tma_b, kb * kBK, brow1, &S.full[ps.stage]);
                     ps.next_stage();
                 }
+                trace_ev(p, S, kEvGemmLoad, (unsigned)g, tp0, trace_now(p), (unsigned)(tp1 - tp0));
             }
             if (dead) {     // let loads already issued land before this CTA can leave
                 const unsigned long long t0 = globaltimer_ns();
@@ -614,6 +653,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
             dead = __any_sync(0xffffffffu, dead);
             if (dead) break;
             tc_fence_after();
+            const unsigned long long te0 = trace_now(p);
             const int r = q * 32 + lane;
             const bool valid = r < ti.nrows;
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)ps.acc * 256u;
@@ -663,6 +703,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                 mbar_arrive(&S.tmem_empty[ps.acc]);
                 __threadfence();
                 red_release_add_u32(ti.type == 0 ? &p.h_ready[ti.mb] : &p.ctl->y_done[ti.chunk], 1u);
+                if (q == 0) trace_ev(p, S, kEvGemmEpi, (unsigned)ti.mb, te0, trace_now(p), (unsigned)(ti.type << 16 | ti.n));
             }
             ps.next_acc();
         }
@@ -698,6 +739,8 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = S.tmem_base;
+    if (tid == 0) S.trace_n = 0u;
+    const unsigned long long tk0 = trace_now(p);
 
     // routing scratch lives in the (not yet used) stage buffers
     unsigned long long *r_mask = reinterpret_cast<unsigned long long *>(stages);          // [256]
@@ -731,7 +774,10 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
         }
         __syncthreads();
     }
+    const unsigned long long tk1 = trace_now(p);
     bool alive = grid_barrier(p, S, (unsigned)n_sm, 1);
+    const unsigned long long tk2 = trace_now(p);
+    if (tid == 0) { trace_ev(p, S, kEvRoute, 0u, tk0, tk1, 0u); trace_ev(p, S, kEvBarrier, 1u, tk1, tk2, 0u); }
 
     // ================= set-up: counts, offsets, plan, segment tables (identical on every CTA)
     int cf[kFine];
@@ -856,6 +902,8 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
     }
     __syncthreads();
 
+    const unsigned long long tk3 = trace_now(p);
+    if (tid == 0) trace_ev(p, S, kEvSetup, 0u, tk2, tk3, 0u);
     // ================= permutation fix-up: in-block rank + rows of earlier blocks + expert offset
     if (alive) {
         int fixed = 0;
@@ -894,6 +942,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
         }
     }
 
+    if (tid == 0) trace_ev(p, S, kEvFixup, 0u, tk3, trace_now(p), 0u);
     // ================= main phases
     PipeState ps;
     if (alive) {
@@ -918,6 +967,9 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
     tc_fence_after();
     if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
     if (tid == 0) {
+        if (p.trace)     // last record of the CTA's slice: how many events were written
+            p.trace[(size_t)blockIdx.x * p.trace_cap + p.trace_cap - 1] =
+                make_uint4(min(S.trace_n, (unsigned)p.trace_cap - 1u), 0u, 0u, 0u);
         __threadfence();
         S.bcast[0] = atom_acqrel_add_u32(&p.ctl->exit_count, 1u) == (unsigned)(n_sm - 1) ? 1 : 0;
     }

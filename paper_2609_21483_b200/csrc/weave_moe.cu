@@ -95,6 +95,8 @@ struct weave_moe {
     int last_T;
     cudaStream_t last_stream;
     int last_cuda_error;
+    void *trace;
+    int trace_cap;
     CUtensorMap tm_xe, tm_wgu, tm_h, tm_wd;
 };
 
@@ -198,6 +200,8 @@ int weave_moe_create(const weave_moe_config *cfg, weave_moe_t *out)
     h->last_T = 0;
     h->last_stream = nullptr;
     h->last_cuda_error = 0;
+    h->trace = nullptr;
+    h->trace_cap = 0;
 
     e = cudaFuncSetAttribute(weave_moe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) { int rc = cuda_fail(h, e); delete h; return rc; }
@@ -275,6 +279,8 @@ int weave_moe_forward(weave_moe_t h, const void *x, const float *logits, void *o
     p.h_ready = reinterpret_cast<unsigned *>(ws + L.h_ready);
     p.bw = reinterpret_cast<const float *>(ws + L.bw);
     p.tf = reinterpret_cast<const float *>(ws + L.tf);
+    p.trace = reinterpret_cast<uint4 *>(h->trace);
+    p.trace_cap = h->trace_cap;
 
     void *args[] = {&p, &h->tm_xe, &h->tm_wgu, &h->tm_h, &h->tm_wd};
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -426,6 +432,15 @@ int weave_moe_debug_withhold_flag(weave_moe_t h, int m_block)
 {
     if (!h) return WEAVE_ERR_INVALID_ARG;
     h->withhold_mb = m_block;
+    return WEAVE_OK;
+}
+
+int weave_moe_set_trace(weave_moe_t h, void *buf, int events_per_cta)
+{
+    if (!h) return WEAVE_ERR_INVALID_ARG;
+    if (buf && (events_per_cta < 2 || ((uintptr_t)buf & 15))) return WEAVE_ERR_INVALID_ARG;
+    h->trace = buf;
+    h->trace_cap = buf ? events_per_cta : 0;
     return WEAVE_OK;
 }
 
