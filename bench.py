@@ -31,6 +31,10 @@ METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
 DEFAULT_CONFIG = "c2_mixtral"
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the megakernel, from the ncu
+# captures summarised under profiles/ (one capture per workload; None = not captured)
+NCU_DRAM_BYTES_PER_LAUNCH = {"c2_mixtral": 3.842e9}
+
 
 def load_peaks():
     """Measured roofline denominators of this machine's B200s, else the documented fallback."""
@@ -285,13 +289,7 @@ def run_ours(args):
         achieved, peak, runit = work["flops"] / layer_s / 1e12, peaks["bf16_tflops"], "TFLOP/s"
     else:
         achieved, peak, runit = work["bytes"] / layer_s / 1e9, peaks["hbm_gbs"], "GB/s"
-    traffic = None
-    tpath = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tpath):
-        try:
-            traffic = json.load(open(tpath)).get(cfg.name)
-        except Exception:
-            traffic = None
+    traffic = NCU_DRAM_BYTES_PER_LAUNCH.get(cfg.name)
 
     cpu_base = None
     if not args.no_cpu_baseline:
