@@ -93,16 +93,17 @@ int weave_moe_destroy(weave_moe_t h);
 
 /* ---- scheduling surface (Section 3; ablation of Section 5.5) -------------------------------- */
 
-/* mode: WEAVE_SCHED_*.  For FIXED: c = number of movement SMs (clamped to [1, n_sm-1]), K = chunk
- * count in {1,2,4,8}, steal = GEMM tiles each movement SM takes after dispatch (Section 3.2.2).
- * Takes effect at the next forward. */
+/* mode: WEAVE_SCHED_*.  For FIXED: c = number of movement SMs (rounded up to whole SM pairs and
+ * clamped to [2, n_sm-2]), K = chunk count in {1,2,4,8} (lowered until K*(E+S) <= 1024), steal =
+ * GEMM tiles each movement SM pair takes after dispatch (Section 3.2.2).  Takes effect at the
+ * next forward. */
 int weave_moe_set_schedule(weave_moe_t h, int mode, int c, int K, int steal);
 
 /* Hardware input of the cost model (Figure 7): bw[i] = bytes/us moved by i movement SMs,
  * tflops[i] = FLOP/us of i GEMM SMs, i in [0, n_sm] (host arrays of n_sm+1 floats, entry 0
  * ignored); eff_chunk[4] = Eq. 9's correction factor for K = 1,2,4,8; alpha = Section 3.1's
  * overlap ratio in [0,1); candidate grid c = c_min, c_min+c_step, ... <= c_max (at most 64
- * values).  Synchronous copy to the device. */
+ * values; c_min and c_step even, c_min >= 2).  Synchronous copy to the device. */
 int weave_moe_set_cost_tables(weave_moe_t h, const float *bw, const float *tflops,
                               const float *eff_chunk, float alpha, int c_min, int c_max, int c_step);
 
@@ -110,11 +111,14 @@ int weave_moe_set_cost_tables(weave_moe_t h, const float *bw, const float *tflop
  * model's predicted layer time in us.  Synchronises the handle's last stream. */
 int weave_moe_get_plan(weave_moe_t h, int *c, int *K, int *n_steal, float *t_total_us);
 
-/* Geometry the scheduler works with: number of SMs (= persistent CTAs), rows per GEMM m-block,
- * h-columns per gemm0 tile, out-columns per gemm1 tile, tokens per routing block, tokens per
- * combine tile.  Any pointer may be NULL. */
+/* Geometry the scheduler works with: number of SMs used (= persistent CTAs; an even number,
+ * because the GEMM phase runs on pairs of neighbouring SMs), rows per m-block (the unit of the
+ * dispatch queue and of the ready flags), h-columns per gemm0 tile, out-columns per gemm1 tile,
+ * tokens per routing block, tokens per combine tile, rows per GEMM tile (two m-blocks of one
+ * expert segment; a segment with an odd number of m-blocks ends in a half-empty tile).
+ * Any pointer may be NULL. */
 int weave_moe_get_geometry(weave_moe_t h, int *n_sm, int *block_m, int *tile_n0, int *tile_n1,
-                           int *route_block, int *combine_tile);
+                           int *route_block, int *combine_tile, int *gemm_tile_m);
 
 /* ---- verification surface ------------------------------------------------------------------- */
 

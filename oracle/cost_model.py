@@ -41,6 +41,8 @@ class CostTables:
     c_min: int = 2
     c_max: int = 74
     c_step: int = 2
+    steal_workers: int = 0   # Eq. 14's N: workers that share W_steal (0 = n_sm; a build whose GEMM
+                             # worker is an SM pair passes n_sm // 2 and counts tiles per pair)
 
 
 @dataclass
@@ -91,7 +93,7 @@ def n_steal(tab: CostTables, c: int, w_comp, w_disp, w_comb, n_tiles: int) -> in
     w_tile = w_comp / f32(n_tiles)
     if not (w_tile > 0):
         return 0
-    ns = w_steal / (f32(tab.n_sm) * w_tile)                         # Eq. 14
+    ns = w_steal / (f32(tab.steal_workers or tab.n_sm) * w_tile)    # Eq. 14
     ns = int(np.floor(ns + f32(0.5)))
     return max(0, min(ns, n_tiles))
 

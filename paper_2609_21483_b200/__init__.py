@@ -90,7 +90,7 @@ def load():
     lib.weave_moe_get_plan.restype = ci
     lib.weave_moe_get_plan.argtypes = [vp, cip, cip, cip, cfp]
     lib.weave_moe_get_geometry.restype = ci
-    lib.weave_moe_get_geometry.argtypes = [vp, cip, cip, cip, cip, cip, cip]
+    lib.weave_moe_get_geometry.argtypes = [vp, cip, cip, cip, cip, cip, cip, cip]
     lib.weave_moe_get_routing.restype = ci
     lib.weave_moe_get_routing.argtypes = [vp, vpp, vpp, vpp, vpp, vpp, vpp]
     lib.weave_moe_get_intermediates.restype = ci
@@ -218,9 +218,9 @@ class WeaveMoE:
         return {"c": c.value, "K": K.value, "n_steal": s.value, "t_total_us": t.value}
 
     def geometry(self):
-        v = [ctypes.c_int() for _ in range(6)]
+        v = [ctypes.c_int() for _ in range(7)]
         _check(self._lib.weave_moe_get_geometry(self._h, *[ctypes.byref(a) for a in v]), "weave_moe_get_geometry")
-        names = ["n_sm", "block_m", "tile_n0", "tile_n1", "route_block", "combine_tile"]
+        names = ["n_sm", "block_m", "tile_n0", "tile_n1", "route_block", "combine_tile", "gemm_tile_m"]
         return {n: a.value for n, a in zip(names, v)}
 
     # ---- verification surface

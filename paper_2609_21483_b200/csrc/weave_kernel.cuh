@@ -5,8 +5,11 @@
 //   set-up   (every CTA, redundantly) counts, offsets, candidate tile counts, cost model -> plan
 //                         (c, K, n_steal), segment tables of the chosen K; permutation fix-up
 //   phase A  (movement CTAs: blockIdx < c)  dispatch tiles: gather x rows into expert-major Xe
-//   phase B  (GEMM CTAs until the queue is empty; movement CTAs for n_steal tiles)
-//                         warp-specialised TMA -> smem ring -> tcgen05.mma -> TMEM -> epilogue
+//   phase B  (GEMM CTA pairs until the queue is empty; movement pairs for n_steal tiles)
+//                         two neighbouring CTAs (a cluster of 2) share a 256-row tile: a scheduler
+//                         warp claims tiles and waits for their inputs, TMA producers feed a
+//                         6-stage smem ring, one thread issues tcgen05.mma.cta_group::2 into TMEM,
+//                         four epilogue warps per CTA drain it through a staged, coalesced store
 //   phase C  (every CTA once it has nothing else)  combine tiles, chunk by chunk as the chunk's
 //                         gemm1 tiles complete
 //
@@ -23,20 +26,21 @@ constexpr int kThreads = 256;
 constexpr int kBM = 128;        // rows per GEMM m-block (UMMA M)
 constexpr int kBK = 64;         // K elements per pipeline stage: 128 bytes of bf16 = one swizzle row
 constexpr int kTN0 = 128;       // h columns per gemm0 tile; the MMA is N = 256 (gate | up)
-constexpr int kStages = 4;
-constexpr int kStageA = kBM * kBK * 2;                  // 16 KB
-constexpr int kStageB = 256 * kBK * 2;                  // 32 KB
-constexpr int kStageBytes = kStageA + kStageB;          // 48 KB
+constexpr int kStages = 6;
+constexpr int kStageA = kBM * kBK * 2;                  // 16 KB: this CTA's 128 rows of A
+constexpr int kStageB = 128 * kBK * 2;                  // 16 KB: this CTA's half (128 rows) of the 256-row B tile
+constexpr int kStageBytes = kStageA + kStageB;          // 32 KB
+constexpr int kEpiStageBytes = 4 * 32 * 64;             // epilogue staging: per warp 32 rows x 64 bytes
 constexpr int kRouteBlock = 64;  // tokens per routing block (one 64-bit mask per expert)
 constexpr int kCombTile = 16;    // tokens per combine tile
 constexpr int kMaxEE = 256;      // routed + shared experts
 constexpr int kMaxTopK = 16;
 constexpr int kFine = 8;         // fine chunks = largest chunk count K
-constexpr int kMaxSeg = kFine * kMaxEE;
+constexpr int kMaxSeg = 1024;     // (chunk, expert) segments: K * (E+S) <= 1024 bounds the chunk count
 constexpr int kTinfo = 4;        // tile-descriptor ring between the producer and its consumers
 constexpr int kTmemCols = 512;
 constexpr int kEpiWarps = 4;     // warps 4..7
-constexpr int kMGroup = 16;      // m-blocks whose A rows are kept L2-resident while all n-tiles pass
+constexpr int kPairGroup = 8;    // 256-row pair tiles (= 16 m-blocks) kept L2-resident while all n-tiles pass
 
 constexpr int kErrNonFinite = -5;
 constexpr int kErrTimeout = -6;
@@ -68,8 +72,7 @@ struct KParams {
     int T, H, I, E, S, k, EE;
     int nblk;             // routing blocks = ceil(T / 64)
     int mode, fixed_c, fixed_K, fixed_steal;
-    int bn1;              // out columns per gemm1 tile: 256, or 128 when H % 256 != 0
-    int nt0, nt1;         // n-tiles per m-block: I / 128, H / bn1
+    int nt0, nt1;         // n-tiles per m-block: I / 128, ceil(H / 256)
     int nmb_max;          // allocated length of the per-m-block flag arrays
     int withhold_mb;      // test hook: this m-block's "dispatched" flag is never published (-1 = off)
     int c_min, c_max, c_step;
@@ -101,7 +104,10 @@ struct KParams {
 
 struct TileInfo {
     int type;   // 0 gemm0 (+SwiGLU), 1 gemm1, 2 no more tiles
-    int mb, row0, nrows, e, n, chunk, nkb;
+    int mb;     // this CTA's m-block (-1: the pair tile has no second half)
+    int row0;   // first row of this CTA's 128 rows of A
+    int nrows;  // valid rows (0 for a missing half)
+    int e, n, chunk, nkb;
 };
 
 struct SmemTail {
@@ -118,17 +124,19 @@ struct SmemTail {
     int c, K, steal, nmb, n_gemm, n_comb;
     unsigned trace_n;
     int chunk_mb0[kFine + 1];
+    int chunk_pt0[kFine + 1];
     int chunk_tile0[kFine + 1];
     int offsets[kMaxEE + 1];
     int tok[kBM];
     int crow[8][kMaxTopK + 8];
     float cgate[8][kMaxTopK + 8];
     int seg_mb0[kMaxSeg + 1];
+    int seg_pt0[kMaxSeg + 1];    // prefix of pair tiles: ceil(m-blocks / 2) per segment
     int seg_row0[kMaxSeg];
     int seg_rows[kMaxSeg];
 };
 
-constexpr int kSmemBytes = kStages * kStageBytes + (int)sizeof(SmemTail) + 1024;
+constexpr int kSmemBytes = kStages * kStageBytes + kEpiStageBytes + (int)sizeof(SmemTail) + 1024;
 static_assert(kSmemBytes <= 232448, "exceeds the 227 KB a CTA may opt into");
 
 // ------------------------------------------------------------------------------------ waits
@@ -316,7 +324,8 @@ __device__ __forceinline__ int model_n_steal(const KParams &p, int n_sm, int c, 
     const float w_steal = fmaxf(0.0f, __fsub_rn(w_comp, w_partial));
     const float w_tile = __fdiv_rn(w_comp, (float)n_tiles);
     if (!(w_tile > 0.0f)) return 0;
-    const float ns = __fdiv_rn(w_steal, __fmul_rn((float)n_sm, w_tile));
+    // a GEMM worker is a CTA pair: W_steal is shared by n_sm / 2 workers (Eq. 14's N)
+    const float ns = __fdiv_rn(w_steal, __fmul_rn((float)(n_sm / 2), w_tile));
     int r = (int)floorf(__fadd_rn(ns, 0.5f));
     return max(0, min(r, n_tiles));
 }
@@ -341,35 +350,52 @@ __device__ __forceinline__ void decode_mblock(const SmemTail &S, int EE, int mb,
     nrows = min(kBM, S.seg_rows[s] - m * kBM);
 }
 
+// largest s in [lo, hi) with (seg_pt0[s] - base) * mul <= key
+__device__ __forceinline__ int seg_search_pt(const SmemTail &S, int lo, int hi, int base, int mul, int key)
+{
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if ((S.seg_pt0[mid] - base) * mul <= key) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
 // GEMM queue order (the chunk-pipeline DAG order): chunk by chunk; inside a chunk all gemm0 tiles,
-// then all gemm1 tiles; inside those expert-major, then m-group, n-tile, m-block fastest (so
-// consecutive tiles share a weight panel, and a group's rows stay in L2 across the n-tiles).
-__device__ __forceinline__ void decode_gemm_tile(const SmemTail &S, const KParams &p, int g, TileInfo &ti)
+// then all gemm1 tiles; inside those expert-major, then groups of kPairGroup pair tiles, n-tile,
+// pair tile fastest (consecutive tiles share a weight panel, and a group's rows stay in L2 while
+// all its n-tiles pass).  A pair tile = two consecutive m-blocks of one segment: `lead` describes
+// the leader CTA's half, `peer` the other CTA's (nrows = 0, mb = -1 when the segment's m-block
+// count is odd and this is its last pair tile).
+__device__ __forceinline__ void decode_pair_tile(const SmemTail &S, const KParams &p, int g, TileInfo &lead,
+                                                 TileInfo &peer)
 {
     int j = 0;
     while (j + 1 < S.K && g >= S.chunk_tile0[j + 1]) ++j;
     int local = g - S.chunk_tile0[j];
-    const int cmb0 = S.chunk_mb0[j];
-    const int nmbj = S.chunk_mb0[j + 1] - cmb0;
+    const int cpt0 = S.chunk_pt0[j];
+    const int nptj = S.chunk_pt0[j + 1] - cpt0;
     int type = 0, nt = p.nt0;
-    if (local >= nmbj * p.nt0) { type = 1; local -= nmbj * p.nt0; nt = p.nt1; }
-    const int s = seg_search(S, j * p.EE, (j + 1) * p.EE, cmb0, nt, local);
-    const int mbs = S.seg_mb0[s + 1] - S.seg_mb0[s];
-    const int within = local - (S.seg_mb0[s] - cmb0) * nt;
-    // inside a segment: groups of kMGroup m-blocks; per group every n-tile, m-block fastest, so the
-    // group's A rows and the expert's weight panels are re-read from L2, not from HBM
-    const int gi = within / (kMGroup * nt);
-    const int wg = within - gi * kMGroup * nt;
-    const int gsize = min(kMGroup, mbs - gi * kMGroup);
-    const int n = wg / gsize, m = gi * kMGroup + (wg - n * gsize);
-    ti.type = type;
-    ti.mb = S.seg_mb0[s] + m;
-    ti.row0 = S.seg_row0[s] + m * kBM;
-    ti.nrows = min(kBM, S.seg_rows[s] - m * kBM);
-    ti.e = s - j * p.EE;
-    ti.n = n;
-    ti.chunk = j;
-    ti.nkb = (type == 0 ? p.H : p.I) / kBK;
+    if (local >= nptj * p.nt0) { type = 1; local -= nptj * p.nt0; nt = p.nt1; }
+    const int s = seg_search_pt(S, j * p.EE, (j + 1) * p.EE, cpt0, nt, local);
+    const int pts = S.seg_pt0[s + 1] - S.seg_pt0[s];
+    const int within = local - (S.seg_pt0[s] - cpt0) * nt;
+    const int gi = within / (kPairGroup * nt);
+    const int wg = within - gi * kPairGroup * nt;
+    const int gsize = min(kPairGroup, pts - gi * kPairGroup);
+    const int n = wg / gsize;
+    const int m0 = 2 * (gi * kPairGroup + (wg - n * gsize));
+    const int rows = S.seg_rows[s];
+    lead.type = peer.type = type;
+    lead.e = peer.e = s - j * p.EE;
+    lead.n = peer.n = n;
+    lead.chunk = peer.chunk = j;
+    lead.nkb = peer.nkb = (type == 0 ? p.H : p.I) / kBK;
+    lead.mb = S.seg_mb0[s] + m0;
+    lead.row0 = S.seg_row0[s] + m0 * kBM;
+    lead.nrows = min(kBM, rows - m0 * kBM);
+    peer.nrows = max(0, min(kBM, rows - (m0 + 1) * kBM));
+    peer.mb = peer.nrows > 0 ? lead.mb + 1 : -1;
+    peer.row0 = lead.row0 + kBM;
 }
 
 // ------------------------------------------------------------------------------------ phase A: dispatch
@@ -533,120 +559,184 @@ __device__ __forceinline__ float silu_mul(float g, float u)
     return __fdividef(g, 1.0f + __expf(-g)) * u;
 }
 
-// budget = how many tiles this CTA may claim (the steal count for a movement CTA).
+// bounded wait on a barrier whose guarded data may come from the peer CTA
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity, const KParams &p, int where)
+{
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    unsigned it = 0;
+    while (!mbar_try_wait_cluster(bar, parity)) {
+        if ((++it & 31u) == 0u) {
+            if (ld_relaxed_u32(&p.ctl->abort)) return false;
+            if (globaltimer_ns() - t0 > p.timeout_ns) {
+                give_up(p.ctl, where);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void linger_after_abort()
+{
+    // lets copies and MMAs that are already in flight land before this CTA can leave
+    const unsigned long long t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 50000ull) __nanosleep(1000);
+}
+
+// One warp's 32 rows x 32 columns of bf16 (16 packed words per thread, thread = row) go through a
+// 2 KB staging buffer so that every global store instruction writes 8 rows x 64 contiguous bytes.
+// 16-byte chunk j of row r sits at r*64 + ((j ^ ((r >> 1) & 3)) << 4): conflict-free both ways.
+__device__ __forceinline__ void staged_store_32x32(uint32_t stg, int lane, const uint32_t (&o)[16],
+                                                   __nv_bfloat16 *dst_row0, size_t ld, int rows_valid)
+{
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+        st_shared_v4(stg + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4),
+                     make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]));
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int row = i * 8 + (lane >> 2), ch = lane & 3;
+        const uint4 v = ld_shared_v4(stg + row * 64 + ((ch ^ ((row >> 1) & 3)) << 4));
+        if (row < rows_valid) st_v4(dst_row0 + (size_t)row * ld + ch * 8, v);
+    }
+    __syncwarp();
+}
+
+// budget = how many pair tiles this CTA pair may claim (the steal count for a movement pair).
+// Called by both CTAs of a pair with the same arguments.
 __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_t *stages, uint32_t tmem_base,
                                            const CUtensorMap *tm_xe, const CUtensorMap *tm_wgu,
                                            const CUtensorMap *tm_h, const CUtensorMap *tm_wd, int budget,
                                            PipeState &ps)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const uint32_t rank = cluster_ctarank();      // 0 = leader (issues the MMAs), 1 = peer
     fence_proxy_async();     // the stage buffers were last touched by ordinary stores (routing scratch)
     __syncthreads();
 
-    if (warp == 0) {
-        // ---------------- producer: claims tiles, waits for their inputs, feeds the smem ring by TMA
+    if (warp == 2 && rank == 0) {
+        // ---------------- scheduler (leader only): claims pair tiles in queue order, waits until their
+        // inputs are ready, then publishes the tile to both CTAs' descriptor rings.  Runs up to
+        // kTinfo tiles ahead of the MMAs, so claim and flag latencies stay off the critical path.
         if (lane == 0) {
             int taken = 0;
-            bool dead = false;
-            // the claim for the next tile is issued before this tile's loads, so the atomic's round
-            // trip to L2 is hidden behind them
             int g_next = budget > 0 ? (int)atomicAdd(&p.ctl->q_gemm, 1u) : 0x7fffffff;
-            while (!dead) {
-                TileInfo ti;
+            for (;;) {
                 const int g = g_next;
                 const unsigned long long tp0 = trace_now(p);
-                if (g >= S.n_gemm) ti.type = 2; else decode_gemm_tile(S, p, g, ti);
-                if (!mbar_wait(&S.ti_empty[ps.slot], ps.slot_phase ^ 1u, p, 30)) { dead = true; break; }
-                S.ti[ps.slot] = ti;
+                TileInfo tl, tp;
+                if (g >= S.n_gemm) { tl.type = tp.type = 2; tl.mb = tp.mb = -1; tl.nrows = tp.nrows = 0; }
+                else decode_pair_tile(S, p, g, tl, tp);
+                if (!mbar_wait(&S.ti_empty[ps.slot], ps.slot_phase ^ 1u, p, 30)) break;
+                S.ti[ps.slot] = tl;
+                {
+                    const uint32_t dst = mapa_u32(smem_u32(&S.ti[ps.slot]), 1u);
+                    const uint32_t *src = reinterpret_cast<const uint32_t *>(&tp);
+#pragma unroll
+                    for (int w = 0; w < (int)(sizeof(TileInfo) / 4); ++w) st_cluster_u32(dst + 4 * w, src[w]);
+                }
+                if (tl.type != 2) {
+                    ++taken;
+                    g_next = taken < budget ? (int)atomicAdd(&p.ctl->q_gemm, 1u) : 0x7fffffff;
+                    bool ok;
+                    if (tl.type == 0) {
+                        ok = flag_wait_ge(&p.xe_ready[tl.mb], 1u, p, 31);
+                        if (ok && tp.nrows > 0) ok = flag_wait_ge(&p.xe_ready[tp.mb], 1u, p, 31);
+                    } else {
+                        const unsigned need = (unsigned)(p.nt0 * kEpiWarps);
+                        ok = flag_wait_ge(&p.h_ready[tl.mb], need, p, 32);
+                        if (ok && tp.nrows > 0) ok = flag_wait_ge(&p.h_ready[tp.mb], need, p, 32);
+                    }
+                    if (!ok) break;
+                    trace_ev(p, S, kEvGemmLoad, (unsigned)g, tp0, trace_now(p), 0u);
+                }
                 mbar_arrive(&S.ti_full[ps.slot]);
+                mbar_arrive_cluster(mapa_u32(smem_u32(&S.ti_full[ps.slot]), 1u));
                 ps.next_slot();
-                if (ti.type == 2) break;
-                ++taken;
-                g_next = taken < budget ? (int)atomicAdd(&p.ctl->q_gemm, 1u) : 0x7fffffff;
-                const CUtensorMap *tma_a, *tma_b;
-                int brow0, brow1;
-                bool ok;
-                if (ti.type == 0) {
-                    ok = flag_wait_ge(&p.xe_ready[ti.mb], 1u, p, 31);
-                    tma_a = tm_xe; tma_b = tm_wgu;
-                    brow0 = ti.e * 2 * p.I + ti.n * kTN0;     // gate rows
-                    brow1 = brow0 + p.I;                       // up rows
-                } else {
-                    ok = flag_wait_ge(&p.h_ready[ti.mb], (unsigned)(p.nt0 * kEpiWarps), p, 32);
-                    tma_a = tm_h; tma_b = tm_wd;
-                    brow0 = ti.e * p.H + ti.n * p.bn1;
-                    brow1 = brow0 + 128;
-                }
-                if (!ok) { dead = true; break; }
-                const unsigned long long tp1 = trace_now(p);
-                fence_proxy_async();     // rows written with ordinary stores elsewhere, read by TMA here
-                const bool two_b = (ti.type == 0) || (p.bn1 == 256);
-                const uint32_t tx = kStageA + (two_b ? kStageB : kStageB / 2);
-                for (int kb = 0; kb < ti.nkb; ++kb) {
-                    if (!mbar_wait(&S.empty[ps.stage], ps.stage_phase ^ 1u, p, 33)) { dead = true; break; }
-                    uint8_t *sa = stages + ps.stage * kStageBytes;
-                    uint8_t *sb = sa + kStageA;
-                    mbar_arrive_expect_tx(&S.full[ps.stage], tx);
-                    tma_load_2d(sa, tma_a, kb * kBK, ti.row0, &S.full[ps.stage]);
-                    tma_load_2d(sb, tma_b, kb * kBK, brow0, &S.full[ps.stage]);
-                    if (two_b) tma_load_2d(sb + kStageB / 2, tma_b, kb * kBK, brow1, &S.full[ps.stage]);
-                    ps.next_stage();
-                }
-                trace_ev(p, S, kEvGemmLoad, (unsigned)g, tp0, trace_now(p), (unsigned)(tp1 - tp0));
-            }
-            if (dead) {     // let loads already issued land before this CTA can leave
-                const unsigned long long t0 = globaltimer_ns();
-                while (globaltimer_ns() - t0 < 50000ull) __nanosleep(1000);
+                if (tl.type == 2) break;
             }
         }
         __syncwarp();
-    } else if (warp == 1) {
-        // ---------------- MMA issuer: one thread drives the tensor core, accumulators live in TMEM
+    } else if (warp == 0) {
+        // ---------------- TMA producer (both CTAs): this CTA's 128 rows of A and its half of B
         if (lane == 0) {
             bool dead = false;
+            while (!dead) {
+                if (!mbar_wait_cluster(&S.ti_full[ps.slot], ps.slot_phase, p, 35)) { dead = true; break; }
+                const TileInfo ti = S.ti[ps.slot];
+                mbar_arrive_cluster(mapa_u32(smem_u32(&S.ti_empty[ps.slot]), 0u));
+                ps.next_slot();
+                if (ti.type == 2) break;
+                fence_proxy_async();     // rows written with ordinary stores elsewhere, read by TMA here
+                const CUtensorMap *tma_a, *tma_b;
+                int brow;
+                if (ti.type == 0) {      // leader holds the gate rows of the n-tile, peer the up rows
+                    tma_a = tm_xe; tma_b = tm_wgu;
+                    brow = ti.e * 2 * p.I + ti.n * kTN0 + (int)rank * p.I;
+                } else {                 // 256 output columns: leader the first 128 weight rows, peer the rest
+                    tma_a = tm_h; tma_b = tm_wd;
+                    brow = ti.e * p.H + ti.n * 256 + (int)rank * 128;
+                }
+                for (int kb = 0; kb < ti.nkb; ++kb) {
+                    if (!mbar_wait(&S.empty[ps.stage], ps.stage_phase ^ 1u, p, 33)) { dead = true; break; }
+                    uint8_t *sa = stages + ps.stage * kStageBytes;
+                    const uint32_t lbar = mapa_u32(smem_u32(&S.full[ps.stage]), 0u);
+                    if (rank == 0) mbar_arrive_expect_tx(&S.full[ps.stage], 2u * kStageBytes);
+                    tma_load_2d_pair(sa, tma_a, kb * kBK, ti.row0, lbar);
+                    tma_load_2d_pair(sa + kStageA, tma_b, kb * kBK, brow, lbar);
+                    ps.next_stage();
+                }
+            }
+            if (dead) linger_after_abort();
+        }
+        __syncwarp();
+    } else if (warp == 1 && rank == 0) {
+        // ---------------- MMA issuer (leader only): one thread drives both SMs' tensor cores
+        if (lane == 0) {
+            bool dead = false;
+            const uint32_t idesc = umma_idesc_bf16(2 * kBM, 256u);
             while (!dead) {
                 if (!mbar_wait(&S.ti_full[ps.slot], ps.slot_phase, p, 40)) { dead = true; break; }
                 const TileInfo ti = S.ti[ps.slot];
                 mbar_arrive(&S.ti_empty[ps.slot]);
                 ps.next_slot();
                 if (ti.type == 2) break;
-                const uint32_t idesc = umma_idesc_bf16(kBM, ti.type == 0 ? 256u : (uint32_t)p.bn1);
-                if (!mbar_wait(&S.tmem_empty[ps.acc], ps.acc_phase ^ 1u, p, 41)) { dead = true; break; }
+                if (!mbar_wait_cluster(&S.tmem_empty[ps.acc], ps.acc_phase ^ 1u, p, 41)) { dead = true; break; }
                 tc_fence_after();
                 const uint32_t d = tmem_base + (uint32_t)ps.acc * 256u;
                 for (int kb = 0; kb < ti.nkb; ++kb) {
-                    if (!mbar_wait(&S.full[ps.stage], ps.stage_phase, p, 42)) { dead = true; break; }
+                    if (!mbar_wait_cluster(&S.full[ps.stage], ps.stage_phase, p, 42)) { dead = true; break; }
                     tc_fence_after();
                     const uint32_t a0 = smem_u32(stages + ps.stage * kStageBytes);
                     const uint32_t b0 = a0 + kStageA;
 #pragma unroll
                     for (int kk = 0; kk < kBK / 16; ++kk)
-                        tc_mma_bf16(d, umma_desc_sw128(a0 + kk * 32), umma_desc_sw128(b0 + kk * 32), idesc,
-                                    (uint32_t)((kb | kk) != 0));
-                    tc_commit(&S.empty[ps.stage]);       // frees the stage when these MMAs have read it
+                        tc_mma_bf16_pair(d, umma_desc_sw128(a0 + kk * 32), umma_desc_sw128(b0 + kk * 32), idesc,
+                                         (uint32_t)((kb | kk) != 0));
+                    tc_commit_pair(&S.empty[ps.stage], 3);      // both CTAs' stage is free once read
                     ps.next_stage();
                 }
                 if (dead) break;
-                tc_commit(&S.tmem_full[ps.acc]);         // accumulator complete
+                tc_commit_pair(&S.tmem_full[ps.acc], 3);        // accumulators complete in both CTAs
                 ps.next_acc();
             }
-            if (dead) {
-                const unsigned long long t0 = globaltimer_ns();
-                while (globaltimer_ns() - t0 < 50000ull) __nanosleep(1000);
-            }
+            if (dead) linger_after_abort();
         }
         __syncwarp();
     } else if (warp >= 4) {
-        // ---------------- epilogue: TMEM -> registers -> (SwiGLU) -> bf16 -> global, row-masked
+        // ---------------- epilogue (both CTAs): TMEM -> registers -> (SwiGLU) -> bf16 -> staged store
         const int q = warp & 3;                      // TMEM lane quadrant this warp may read
+        const uint32_t stg = smem_u32(stages + kStages * kStageBytes) + (uint32_t)q * 2048u;
         bool dead = false;
         while (!dead) {
-            if (!mbar_wait(&S.ti_full[ps.slot], ps.slot_phase, p, 50)) { dead = true; }
+            if (!mbar_wait_cluster(&S.ti_full[ps.slot], ps.slot_phase, p, 50)) { dead = true; }
             dead = __any_sync(0xffffffffu, dead);
             if (dead) break;
             const TileInfo ti = S.ti[ps.slot];
             __syncwarp();
-            if (lane == 0) mbar_arrive(&S.ti_empty[ps.slot]);
+            if (lane == 0) mbar_arrive_cluster(mapa_u32(smem_u32(&S.ti_empty[ps.slot]), 0u));
             ps.next_slot();
             if (ti.type == 2) break;
             if (!mbar_wait(&S.tmem_full[ps.acc], ps.acc_phase, p, 51)) { dead = true; }
@@ -654,62 +744,58 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
             if (dead) break;
             tc_fence_after();
             const unsigned long long te0 = trace_now(p);
-            const int r = q * 32 + lane;
-            const bool valid = r < ti.nrows;
+            const int rows_valid = ti.nrows - q * 32;          // rows of this warp's quadrant that exist
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)ps.acc * 256u;
-            if (ti.type == 0) {
-                __nv_bfloat16 *dst = p.hbuf + (size_t)(ti.row0 + r) * p.I + (size_t)ti.n * kTN0;
+            if (rows_valid > 0) {
+                if (ti.type == 0) {
+                    __nv_bfloat16 *dst = p.hbuf + (size_t)(ti.row0 + q * 32) * p.I + (size_t)ti.n * kTN0;
 #pragma unroll 1
-                for (int c = 0; c < kTN0 / 32; ++c) {
-                    uint32_t gr[32], ur[32];
-                    tmem_ld_32x32(taddr + c * 32, gr);
-                    tmem_ld_32x32(taddr + 128 + c * 32, ur);
-                    tmem_ld_wait();
-                    uint32_t o[16];
+                    for (int c = 0; c < kTN0 / 32; ++c) {
+                        uint32_t gr[32], ur[32];
+                        tmem_ld_32x32(taddr + c * 32, gr);
+                        tmem_ld_32x32(taddr + 128 + c * 32, ur);
+                        tmem_ld_wait();
+                        uint32_t o[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        o[i] = pack_bf16x2(silu_mul(__uint_as_float(gr[2 * i]), __uint_as_float(ur[2 * i])),
-                                           silu_mul(__uint_as_float(gr[2 * i + 1]), __uint_as_float(ur[2 * i + 1])));
-                    if (valid) {
-#pragma unroll
-                        for (int i = 0; i < 4; ++i)
-                            st_v4(dst + c * 32 + i * 8, make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]));
+                        for (int i = 0; i < 16; ++i)
+                            o[i] = pack_bf16x2(silu_mul(__uint_as_float(gr[2 * i]), __uint_as_float(ur[2 * i])),
+                                               silu_mul(__uint_as_float(gr[2 * i + 1]), __uint_as_float(ur[2 * i + 1])));
+                        staged_store_32x32(stg, lane, o, dst + c * 32, (size_t)p.I, rows_valid);
                     }
-                }
-            } else {
-                __nv_bfloat16 *dst = p.y + (size_t)(ti.row0 + r) * p.H + (size_t)ti.n * p.bn1;
-                const int nc = p.bn1 / 32;
+                } else {
+                    __nv_bfloat16 *dst = p.y + (size_t)(ti.row0 + q * 32) * p.H + (size_t)ti.n * 256;
+                    const int nc = min(256, p.H - ti.n * 256) / 32;   // the last n-tile may be half wide
 #pragma unroll 1
-                for (int c = 0; c < nc; ++c) {
-                    uint32_t ar[32];
-                    tmem_ld_32x32(taddr + c * 32, ar);
-                    tmem_ld_wait();
-                    if (valid) {
+                    for (int c = 0; c < nc; ++c) {
+                        uint32_t ar[32];
+                        tmem_ld_32x32(taddr + c * 32, ar);
+                        tmem_ld_wait();
+                        uint32_t o[16];
 #pragma unroll
-                        for (int i = 0; i < 4; ++i)
-                            st_v4(dst + c * 32 + i * 8,
-                                  make_uint4(pack_bf16x2(__uint_as_float(ar[8 * i]), __uint_as_float(ar[8 * i + 1])),
-                                             pack_bf16x2(__uint_as_float(ar[8 * i + 2]), __uint_as_float(ar[8 * i + 3])),
-                                             pack_bf16x2(__uint_as_float(ar[8 * i + 4]), __uint_as_float(ar[8 * i + 5])),
-                                             pack_bf16x2(__uint_as_float(ar[8 * i + 6]), __uint_as_float(ar[8 * i + 7]))));
+                        for (int i = 0; i < 16; ++i)
+                            o[i] = pack_bf16x2(__uint_as_float(ar[2 * i]), __uint_as_float(ar[2 * i + 1]));
+                        staged_store_32x32(stg, lane, o, dst + c * 32, (size_t)p.H, rows_valid);
                     }
                 }
             }
-            // accumulator may be overwritten by the next-but-one tile
+            // the accumulator may be overwritten by the next-but-one tile; the rows just stored are read
+            // by TMA (gemm1) or by ordinary loads (combine) on other SMs once the counter says so
             tc_fence_before();
-            fence_proxy_async();     // h rows are read by TMA on another SM
+            fence_proxy_async();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(&S.tmem_empty[ps.acc]);
-                __threadfence();
-                red_release_add_u32(ti.type == 0 ? &p.h_ready[ti.mb] : &p.ctl->y_done[ti.chunk], 1u);
-                if (q == 0) trace_ev(p, S, kEvGemmEpi, (unsigned)ti.mb, te0, trace_now(p), (unsigned)(ti.type << 16 | ti.n));
+                mbar_arrive_cluster(mapa_u32(smem_u32(&S.tmem_empty[ps.acc]), 0u));
+                if (ti.nrows > 0)
+                    red_release_add_u32(ti.type == 0 ? &p.h_ready[ti.mb] : &p.ctl->y_done[ti.chunk], 1u);
+                if (q == 0) trace_ev(p, S, kEvGemmEpi, (unsigned)(ti.mb & 0xFFFFFF), te0, trace_now(p),
+                                     (unsigned)(ti.type << 16 | ti.n));
             }
             ps.next_acc();
         }
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();      // nobody targets the other CTA's shared memory or barriers after this
     tc_fence_after();
 }
 
@@ -722,21 +808,25 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *stages = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    SmemTail &S = *reinterpret_cast<SmemTail *>(stages + kStages * kStageBytes);
+    // [stage ring | epilogue staging | SmemTail]
+    SmemTail &S = *reinterpret_cast<SmemTail *>(stages + kStages * kStageBytes + kEpiStageBytes);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_sm = (int)gridDim.x;
     const int EE = p.EE;
 
     if (tid == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(&S.full[i], 1); mbar_init(&S.empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&S.tmem_full[i], 1); mbar_init(&S.tmem_empty[i], kEpiWarps); }
-        for (int i = 0; i < kTinfo; ++i) { mbar_init(&S.ti_full[i], 1); mbar_init(&S.ti_empty[i], 1 + kEpiWarps); }
+        // accumulator free: 4 epilogue warps in each CTA of the pair arrive on the leader's barrier
+        for (int i = 0; i < 2; ++i) { mbar_init(&S.tmem_full[i], 1); mbar_init(&S.tmem_empty[i], 2 * kEpiWarps); }
+        // tile descriptor consumed: leader's producer + MMA + 4 epilogue warps, peer's producer + 4 warps
+        for (int i = 0; i < kTinfo; ++i) { mbar_init(&S.ti_full[i], 1); mbar_init(&S.ti_empty[i], 3 + 2 * kEpiWarps); }
         fence_mbar_init();
         tma_prefetch_desc(&tm_xe); tma_prefetch_desc(&tm_wgu); tma_prefetch_desc(&tm_h); tma_prefetch_desc(&tm_wd);
     }
-    if (warp == 1) { tmem_alloc(&S.tmem_base, kTmemCols); tmem_relinquish(); }
+    if (warp == 1) { tmem_alloc_pair(&S.tmem_base, kTmemCols); tmem_relinquish_pair(); }
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();      // the peer's barriers exist before anything is sent to them
     tc_fence_after();
     const uint32_t tmem_base = S.tmem_base;
     if (tid == 0) S.trace_n = 0u;
@@ -796,7 +886,8 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
         p.offsets[tid] = off;
         if (tid == 0) p.offsets[EE] = total_rows;
     }
-    // m-blocks of the layer for each candidate K (a segment = one expert's rows inside one chunk)
+    // pair tiles (256 rows) of the layer for each candidate K (a segment = one expert's rows inside
+    // one chunk; its last pair tile may be half empty)
     int mbk[4];
 #pragma unroll
     for (int ki = 0; ki < 4; ++ki) {
@@ -806,7 +897,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
             int rows = 0;
 #pragma unroll
             for (int f = 0; f < kFine; ++f) if (f / g == j) rows += cf[f];
-            acc += (rows + kBM - 1) / kBM;
+            acc += (rows + 2 * kBM - 1) / (2 * kBM);
         }
         mbk[ki] = acc;
 #pragma unroll
@@ -835,7 +926,8 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
         const int ci = tid >> 2, ki = tid & 3;
         const int cc = p.c_min + ci * p.c_step;
         float t = __int_as_float(0x7f800000);
-        if (cc >= 1 && cc <= p.c_max && cc <= n_sm - 1) t = model_t_total(p, n_sm, cc, ki, w_comp, w_disp, w_comb);
+        if (cc >= 2 && cc <= p.c_max && cc <= n_sm - 2 && (EE << ki) <= kMaxSeg)
+            t = model_t_total(p, n_sm, cc, ki, w_comp, w_disp, w_comb);
         int bi = tid;       // candidate order = (c ascending, K ascending): ties go to the smaller index
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
@@ -854,11 +946,12 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
         plan_c = p.c_min + (bi >> 2) * p.c_step;
         plan_ki = bi & 3;
         plan_t = t;
-        plan_steal = model_n_steal(p, n_sm, plan_c, w_comp, w_disp, w_comb, n_tiles_k[plan_ki]);
+        plan_steal = model_n_steal(p, n_sm, plan_c, w_comp, w_disp, w_comb, n_tiles_k[plan_ki]);   // per CTA pair
         __syncthreads();
     } else if (p.mode == kModeFixed) {
-        plan_c = max(1, min(p.fixed_c, n_sm - 1));
+        plan_c = max(2, min((p.fixed_c + 1) & ~1, n_sm - 2));     // whole CTA pairs
         plan_ki = p.fixed_K >= 8 ? 3 : p.fixed_K >= 4 ? 2 : p.fixed_K >= 2 ? 1 : 0;
+        while (plan_ki > 0 && (EE << plan_ki) > kMaxSeg) --plan_ki;
         plan_steal = max(0, p.fixed_steal);
     } else {
         plan_c = n_sm;
@@ -869,34 +962,43 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
     {
         const int g = kFine / K;
         int run_row = tid < EE ? off : 0;
-        int mb_base = 0;
+        int mb_base = 0, pt_base = 0;
         for (int j = 0; j < K; ++j) {
             int rows = 0;
 #pragma unroll
             for (int f = 0; f < kFine; ++f) if (f / g == j) rows += cf[f];
             const int mbs = (rows + kBM - 1) / kBM;
-            int tot;
+            int tot, ptot;
             const int ex = block_excl_scan(mbs, S, tot);
+            const int pex = block_excl_scan((mbs + 1) >> 1, S, ptot);
             if (tid < EE) {
                 S.seg_mb0[j * EE + tid] = mb_base + ex;
+                S.seg_pt0[j * EE + tid] = pt_base + pex;
                 S.seg_row0[j * EE + tid] = run_row;
                 S.seg_rows[j * EE + tid] = rows;
             }
-            if (tid == 0) { S.chunk_mb0[j] = mb_base; S.chunk_tile0[j] = mb_base * (p.nt0 + p.nt1); }
+            if (tid == 0) {
+                S.chunk_mb0[j] = mb_base;
+                S.chunk_pt0[j] = pt_base;
+                S.chunk_tile0[j] = pt_base * (p.nt0 + p.nt1);
+            }
             run_row += rows;
             mb_base += tot;
+            pt_base += ptot;
         }
         if (tid == 0) {
             S.seg_mb0[K * EE] = mb_base;
+            S.seg_pt0[K * EE] = pt_base;
             S.chunk_mb0[K] = mb_base;
-            S.chunk_tile0[K] = mb_base * (p.nt0 + p.nt1);
+            S.chunk_pt0[K] = pt_base;
+            S.chunk_tile0[K] = pt_base * (p.nt0 + p.nt1);
             S.c = plan_c; S.K = K; S.steal = plan_steal;
             S.nmb = mb_base;
-            S.n_gemm = mb_base * (p.nt0 + p.nt1);
+            S.n_gemm = pt_base * (p.nt0 + p.nt1);
             S.n_comb = (p.T + kCombTile - 1) / kCombTile;
             if (blockIdx.x == 0) {
                 p.ctl->plan_c = plan_c; p.ctl->plan_K = K; p.ctl->plan_steal = plan_steal; p.ctl->plan_t = plan_t;
-                p.ctl->plan_nmb = mb_base; p.ctl->plan_ngemm = mb_base * (p.nt0 + p.nt1);
+                p.ctl->plan_nmb = mb_base; p.ctl->plan_ngemm = pt_base * (p.nt0 + p.nt1);
             }
         }
     }
@@ -965,7 +1067,8 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+    cluster_sync_all();
+    if (warp == 1) tmem_dealloc_pair(tmem_base, kTmemCols);
     if (tid == 0) {
         if (p.trace)     // last record of the CTA's slice: how many events were written
             p.trace[(size_t)blockIdx.x * p.trace_cap + p.trace_cap - 1] =

@@ -85,7 +85,8 @@ struct weave_moe {
     weave_moe_config cfg;
     Layout L;
     uint8_t *ws;
-    int n_sm;
+    int n_sm;      // SMs of the device
+    int n_cta;     // persistent CTAs = SMs rounded down to whole pairs
     int device;
     int mode, fixed_c, fixed_K, fixed_steal;
     int c_min, c_max, c_step;
@@ -177,17 +178,18 @@ int weave_moe_create(const weave_moe_config *cfg, weave_moe_t *out)
     if (e != cudaSuccess) return WEAVE_ERR_CUDA;
     if (prop.major != 10 || !prop.cooperativeLaunch) return WEAVE_ERR_UNSUPPORTED_DEVICE;
     if ((int)prop.sharedMemPerBlockOptin < kSmemBytes) return WEAVE_ERR_UNSUPPORTED_DEVICE;
-    if (prop.multiProcessorCount + 1 > 1024) return WEAVE_ERR_UNSUPPORTED_DEVICE;
+    if (prop.multiProcessorCount + 1 > 1024 || prop.multiProcessorCount < 4) return WEAVE_ERR_UNSUPPORTED_DEVICE;
 
     weave_moe *h = new (std::nothrow) weave_moe();
     if (!h) return WEAVE_ERR_INVALID_ARG;
     h->cfg = *cfg;
     h->L = L;
     h->ws = static_cast<uint8_t *>(cfg->workspace);
-    h->n_sm = prop.multiProcessorCount;
+    h->n_sm = prop.multiProcessorCount & ~1;     // the scheduler counts SMs in whole CTA pairs
+    h->n_cta = h->n_sm;
     h->device = dev;
     h->mode = WEAVE_SCHED_AUTO;
-    h->fixed_c = h->n_sm * 15 / 100;
+    h->fixed_c = (h->n_sm * 15 / 100 + 1) & ~1;
     h->fixed_K = 1;
     h->fixed_steal = 0;
     h->c_min = 2;
@@ -205,9 +207,22 @@ int weave_moe_create(const weave_moe_config *cfg, weave_moe_t *out)
 
     e = cudaFuncSetAttribute(weave_moe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) { int rc = cuda_fail(h, e); delete h; return rc; }
+    e = cudaFuncSetAttribute(weave_moe_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 0);
     int occ = 0;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, weave_moe_kernel, kThreads, kSmemBytes);
     if (e != cudaSuccess || occ < 1) { delete h; return WEAVE_ERR_UNSUPPORTED_DEVICE; }
+    {
+        cudaLaunchConfig_t lc;
+        memset(&lc, 0, sizeof(lc));
+        lc.gridDim = dim3(h->n_cta); lc.blockDim = dim3(kThreads); lc.dynamicSmemBytes = (size_t)kSmemBytes;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+        lc.attrs = at; lc.numAttrs = 1;
+        int ncl = 0;
+        e = cudaOccupancyMaxActiveClusters(&ncl, (const void *)weave_moe_kernel, &lc);
+        if (e != cudaSuccess || ncl * 2 < h->n_cta) { delete h; return WEAVE_ERR_UNSUPPORTED_DEVICE; }
+    }
 
     void *fnp = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -250,9 +265,8 @@ int weave_moe_forward(weave_moe_t h, const void *x, const float *logits, void *o
     p.EE = c.num_experts + c.num_shared;
     p.nblk = (T + kRouteBlock - 1) / kRouteBlock;
     p.mode = h->mode; p.fixed_c = h->fixed_c; p.fixed_K = h->fixed_K; p.fixed_steal = h->fixed_steal;
-    p.bn1 = (c.hidden % 256 == 0) ? 256 : 128;
     p.nt0 = c.ffn / kTN0;
-    p.nt1 = c.hidden / p.bn1;
+    p.nt1 = (c.hidden + 255) / 256;
     p.nmb_max = L.nmb_max;
     p.withhold_mb = h->withhold_mb;
     p.c_min = h->c_min; p.c_max = h->c_max; p.c_step = h->c_step;
@@ -284,8 +298,22 @@ int weave_moe_forward(weave_moe_t h, const void *x, const float *logits, void *o
 
     void *args[] = {&p, &h->tm_xe, &h->tm_wgu, &h->tm_h, &h->tm_wd};
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    cudaError_t e = cudaLaunchCooperativeKernel((const void *)weave_moe_kernel, dim3(h->n_sm), dim3(kThreads), args,
-                                                (size_t)kSmemBytes, st);
+    // one CTA per SM, in clusters of two neighbouring SMs (the GEMM phase's CTA pairs); cooperative,
+    // so that all CTAs are co-resident for the in-kernel grid barrier and flag waits
+    cudaLaunchConfig_t lc;
+    memset(&lc, 0, sizeof(lc));
+    lc.gridDim = dim3(h->n_cta);
+    lc.blockDim = dim3(kThreads);
+    lc.dynamicSmemBytes = (size_t)kSmemBytes;
+    lc.stream = st;
+    cudaLaunchAttribute at[2];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeCooperative;
+    at[1].val.cooperative = 1;
+    lc.attrs = at;
+    lc.numAttrs = 2;
+    cudaError_t e = cudaLaunchKernelExC(&lc, (const void *)weave_moe_kernel, args);
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->last_T = T;
     h->last_stream = st;
@@ -336,7 +364,8 @@ int weave_moe_set_cost_tables(weave_moe_t h, const float *bw, const float *tflop
                               float alpha, int c_min, int c_max, int c_step)
 {
     if (!h || !bw || !tflops || !eff_chunk) return WEAVE_ERR_INVALID_ARG;
-    if (!(alpha >= 0.f && alpha < 1.f) || c_min < 1 || c_step < 1 || c_max < c_min) return WEAVE_ERR_INVALID_ARG;
+    if (!(alpha >= 0.f && alpha < 1.f) || c_min < 2 || c_step < 2 || c_max < c_min) return WEAVE_ERR_INVALID_ARG;
+    if ((c_min & 1) || (c_step & 1)) return WEAVE_ERR_INVALID_ARG;     // movement SMs come in CTA pairs
     if ((c_max - c_min) / c_step + 1 > 64) return WEAVE_ERR_INVALID_ARG;
     for (int i = 1; i <= h->n_sm; ++i)
         if (!(bw[i] > 0.f) || !(tflops[i] > 0.f)) return WEAVE_ERR_INVALID_ARG;
@@ -366,13 +395,14 @@ int weave_moe_get_plan(weave_moe_t h, int *c, int *K, int *n_steal, float *t_tot
 }
 
 int weave_moe_get_geometry(weave_moe_t h, int *n_sm, int *block_m, int *tile_n0, int *tile_n1, int *route_block,
-                           int *combine_tile)
+                           int *combine_tile, int *gemm_tile_m)
 {
     if (!h) return WEAVE_ERR_INVALID_ARG;
     if (n_sm) *n_sm = h->n_sm;
     if (block_m) *block_m = kBM;
     if (tile_n0) *tile_n0 = kTN0;
-    if (tile_n1) *tile_n1 = (h->cfg.hidden % 256 == 0) ? 256 : 128;
+    if (tile_n1) *tile_n1 = 256;
+    if (gemm_tile_m) *gemm_tile_m = 2 * kBM;
     if (route_block) *route_block = kRouteBlock;
     if (combine_tile) *combine_tile = kCombTile;
     return WEAVE_OK;

@@ -37,7 +37,9 @@ def test_c1_tiny_every_schedule_matches_oracle_and_each_other():
         assert torch.equal(out.view(torch.int16), ref_bits), f"schedule {s} changed the output bits"
         if s[0] == pk.SCHED_FIXED:
             p = moe.plan()
-            assert (p["c"], p["K"], p["n_steal"]) == (s[1], s[2], s[3])
+            n_sm = moe.geometry()["n_sm"]
+            c_eff = max(2, min((s[1] + 1) & ~1, n_sm - 2))      # whole SM pairs, both groups non-empty
+            assert (p["c"], p["K"], p["n_steal"]) == (c_eff, s[2], s[3])
     moe.close()
 
 
@@ -221,15 +223,15 @@ def test_forward_host_equals_forward():
 
 def _n_tiles_of_K(counts_fine, geo, H, I):
     """GEMM tiles of the layer for K = 1,2,4,8 from per-(fine chunk, expert) row counts."""
-    nt = I // geo["tile_n0"] + H // geo["tile_n1"]
+    nt = I // geo["tile_n0"] + (H + geo["tile_n1"] - 1) // geo["tile_n1"]
     res = []
     for K in (1, 2, 4, 8):
         g = 8 // K
-        mb = 0
+        tiles = 0
         for j in range(K):
             rows = counts_fine[j * g:(j + 1) * g].sum(axis=0)
-            mb += int(((rows + geo["block_m"] - 1) // geo["block_m"]).sum())
-        res.append(mb * nt)
+            tiles += int(((rows + geo["gemm_tile_m"] - 1) // geo["gemm_tile_m"]).sum())
+        res.append(tiles * nt)
     return res
 
 
@@ -267,7 +269,7 @@ def test_device_plan_equals_cpu_cost_model(name):
         bw[0], tf[0] = bw[1], tf[1]
         eff = np.array([1.0, rng.uniform(.8, 1), rng.uniform(.6, .9), rng.uniform(.4, .8)], np.float32)
         alpha = float(rng.uniform(0, 0.95))
-        tab = cm.CostTables(N, bw, tf, eff, alpha, c_min=2, c_max=N // 2, c_step=2)
+        tab = cm.CostTables(N, bw, tf, eff, alpha, c_min=2, c_max=N // 2, c_step=2, steal_workers=N // 2)
         want = cm.plan(tab, cfg.T, cfg.P, cfg.H, cfg.I, nt)
         moe.set_cost_tables(bw, tf, eff, alpha, 2, N // 2, 2)
         moe.set_schedule(pk.SCHED_AUTO)
