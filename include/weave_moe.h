@@ -48,7 +48,7 @@ enum {
 enum { WEAVE_SCHED_AUTO = 0, WEAVE_SCHED_FIXED = 1, WEAVE_SCHED_SERIAL = 2 };
 
 typedef struct weave_moe_config {
-    int hidden;       /* H: model width, multiple of 128                                          */
+    int hidden;       /* H: model width, multiple of 128, at most 16384                           */
     int ffn;          /* I: per-expert intermediate width, multiple of 128                         */
     int num_experts;  /* E: routed experts, >= 1                                                  */
     int top_k;        /* k: experts per token, 1 <= k <= min(E, 16)                               */

@@ -110,11 +110,25 @@ struct TileInfo {
     int e, n, chunk, nkb;
 };
 
+// what one movement buffer (a 32 KB stage) currently holds
+struct MvDesc {
+    int a;      // dispatch: first destination row        combine: token
+    int b;      // dispatch: rows in the buffer            combine: first column
+    int c;      // dispatch: m-block                       combine: columns
+    int d;      // dispatch: 1 = last buffer of its tile;  2 = no more work (both phases)
+    float g[kMaxTopK + 8];   // combine: weight of each gathered row
+};
+constexpr int kMvBuf = kStageBytes;     // 32 KB
+constexpr int kCombWarps = 6;           // warps 2..7 reduce
+
 struct SmemTail {
     uint64_t full[kStages], empty[kStages];
     uint64_t tmem_full[2], tmem_empty[2];
     uint64_t ti_full[kTinfo], ti_empty[kTinfo];
+    uint64_t dv_full[kStages], dv_empty[kStages];   // dispatch: loader -> storer ring over the stage buffers
+    uint64_t cb_full[kStages], cb_empty[kStages];   // combine: loader -> reducing warps
     TileInfo ti[kTinfo];
+    MvDesc mv[kStages];
     uint32_t tmem_base;
     int bcast[3];
     int red_i[8][4];
@@ -128,8 +142,8 @@ struct SmemTail {
     int chunk_tile0[kFine + 1];
     int offsets[kMaxEE + 1];
     int tok[kBM];
-    int crow[8][kMaxTopK + 8];
-    float cgate[8][kMaxTopK + 8];
+    int crow[kCombTile][kMaxTopK + 8];
+    float cgate[kCombTile][kMaxTopK + 8];
     int seg_mb0[kMaxSeg + 1];
     int seg_pt0[kMaxSeg + 1];    // prefix of pair tiles: ceil(m-blocks / 2) per segment
     int seg_row0[kMaxSeg];
@@ -400,145 +414,202 @@ __device__ __forceinline__ void decode_pair_tile(const SmemTail &S, const KParam
 
 // ------------------------------------------------------------------------------------ phase A: dispatch
 
-// Tile = one m-block: Xe[row0 + r] = x[token_of[row0 + r]].  16-byte vectors, 8 loads in flight
-// per thread; the m-block's ready flag is released when its rows are written.
-__device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S)
+// Tile = one m-block: Xe[row0 + r] = x[token_of[row0 + r]].  The copy engine does the moving: warp 0
+// gathers the source rows with bulk loads into a ring of 32 KB buffers, one thread of warp 1
+// writes each full buffer to its (contiguous) destination rows with one bulk store.  About 96 KB
+// of loads and as much of stores are in flight per SM.  The m-block's ready flag is released once
+// its last store has completed.
+__device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, uint8_t *stages)
 {
-    const int tid = threadIdx.x;
-    if (tid == 0) S.bcast[1] = flag_wait_ge(&p.ctl->fix_done, (unsigned)p.nblk, p, 10) ? 1 : 0;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    fence_proxy_async();      // the buffers held routing scratch written with ordinary stores
     __syncthreads();
-    if (!S.bcast[1]) return;
-    const int n16 = p.H >> 3;
-    for (;;) {
-        if (tid == 0) S.bcast[0] = (int)atomicAdd(&p.ctl->q_disp, 1u);
-        __syncthreads();
-        const int mb = S.bcast[0];
-        if (mb >= S.nmb) break;
-        int row0, nrows;
-        decode_mblock(S, p.EE, mb, row0, nrows);
-        const unsigned long long tr0 = trace_now(p);
-        for (int i = tid; i < nrows; i += kThreads) S.tok[i] = __ldcg(p.token_of + row0 + i);
-        __syncthreads();
-        const int total = nrows * n16;
-        constexpr int U = 8;
-        for (int base = tid; base < total; base += kThreads * U) {
-            uint4 v[U];
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int i = base + u * kThreads;
-                if (i < total) {
-                    const int r = i / n16, c = i - r * n16;
-                    v[u] = ld_nc_v4(p.x + (size_t)S.tok[r] * p.H + (size_t)c * 8);
+    const uint32_t rowb = (uint32_t)p.H * 2u;
+    const int R = max(1, kMvBuf / (int)rowb);     // rows per buffer
+    if (warp == 0) {
+        // ---- loader
+        int b = 0;
+        uint32_t ph = 0;
+        bool ok = true;
+        if (lane == 0) ok = flag_wait_ge(&p.ctl->fix_done, (unsigned)p.nblk, p, 10);
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        while (ok) {
+            int mb = 0;
+            if (lane == 0) mb = (int)atomicAdd(&p.ctl->q_disp, 1u);
+            mb = __shfl_sync(0xffffffffu, mb, 0);
+            if (mb >= S.nmb) break;
+            int row0, nrows;
+            decode_mblock(S, p.EE, mb, row0, nrows);
+            for (int i = lane; i < nrows; i += 32) S.tok[i] = __ldcg(p.token_of + row0 + i);
+            __syncwarp();
+            if (lane == 0) {
+                for (int r0 = 0; r0 < nrows; r0 += R) {
+                    const int nr = min(R, nrows - r0);
+                    if (!mbar_wait(&S.dv_empty[b], ph ^ 1u, p, 11)) { ok = false; break; }
+                    S.mv[b].a = row0 + r0; S.mv[b].b = nr; S.mv[b].c = mb; S.mv[b].d = (r0 + nr >= nrows) ? 1 : 0;
+                    mbar_arrive_expect_tx(&S.dv_full[b], (uint32_t)nr * rowb);
+                    const uint32_t dst = smem_u32(stages + b * kMvBuf);
+                    for (int i = 0; i < nr; ++i)
+                        bulk_load(dst + (uint32_t)i * rowb, p.x + (size_t)S.tok[r0 + i] * p.H, rowb, &S.dv_full[b]);
+                    if (++b == kStages) { b = 0; ph ^= 1u; }
                 }
             }
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int i = base + u * kThreads;
-                if (i < total) {
-                    const int r = i / n16, c = i - r * n16;
-                    st_v4(p.xe + (size_t)(row0 + r) * p.H + (size_t)c * 8, v[u]);
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            __syncwarp();
+        }
+        if (lane == 0 && ok && mbar_wait(&S.dv_empty[b], ph ^ 1u, p, 12)) {
+            S.mv[b].d = 2;
+            mbar_arrive(&S.dv_full[b]);
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ---- storer
+        if (lane == 0) {
+            int b = 0, n = 0;
+            uint32_t ph = 0;
+            int h_buf[3] = {0, 0, 0}, h_mb[3] = {0, 0, 0}, h_last[3] = {0, 0, 0}, h_rows[3] = {0, 0, 0};
+            unsigned long long h_t0[3] = {0ull, 0ull, 0ull};
+            auto retire = [&](int i) {
+                const int s3 = i % 3;
+                mbar_arrive(&S.dv_empty[h_buf[s3]]);
+                if (h_last[s3]) {
+                    if (h_mb[s3] != p.withhold_mb) {
+                        fence_proxy_async();      // these rows are read by TMA on another SM
+                        __threadfence();
+                        st_release_u32(&p.xe_ready[h_mb[s3]], 1u);
+                    }
+                    trace_ev(p, S, kEvDispatch, (unsigned)h_mb[s3], h_t0[s3], trace_now(p), (unsigned)h_rows[s3]);
                 }
+            };
+            unsigned long long tile_t0 = trace_now(p);
+            for (;;) {
+                if (!mbar_wait(&S.dv_full[b], ph, p, 13)) break;
+                const int da = S.mv[b].a, db = S.mv[b].b, dc = S.mv[b].c, dd = S.mv[b].d;
+                if (dd == 2) break;
+                bulk_store(p.xe + (size_t)da * p.H, smem_u32(stages + b * kMvBuf), (uint32_t)db * rowb);
+                bulk_commit();
+                h_buf[n % 3] = b; h_mb[n % 3] = dc; h_last[n % 3] = dd; h_rows[n % 3] = db; h_t0[n % 3] = tile_t0;
+                if (dd == 1) tile_t0 = trace_now(p);
+                ++n;
+                if (n >= 3) { bulk_wait<2>(); retire(n - 3); }
+                if (++b == kStages) { b = 0; ph ^= 1u; }
             }
+            bulk_wait<0>();
+            for (int i = max(0, n - 2); i < n; ++i) retire(i);
         }
-        fence_proxy_async();      // these rows are read by TMA (async proxy) on another SM
-        __syncthreads();
-        if (tid == 0 && mb != p.withhold_mb) {
-            __threadfence();
-            st_release_u32(&p.xe_ready[mb], 1u);
-        }
-        if (tid == 0) trace_ev(p, S, kEvDispatch, (unsigned)mb, tr0, trace_now(p), (unsigned)nrows);
+        __syncwarp();
     }
     __syncthreads();
 }
 
 // ------------------------------------------------------------------------------------ phase C: combine
 
-// Tile = 16 tokens; a warp owns two of them.  out[t] = sum_j gate[t,j] * y[row_of[t,j]] in slot
-// order, then the shared experts with weight 1; fp32 accumulate, bf16 store.
-__device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S)
+// Tile = 16 tokens.  out[t] = sum_j gate[t,j] * y[row_of[t,j]] in slot order, then the shared
+// experts with weight 1; fp32 accumulate, bf16 store.  Warp 0 gathers, per token and per piece of
+// W columns, the k+S source rows with bulk loads into a ring of 32 KB buffers; warps 2..7 reduce
+// each full buffer from shared memory and write the output row piece with coalesced stores.
+__device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uint8_t *stages)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int n16 = p.H >> 3;
+    fence_proxy_async();
+    __syncthreads();
     const int kk = p.k + p.S;
+    const int W = min(p.H, ((kMvBuf / (2 * kk)) / 64) * 64);     // columns per piece (128-byte multiple)
     const int g = kFine / S.K;
-    int ready_upto = -1;     // chunks [0, ready_upto] are known complete
-    for (;;) {
-        if (tid == 0) S.bcast[0] = (int)atomicAdd(&p.ctl->q_comb, 1u);
-        __syncthreads();
-        const int q = S.bcast[0];
-        if (q >= S.n_comb) break;
-        const int t0 = q * kCombTile;
-        const int chunk = (((t0 / kRouteBlock) * kFine) / p.nblk) / g;
-        if (chunk > ready_upto) {
-            if (tid == 0) {
-                const unsigned long long tw0 = trace_now(p);
-                bool ok = flag_wait_ge(&p.ctl->fix_done, (unsigned)p.nblk, p, 20);
-                for (int j = ready_upto + 1; ok && j <= chunk; ++j) {
-                    const unsigned target = (unsigned)((S.chunk_mb0[j + 1] - S.chunk_mb0[j]) * p.nt1 * kEpiWarps);
-                    ok = flag_wait_ge(&p.ctl->y_done[j], target, p, 21);
+    if (warp == 0) {
+        // ---- loader
+        int b = 0;
+        uint32_t ph = 0;
+        int ready_upto = -1;     // chunks [0, ready_upto] are known complete
+        bool ok = true;
+        for (;;) {
+            int q = 0;
+            if (lane == 0) q = (int)atomicAdd(&p.ctl->q_comb, 1u);
+            q = __shfl_sync(0xffffffffu, q, 0);
+            if (q >= S.n_comb) break;
+            const int t0 = q * kCombTile;
+            const int chunk = (((t0 / kRouteBlock) * kFine) / p.nblk) / g;
+            if (chunk > ready_upto) {
+                if (lane == 0) {
+                    const unsigned long long tw0 = trace_now(p);
+                    ok = flag_wait_ge(&p.ctl->fix_done, (unsigned)p.nblk, p, 20);
+                    for (int j = ready_upto + 1; ok && j <= chunk; ++j) {
+                        const unsigned target = (unsigned)((S.chunk_mb0[j + 1] - S.chunk_mb0[j]) * p.nt1 * kEpiWarps);
+                        ok = flag_wait_ge(&p.ctl->y_done[j], target, p, 21);
+                    }
+                    trace_ev(p, S, kEvWaitChunk, (unsigned)chunk, tw0, trace_now(p), 0u);
                 }
-                S.bcast[1] = ok ? 1 : 0;
-                trace_ev(p, S, kEvWaitChunk, (unsigned)chunk, tw0, trace_now(p), 0u);
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                ready_upto = chunk;
             }
-            __syncthreads();
-            if (!S.bcast[1]) break;
-            ready_upto = chunk;
-        }
-        const unsigned long long tc0 = trace_now(p);
-        for (int tt = 0; tt < kCombTile / 8; ++tt) {
-            const int t = t0 + warp * (kCombTile / 8) + tt;
-            if (t >= p.T) break;                                   // warp-uniform
-            if (lane < p.k) {
-                S.crow[warp][lane] = __ldcg(p.row_of + (size_t)t * p.k + lane);
-                S.cgate[warp][lane] = __ldcg(p.gates + (size_t)t * p.k + lane);
-            } else if (lane < kk) {
-                S.crow[warp][lane] = S.offsets[p.E + (lane - p.k)] + t;
-                S.cgate[warp][lane] = 1.0f;
+            const unsigned long long tc0 = trace_now(p);
+            const int ntok = min(kCombTile, p.T - t0);
+            for (int i = lane; i < ntok * kk; i += 32) {
+                const int tt = i / kk, j = i - tt * kk, t = t0 + tt;
+                S.crow[tt][j] = j < p.k ? __ldcg(p.row_of + (size_t)t * p.k + j) : S.offsets[p.E + (j - p.k)] + t;
+                S.cgate[tt][j] = j < p.k ? __ldcg(p.gates + (size_t)t * p.k + j) : 1.0f;
             }
             __syncwarp();
-            for (int v = lane; v < n16; v += 64) {
-                const bool has1 = (v + 32) < n16;
-                float a0[8], a1[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) { a0[i] = 0.f; a1[i] = 0.f; }
-                for (int j0 = 0; j0 < kk; j0 += 4) {
-                    uint4 q0[4], q1[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        if (j0 + u < kk) {
-                            const __nv_bfloat16 *src = p.y + (size_t)S.crow[warp][j0 + u] * p.H + (size_t)v * 8;
-                            q0[u] = ld_cg_v4(src);
-                            if (has1) q1[u] = ld_cg_v4(src + 256);
-                        }
-                    }
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        if (j0 + u < kk) {
-                            const float gw = S.cgate[warp][j0 + u];
-                            a0[0] = fmaf(gw, bf16lo_to_f32(q0[u].x), a0[0]); a0[1] = fmaf(gw, bf16hi_to_f32(q0[u].x), a0[1]);
-                            a0[2] = fmaf(gw, bf16lo_to_f32(q0[u].y), a0[2]); a0[3] = fmaf(gw, bf16hi_to_f32(q0[u].y), a0[3]);
-                            a0[4] = fmaf(gw, bf16lo_to_f32(q0[u].z), a0[4]); a0[5] = fmaf(gw, bf16hi_to_f32(q0[u].z), a0[5]);
-                            a0[6] = fmaf(gw, bf16lo_to_f32(q0[u].w), a0[6]); a0[7] = fmaf(gw, bf16hi_to_f32(q0[u].w), a0[7]);
-                            if (has1) {
-                                a1[0] = fmaf(gw, bf16lo_to_f32(q1[u].x), a1[0]); a1[1] = fmaf(gw, bf16hi_to_f32(q1[u].x), a1[1]);
-                                a1[2] = fmaf(gw, bf16lo_to_f32(q1[u].y), a1[2]); a1[3] = fmaf(gw, bf16hi_to_f32(q1[u].y), a1[3]);
-                                a1[4] = fmaf(gw, bf16lo_to_f32(q1[u].z), a1[4]); a1[5] = fmaf(gw, bf16hi_to_f32(q1[u].z), a1[5]);
-                                a1[6] = fmaf(gw, bf16lo_to_f32(q1[u].w), a1[6]); a1[7] = fmaf(gw, bf16hi_to_f32(q1[u].w), a1[7]);
-                            }
-                        }
+            if (lane == 0) {
+                for (int tt = 0; tt < ntok && ok; ++tt) {
+                    for (int col0 = 0; col0 < p.H; col0 += W) {
+                        const int w = min(W, p.H - col0);
+                        if (!mbar_wait(&S.cb_empty[b], ph ^ 1u, p, 22)) { ok = false; break; }
+                        S.mv[b].a = t0 + tt; S.mv[b].b = col0; S.mv[b].c = w; S.mv[b].d = 0;
+                        for (int j = 0; j < kk; ++j) S.mv[b].g[j] = S.cgate[tt][j];
+                        mbar_arrive_expect_tx(&S.cb_full[b], (uint32_t)(kk * w * 2));
+                        const uint32_t dst = smem_u32(stages + b * kMvBuf);
+                        for (int j = 0; j < kk; ++j)
+                            bulk_load(dst + (uint32_t)(j * w * 2), p.y + (size_t)S.crow[tt][j] * p.H + col0,
+                                      (uint32_t)(w * 2), &S.cb_full[b]);
+                        if (++b == kStages) { b = 0; ph ^= 1u; }
                     }
                 }
-                __nv_bfloat16 *dst = p.out + (size_t)t * p.H + (size_t)v * 8;
-                st_cs_v4(dst, make_uint4(pack_bf16x2(a0[0], a0[1]), pack_bf16x2(a0[2], a0[3]),
-                                         pack_bf16x2(a0[4], a0[5]), pack_bf16x2(a0[6], a0[7])));
-                if (has1)
-                    st_cs_v4(dst + 256, make_uint4(pack_bf16x2(a1[0], a1[1]), pack_bf16x2(a1[2], a1[3]),
-                                                   pack_bf16x2(a1[4], a1[5]), pack_bf16x2(a1[6], a1[7])));
+                trace_ev(p, S, kEvCombine, (unsigned)q, tc0, trace_now(p), 0u);
             }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
             __syncwarp();
         }
-        __syncthreads();
-        if (tid == 0) trace_ev(p, S, kEvCombine, (unsigned)q, tc0, trace_now(p), 0u);
+        if (lane == 0 && ok && mbar_wait(&S.cb_empty[b], ph ^ 1u, p, 23)) {
+            S.mv[b].d = 2;
+            mbar_arrive(&S.cb_full[b]);
+        }
+        __syncwarp();
+    } else if (warp >= 2) {
+        // ---- reducers
+        const int ctid = tid - 64;
+        int b = 0;
+        uint32_t ph = 0;
+        for (;;) {
+            bool ok = mbar_wait(&S.cb_full[b], ph, p, 24);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const MvDesc &d = S.mv[b];
+            if (d.d == 2) break;
+            const int w = d.c, nv = w >> 3;
+            const uint32_t src = smem_u32(stages + b * kMvBuf);
+            __nv_bfloat16 *dst = p.out + (size_t)d.a * p.H + d.b;
+            for (int v = ctid; v < nv; v += kCombWarps * 32) {
+                float a0[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) a0[i] = 0.f;
+                for (int j = 0; j < kk; ++j) {
+                    const uint4 q4 = ld_shared_v4(src + (uint32_t)(j * w * 2 + v * 16));
+                    const float gw = d.g[j];
+                    a0[0] = fmaf(gw, bf16lo_to_f32(q4.x), a0[0]); a0[1] = fmaf(gw, bf16hi_to_f32(q4.x), a0[1]);
+                    a0[2] = fmaf(gw, bf16lo_to_f32(q4.y), a0[2]); a0[3] = fmaf(gw, bf16hi_to_f32(q4.y), a0[3]);
+                    a0[4] = fmaf(gw, bf16lo_to_f32(q4.z), a0[4]); a0[5] = fmaf(gw, bf16hi_to_f32(q4.z), a0[5]);
+                    a0[6] = fmaf(gw, bf16lo_to_f32(q4.w), a0[6]); a0[7] = fmaf(gw, bf16hi_to_f32(q4.w), a0[7]);
+                }
+                st_cs_v4(dst + v * 8, make_uint4(pack_bf16x2(a0[0], a0[1]), pack_bf16x2(a0[2], a0[3]),
+                                                 pack_bf16x2(a0[4], a0[5]), pack_bf16x2(a0[6], a0[7])));
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&S.cb_empty[b]);
+            if (++b == kStages) { b = 0; ph ^= 1u; }
+        }
     }
     __syncthreads();
 }
@@ -820,6 +891,10 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
         for (int i = 0; i < 2; ++i) { mbar_init(&S.tmem_full[i], 1); mbar_init(&S.tmem_empty[i], 2 * kEpiWarps); }
         // tile descriptor consumed: leader's producer + MMA + 4 epilogue warps, peer's producer + 4 warps
         for (int i = 0; i < kTinfo; ++i) { mbar_init(&S.ti_full[i], 1); mbar_init(&S.ti_empty[i], 3 + 2 * kEpiWarps); }
+        for (int i = 0; i < kStages; ++i) {
+            mbar_init(&S.dv_full[i], 1); mbar_init(&S.dv_empty[i], 1);
+            mbar_init(&S.cb_full[i], 1); mbar_init(&S.cb_empty[i], kCombWarps);
+        }
         fence_mbar_init();
         tma_prefetch_desc(&tm_xe); tma_prefetch_desc(&tm_wgu); tma_prefetch_desc(&tm_h); tma_prefetch_desc(&tm_wd);
     }
@@ -1049,17 +1124,17 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
     PipeState ps;
     if (alive) {
         if (p.mode == kModeSerial) {
-            dispatch_phase(p, S);
+            dispatch_phase(p, S, stages);
             alive = grid_barrier(p, S, 2u * n_sm, 2);
             if (alive) gemm_phase(p, S, stages, tmem_base, &tm_xe, &tm_wgu, &tm_h, &tm_wd, 0x7fffffff, ps);
             alive = alive && grid_barrier(p, S, 3u * n_sm, 3);
-            if (alive) combine_phase(p, S);
+            if (alive) combine_phase(p, S, stages);
         } else {
             const bool mover = (int)blockIdx.x < plan_c;      // role from c* and the block index
-            if (mover) dispatch_phase(p, S);
+            if (mover) dispatch_phase(p, S, stages);
             const int budget = mover ? plan_steal : 0x7fffffff;
             if (budget > 0) gemm_phase(p, S, stages, tmem_base, &tm_xe, &tm_wgu, &tm_h, &tm_wd, budget, ps);
-            combine_phase(p, S);
+            combine_phase(p, S, stages);
         }
     }
 

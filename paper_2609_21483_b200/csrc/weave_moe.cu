@@ -29,6 +29,7 @@ bool shape_ok(const weave_moe_config *c)
 {
     if (!c) return false;
     if (c->hidden < 128 || c->hidden % 128 || c->ffn < 128 || c->ffn % 128) return false;
+    if (c->hidden > 16384) return false;     // one bf16 row must fit a 32 KB movement buffer
     if (c->num_experts < 1 || c->num_shared < 0 || c->num_experts + c->num_shared > kMaxEE) return false;
     if (c->top_k < 1 || c->top_k > c->num_experts || c->top_k > kMaxTopK || c->num_shared > 8) return false;
     if (c->max_tokens < 1 || c->max_tokens > (1 << 20)) return false;
