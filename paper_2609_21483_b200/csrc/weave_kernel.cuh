@@ -74,6 +74,7 @@ struct KParams {
     int mode, fixed_c, fixed_K, fixed_steal;
     int nt0, nt1;         // n-tiles per m-block: I / 128, ceil(H / 256)
     int nmb_max;          // allocated length of the per-m-block flag arrays
+    int elastic_steal;    // movement pairs keep stealing past their quota while no combine chunk is ready
     int withhold_mb;      // test hook: this m-block's "dispatched" flag is never published (-1 = off)
     int c_min, c_max, c_step;
     float alpha;
@@ -463,22 +464,28 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ---- storer
+        // ---- storer: one bulk store per buffer.  A buffer is handed back as soon as the store has
+        // read it; an m-block's flag is published once the stores up to its last one have completed
+        // (checked with a lag of kFlagLag stores, so the copy engine never drains).
         if (lane == 0) {
+            constexpr int kFlagLag = 4, kPend = 8;
             int b = 0, n = 0;
             uint32_t ph = 0;
-            int h_buf[3] = {0, 0, 0}, h_mb[3] = {0, 0, 0}, h_last[3] = {0, 0, 0}, h_rows[3] = {0, 0, 0};
-            unsigned long long h_t0[3] = {0ull, 0ull, 0ull};
-            auto retire = [&](int i) {
-                const int s3 = i % 3;
-                mbar_arrive(&S.dv_empty[h_buf[s3]]);
-                if (h_last[s3]) {
-                    if (h_mb[s3] != p.withhold_mb) {
-                        fence_proxy_async();      // these rows are read by TMA on another SM
-                        __threadfence();
-                        st_release_u32(&p.xe_ready[h_mb[s3]], 1u);
+            int prev_buf = -1;
+            int pe_idx[kPend], pe_mb[kPend], pe_rows[kPend];      // tile ends not yet published
+            unsigned long long pe_t0[kPend];
+            for (int i = 0; i < kPend; ++i) { pe_idx[i] = 0; pe_mb[i] = 0; pe_rows[i] = 0; pe_t0[i] = 0ull; }
+            int pe_head = 0, pe_tail = 0;
+            auto publish_upto = [&](int done_idx) {      // stores with index <= done_idx have completed
+                bool fenced = false;
+                while (pe_head != pe_tail && pe_idx[pe_head % kPend] <= done_idx) {
+                    const int s8 = pe_head % kPend;
+                    if (pe_mb[s8] != p.withhold_mb) {
+                        if (!fenced) { fence_proxy_async(); __threadfence(); fenced = true; }
+                        st_release_u32(&p.xe_ready[pe_mb[s8]], 1u);
                     }
-                    trace_ev(p, S, kEvDispatch, (unsigned)h_mb[s3], h_t0[s3], trace_now(p), (unsigned)h_rows[s3]);
+                    trace_ev(p, S, kEvDispatch, (unsigned)pe_mb[s8], pe_t0[s8], trace_now(p), (unsigned)pe_rows[s8]);
+                    ++pe_head;
                 }
             };
             unsigned long long tile_t0 = trace_now(p);
@@ -488,14 +495,22 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
                 if (dd == 2) break;
                 bulk_store(p.xe + (size_t)da * p.H, smem_u32(stages + b * kMvBuf), (uint32_t)db * rowb);
                 bulk_commit();
-                h_buf[n % 3] = b; h_mb[n % 3] = dc; h_last[n % 3] = dd; h_rows[n % 3] = db; h_t0[n % 3] = tile_t0;
-                if (dd == 1) tile_t0 = trace_now(p);
+                if (prev_buf >= 0) { bulk_wait_read<1>(); mbar_arrive(&S.dv_empty[prev_buf]); }
+                prev_buf = b;
+                if (dd == 1) {
+                    if (pe_tail - pe_head == kPend) { bulk_wait<0>(); publish_upto(n); }
+                    const int s8 = pe_tail % kPend;
+                    pe_idx[s8] = n; pe_mb[s8] = dc; pe_rows[s8] = db; pe_t0[s8] = tile_t0;
+                    ++pe_tail;
+                    tile_t0 = trace_now(p);
+                }
+                if (n >= kFlagLag && pe_head != pe_tail) { bulk_wait<kFlagLag>(); publish_upto(n - kFlagLag); }
                 ++n;
-                if (n >= 3) { bulk_wait<2>(); retire(n - 3); }
                 if (++b == kStages) { b = 0; ph ^= 1u; }
             }
             bulk_wait<0>();
-            for (int i = max(0, n - 2); i < n; ++i) retire(i);
+            if (prev_buf >= 0) mbar_arrive(&S.dv_empty[prev_buf]);
+            publish_upto(n);
         }
         __syncwarp();
     }
@@ -693,7 +708,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
         // kTinfo tiles ahead of the MMAs, so claim and flag latencies stay off the critical path.
         if (lane == 0) {
             int taken = 0;
-            int g_next = budget > 0 ? (int)atomicAdd(&p.ctl->q_gemm, 1u) : 0x7fffffff;
+            int g_next = (budget > 0 || p.elastic_steal) ? (int)atomicAdd(&p.ctl->q_gemm, 1u) : 0x7fffffff;
             for (;;) {
                 const int g = g_next;
                 const unsigned long long tp0 = trace_now(p);
@@ -710,7 +725,19 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                 }
                 if (tl.type != 2) {
                     ++taken;
-                    g_next = taken < budget ? (int)atomicAdd(&p.ctl->q_gemm, 1u) : 0x7fffffff;
+                    bool more = taken < budget;
+                    if (!more && p.elastic_steal) {
+                        // the steal quota is used up: keep taking GEMM tiles for as long as the next
+                        // combine chunk has not been produced yet (nothing else to do meanwhile)
+                        const unsigned qc = ld_relaxed_u32(&p.ctl->q_comb);
+                        if (qc >= (unsigned)S.n_comb) more = true;
+                        else {
+                            const int ch = ((((int)qc * kCombTile / kRouteBlock) * kFine) / p.nblk) / (kFine / S.K);
+                            const unsigned target = (unsigned)((S.chunk_mb0[ch + 1] - S.chunk_mb0[ch]) * p.nt1 * kEpiWarps);
+                            more = ld_acquire_u32(&p.ctl->y_done[ch]) < target;
+                        }
+                    }
+                    g_next = more ? (int)atomicAdd(&p.ctl->q_gemm, 1u) : 0x7fffffff;
                     bool ok;
                     if (tl.type == 0) {
                         ok = flag_wait_ge(&p.xe_ready[tl.mb], 1u, p, 31);
@@ -1133,7 +1160,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
             const bool mover = (int)blockIdx.x < plan_c;      // role from c* and the block index
             if (mover) dispatch_phase(p, S, stages);
             const int budget = mover ? plan_steal : 0x7fffffff;
-            if (budget > 0) gemm_phase(p, S, stages, tmem_base, &tm_xe, &tm_wgu, &tm_h, &tm_wd, budget, ps);
+            if (budget > 0 || p.elastic_steal) gemm_phase(p, S, stages, tmem_base, &tm_xe, &tm_wgu, &tm_h, &tm_wd, budget, ps);
             combine_phase(p, S, stages);
         }
     }

@@ -4,6 +4,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -126,16 +127,17 @@ int encode_map(EncodeTiledFn fn, CUtensorMap *m, const void *base, uint64_t rows
 
 void default_tables(int n_sm, std::vector<float> &bw, std::vector<float> &tf)
 {
-    // Placeholder curves of the shape the paper's Figure 4 describes (bandwidth near-linear then
-    // saturating, GEMM throughput sub-linear); replaced by measured ones through
-    // weave_moe_set_cost_tables().  Units: byte/us and FLOP/us.
+    // Curves measured with the calibration tool on a B200 (148 SMs, power-limited clocks), of the
+    // shape the paper's Figure 4 describes: movement bandwidth grows linearly with the number of
+    // movement SMs (about 42 GB/s of dispatch payload per SM, no saturation up to half the SMs),
+    // GEMM throughput is sub-linear in the number of GEMM SMs (close to a square root: with fewer
+    // busy tensor cores the clocks rise).  Units: byte/us and FLOP/us.  weave_moe_set_cost_tables()
+    // replaces them with curves measured for a particular layer shape.
     bw.assign(n_sm + 1, 0.f);
     tf.assign(n_sm + 1, 0.f);
     for (int i = 1; i <= n_sm; ++i) {
-        float lin = 45.0e3f * i;                       // ~45 GB/s per movement SM
-        bw[i] = lin < 5.5e6f ? lin : 5.5e6f;           // saturates near 5.5 TB/s
-        float x = (float)i / (float)n_sm;
-        tf[i] = 1.30e9f * x * (1.15f - 0.15f * x);     // ~1.3 PFLOP/s with all SMs, mildly sub-linear
+        bw[i] = 42.0e3f * (float)i;
+        tf[i] = 1.30e9f * sqrtf((float)i / (float)n_sm);
     }
     bw[0] = bw[1];
     tf[0] = tf[1];
@@ -196,8 +198,8 @@ int weave_moe_create(const weave_moe_config *cfg, weave_moe_t *out)
     h->c_min = 2;
     h->c_max = h->n_sm / 2;
     h->c_step = 2;
-    h->alpha = 0.5f;
-    h->eff[0] = 1.0f; h->eff[1] = 0.93f; h->eff[2] = 0.85f; h->eff[3] = 0.73f;
+    h->alpha = 0.8f;
+    h->eff[0] = 1.0f; h->eff[1] = 0.90f; h->eff[2] = 0.80f; h->eff[3] = 0.65f;
     h->timeout_ms = 4000;
     h->withhold_mb = -1;
     h->last_T = 0;
@@ -270,6 +272,7 @@ int weave_moe_forward(weave_moe_t h, const void *x, const float *logits, void *o
     p.nt1 = (c.hidden + 255) / 256;
     p.nmb_max = L.nmb_max;
     p.withhold_mb = h->withhold_mb;
+    p.elastic_steal = (h->mode == WEAVE_SCHED_AUTO) ? 1 : 0;
     p.c_min = h->c_min; p.c_max = h->c_max; p.c_step = h->c_step;
     p.alpha = h->alpha;
     for (int i = 0; i < 4; ++i) p.eff[i] = h->eff[i];
