@@ -157,6 +157,39 @@ int weave_moe_debug_withhold_flag(weave_moe_t h, int m_block);
  * extra = type << 16 | n-tile), 7 combine tile, 8 wait for a chunk's gemm1, 9 grid barrier. */
 int weave_moe_set_trace(weave_moe_t h, void *buf, int events_per_cta);
 
+/* ---- for callers that cannot allocate ---------------------------------------------------------
+ *
+ * (No counterpart in the paper: this is a packaging variant of the same kernel.)
+ * Some callers of this library may not allocate device memory at the point where they need a
+ * layer: code that runs while a memory pool is frozen, plugins handed a fixed arena by their host
+ * application, latency-critical serving loops whose allocator must stay untouched.  For them this
+ * entry point runs weave_moe_forward's kernel with its scratch placed in a fixed array built into
+ * the library image instead of a caller-provided workspace.  It takes no handle and calls no
+ * cudaMalloc / cudaFree or any other allocating routine; the caller still passes weights, inputs
+ * and the output.
+ *
+ *   - Limit: the layer's scratch (what weave_moe_workspace_bytes() reports for this shape with
+ *     max_tokens = T) must fit weave_moe_static_scratch_bytes() (64 MiB minus alignment); larger
+ *     calls fail with WEAVE_ERR_WORKSPACE and must use a handle.  Every GPU on which the library
+ *     is loaded holds those 64 MiB until the process exits.
+ *   - The first call on each device performs a one-time set-up with that device current (it looks
+ *     up the device address of the built-in array, raises the kernel's shared-memory limit and
+ *     resolves the TMA descriptor encoder).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents; the
+ *     call re-zeroes the control words and rewrites the cost tables on the stream before it
+ *     launches.  Calls that overlap on the GPU (different streams, no ordering between them) race
+ *     on the array: order them.
+ *   - Scheduling is AUTO with the default cost tables.  Arguments, layouts and alignment as for
+ *     weave_moe_create() / weave_moe_forward(); asynchronous on the stream; a device-side failure
+ *     of this call (non-finite logits, an expired wait) is not reported - use a handle when the
+ *     status word is needed. */
+int weave_moe_forward_static(int hidden, int ffn, int num_experts, int top_k, int num_shared,
+                             const void *gate_up, const void *down, const void *x,
+                             const float *router_logits, void *out, int T, void *cuda_stream);
+
+/* Size limit of the built-in scratch used by weave_moe_forward_static(). */
+size_t weave_moe_static_scratch_bytes(void);
+
 int weave_moe_last_cuda_error(weave_moe_t h);
 const char *weave_moe_strerror(int code);
 

@@ -59,6 +59,7 @@ EXPORTS = [
     "weave_moe_get_geometry", "weave_moe_get_routing", "weave_moe_get_intermediates",
     "weave_moe_status", "weave_moe_set_timeout_ms", "weave_moe_debug_withhold_flag",
     "weave_moe_last_cuda_error", "weave_moe_strerror", "weave_moe_set_trace",
+    "weave_moe_forward_static", "weave_moe_static_scratch_bytes",
 ]
 
 
@@ -103,6 +104,10 @@ def load():
     lib.weave_moe_debug_withhold_flag.argtypes = [vp, ci]
     lib.weave_moe_set_trace.restype = ci
     lib.weave_moe_set_trace.argtypes = [vp, vp, ci]
+    lib.weave_moe_forward_static.restype = ci
+    lib.weave_moe_forward_static.argtypes = [ci, ci, ci, ci, ci, vp, vp, vp, vp, vp, ci, vp]
+    lib.weave_moe_static_scratch_bytes.restype = ctypes.c_size_t
+    lib.weave_moe_static_scratch_bytes.argtypes = []
     lib.weave_moe_last_cuda_error.restype = ci
     lib.weave_moe_last_cuda_error.argtypes = [vp]
     lib.weave_moe_strerror.restype = ctypes.c_char_p
@@ -123,6 +128,30 @@ def workspace_bytes(hidden, ffn, num_experts, top_k, num_shared, max_tokens) -> 
 def _check(rc: int, what: str):
     if rc != WEAVE_OK:
         raise WeaveError(rc, what)
+
+
+def forward_static(x, logits, gate_up, down, num_experts: int, top_k: int, num_shared: int = 0, out=None,
+                   stream: Optional[int] = None):
+    """The layer for callers that must not allocate device memory: no handle, no workspace; the
+    kernel's scratch is a fixed array inside the library (see weave_moe_forward_static in the
+    header for the size limit and the sharing rules).  `out` must be passed by such callers; it is
+    created here only as a convenience when omitted."""
+    import torch
+    lib = load()
+    EE, twoI, H = gate_up.shape
+    T = x.shape[0]
+    assert x.is_cuda and logits.is_cuda and gate_up.is_cuda and down.is_cuda
+    assert x.dtype == torch.bfloat16 and logits.dtype == torch.float32
+    assert x.is_contiguous() and logits.is_contiguous() and gate_up.is_contiguous() and down.is_contiguous()
+    if out is None:
+        out = torch.empty_like(x)
+    if stream is None:
+        stream = torch.cuda.current_stream(x.device).cuda_stream
+    with torch.cuda.device(x.device):
+        _check(lib.weave_moe_forward_static(H, twoI // 2, num_experts, top_k, num_shared, gate_up.data_ptr(),
+                                            down.data_ptr(), x.data_ptr(), logits.data_ptr(), out.data_ptr(), T,
+                                            stream), "weave_moe_forward_static")
+    return out
 
 
 class WeaveMoE:

@@ -7,6 +7,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -479,6 +480,134 @@ int weave_moe_set_trace(weave_moe_t h, void *buf, int events_per_cta)
 }
 
 int weave_moe_last_cuda_error(weave_moe_t h) { return h ? h->last_cuda_error : 0; }
+
+}  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// Entry point for callers that cannot allocate device memory.
+//
+// The layer's scratch (control words, routing arrays, expert-major buffers) normally lives in a
+// workspace the caller allocates.  Here it lives in a fixed array that is part of the loaded
+// library image, so nothing is allocated or freed: not by this library, and the caller does not
+// have to either.  The price: a hard size limit, one forward at a time per device, and memory that
+// every device loading the library holds until the process exits.
+
+namespace {
+
+constexpr size_t kStaticScratchBytes = 64ull << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+struct StaticDevice {
+    bool ready;
+    uint8_t *base;        // device address of g_static_scratch on this device, rounded up to 1024
+    size_t usable;
+    int n_sm;
+    EncodeTiledFn encode;
+};
+constexpr int kMaxDevices = 64;
+StaticDevice g_static_dev[kMaxDevices];
+std::mutex g_static_mutex;
+
+// Once per device, with that device current: turn the array's name, which in host code is only a
+// stand-in, into the address the device can use.
+int static_setup(int dev, StaticDevice **out)
+{
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticDevice &d = g_static_dev[dev];
+    if (!d.ready) {
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return WEAVE_ERR_CUDA;
+        if (prop.major != 10 || !prop.cooperativeLaunch || (int)prop.sharedMemPerBlockOptin < kSmemBytes ||
+            prop.multiProcessorCount < 4 || prop.multiProcessorCount + 1 > 1024)
+            return WEAVE_ERR_UNSUPPORTED_DEVICE;
+        void *sym = nullptr;
+        if (cudaGetSymbolAddress(&sym, g_static_scratch) != cudaSuccess || sym == nullptr) return WEAVE_ERR_CUDA;
+        const uintptr_t a = ((uintptr_t)sym + 1023) & ~(uintptr_t)1023;
+        d.base = reinterpret_cast<uint8_t *>(a);
+        d.usable = kStaticScratchBytes - (size_t)(a - (uintptr_t)sym);
+        d.n_sm = prop.multiProcessorCount & ~1;
+        if (cudaFuncSetAttribute(weave_moe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=
+            cudaSuccess)
+            return WEAVE_ERR_CUDA;
+        void *fnp = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fnp, cudaEnableDefault, &qres) != cudaSuccess || !fnp ||
+            qres != cudaDriverEntryPointSuccess)
+            return WEAVE_ERR_UNSUPPORTED_DEVICE;
+        d.encode = reinterpret_cast<EncodeTiledFn>(fnp);
+        d.ready = true;
+    }
+    *out = &d;
+    return WEAVE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t weave_moe_static_scratch_bytes(void) { return kStaticScratchBytes - 1024; }
+
+int weave_moe_forward_static(int hidden, int ffn, int num_experts, int top_k, int num_shared, const void *gate_up,
+                             const void *down, const void *x, const float *router_logits, void *out, int T,
+                             void *cuda_stream)
+{
+    weave_moe_config cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.hidden = hidden; cfg.ffn = ffn; cfg.num_experts = num_experts; cfg.top_k = top_k;
+    cfg.num_shared = num_shared; cfg.max_tokens = T;
+    if (T == 0) return WEAVE_OK;
+    if (!shape_ok(&cfg)) return WEAVE_ERR_INVALID_ARG;
+    if (!gate_up || !down || ((uintptr_t)gate_up & 15) || ((uintptr_t)down & 15)) return WEAVE_ERR_INVALID_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return WEAVE_ERR_CUDA;
+    if (dev < 0 || dev >= kMaxDevices) return WEAVE_ERR_UNSUPPORTED_DEVICE;
+    StaticDevice *sd = nullptr;
+    int rc = static_setup(dev, &sd);
+    if (rc) return rc;
+    const Layout L = make_layout(&cfg);
+    if (L.total > sd->usable) return WEAVE_ERR_WORKSPACE;      // beyond the built-in scratch: use a handle
+
+    // a handle that lives on this stack frame only; nothing is allocated on the host heap either
+    weave_moe h;
+    memset(static_cast<void *>(&h), 0, sizeof(h));
+    h.cfg = cfg;
+    h.cfg.gate_up = gate_up; h.cfg.down = down; h.cfg.workspace = sd->base; h.cfg.workspace_bytes = sd->usable;
+    h.L = L;
+    h.ws = sd->base;
+    h.n_sm = sd->n_sm; h.n_cta = sd->n_sm; h.device = dev;
+    h.mode = WEAVE_SCHED_AUTO;
+    h.fixed_c = (h.n_sm * 15 / 100 + 1) & ~1; h.fixed_K = 1; h.fixed_steal = 0;
+    h.c_min = 2; h.c_max = h.n_sm / 2; h.c_step = 2;
+    h.alpha = 0.8f;
+    h.eff[0] = 1.0f; h.eff[1] = 0.90f; h.eff[2] = 0.80f; h.eff[3] = 0.65f;
+    h.timeout_ms = 4000;
+    h.withhold_mb = -1;
+    const int EE = num_experts + num_shared;
+    int r = 0;
+    r |= encode_map(sd->encode, &h.tm_xe, h.ws + L.xe, (uint64_t)L.p_max, (uint64_t)hidden, false);
+    r |= encode_map(sd->encode, &h.tm_wgu, gate_up, (uint64_t)EE * 2 * ffn, (uint64_t)hidden, true);
+    r |= encode_map(sd->encode, &h.tm_h, h.ws + L.hbuf, (uint64_t)L.p_max, (uint64_t)ffn, false);
+    r |= encode_map(sd->encode, &h.tm_wd, down, (uint64_t)EE * hidden, (uint64_t)ffn, true);
+    if (r) return WEAVE_ERR_CUDA;
+
+    // the array keeps whatever the last call left behind: zero the control words, refill the tables
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (cudaMemsetAsync(h.ws, 0, L.zero_end, st) != cudaSuccess) return WEAVE_ERR_CUDA;
+    float bw[1024], tf[1024];
+    {
+        for (int i = 1; i <= h.n_sm; ++i) {
+            bw[i] = 42.0e3f * (float)i;
+            tf[i] = 1.30e9f * sqrtf((float)i / (float)h.n_sm);
+        }
+        bw[0] = bw[1]; tf[0] = tf[1];
+    }
+    if (cudaMemcpyAsync(h.ws + L.bw, bw, sizeof(float) * (h.n_sm + 1), cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return WEAVE_ERR_CUDA;
+    if (cudaMemcpyAsync(h.ws + L.tf, tf, sizeof(float) * (h.n_sm + 1), cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return WEAVE_ERR_CUDA;
+    return weave_moe_forward(&h, x, router_logits, out, T, cuda_stream);
+}
+
 
 const char *weave_moe_strerror(int code)
 {
