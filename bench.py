@@ -222,7 +222,7 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
     sched = {"auto": (pk.SCHED_AUTO, 0, 1, 0), "serial": (pk.SCHED_SERIAL, 0, 1, 0)}
     geo = moe.geometry()
-    fixed_c = max(1, int(round(0.15 * geo["n_sm"])))
+    fixed_c = max(2, int(round(0.15 * geo["n_sm"])))
     sched["fixed"] = (pk.SCHED_FIXED, fixed_c, 1, 0)
 
     def step_dev():
@@ -265,12 +265,18 @@ def run_ours(args):
     moe.check()
 
     ablation = {}
-    if rank == 0 and not args.no_ablation:
-        for name in ("auto", "fixed", "serial"):
-            moe.set_schedule(*sched[name])
-            s = timed(step_dev, max(3, min(args.steps, 10)), 3) if world == 1 else None
-            if s is not None:
-                ablation[name + "_us_per_layer"] = s / max(3, min(args.steps, 10)) / L * 1e6
+    if rank == 0 and not args.no_ablation and world == 1:
+        # the three schedules take turns (round robin), so that clock / power drift over the run
+        # hits them alike
+        n_abl, rounds = max(2, min(args.steps, 5)), 3
+        tot = {"auto": 0.0, "fixed": 0.0, "serial": 0.0}
+        for _ in range(rounds):
+            for name in tot:
+                moe.set_schedule(*sched[name])
+                tot[name] += timed(step_dev, n_abl, 1)
+        for name, s in tot.items():
+            ablation[name + "_us_per_layer"] = s / (n_abl * rounds) / L * 1e6
+        ablation["fixed_c"] = fixed_c
         moe.set_schedule(*sched[args.sched])
         moe.check()
 

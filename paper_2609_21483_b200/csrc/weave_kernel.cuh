@@ -104,7 +104,8 @@ struct KParams {
 };
 
 struct TileInfo {
-    int type;   // 0 gemm0 (+SwiGLU), 1 gemm1, 2 no more tiles
+    int type;   // 0 gemm0 (+SwiGLU), 1 gemm1, 2 no more tiles; 3 / 4 = gemm0 / gemm1 of a single m-block
+                // with the operands swapped (weights on the MMA's M axis, the m-block's rows on N)
     int mb;     // this CTA's m-block (-1: the pair tile has no second half)
     int row0;   // first row of this CTA's 128 rows of A
     int nrows;  // valid rows (0 for a missing half)
@@ -128,6 +129,7 @@ struct SmemTail {
     uint64_t ti_full[kTinfo], ti_empty[kTinfo];
     uint64_t dv_full[kStages], dv_empty[kStages];   // dispatch: loader -> storer ring over the stage buffers
     uint64_t cb_full[kStages], cb_empty[kStages];   // combine: loader -> reducing warps
+    uint64_t xg_full, xg_empty;                     // swapped gemm0 epilogue: up warps -> gate warps
     TileInfo ti[kTinfo];
     MvDesc mv[kStages];
     uint32_t tmem_base;
@@ -140,6 +142,7 @@ struct SmemTail {
     unsigned trace_n;
     int chunk_mb0[kFine + 1];
     int chunk_pt0[kFine + 1];
+    int chunk_nswap[kFine];      // per chunk: segments with an odd number of m-blocks
     int chunk_tile0[kFine + 1];
     int offsets[kMaxEE + 1];
     int tok[kBM];
@@ -408,9 +411,23 @@ __device__ __forceinline__ void decode_pair_tile(const SmemTail &S, const KParam
     lead.mb = S.seg_mb0[s] + m0;
     lead.row0 = S.seg_row0[s] + m0 * kBM;
     lead.nrows = min(kBM, rows - m0 * kBM);
-    peer.nrows = max(0, min(kBM, rows - (m0 + 1) * kBM));
-    peer.mb = peer.nrows > 0 ? lead.mb + 1 : -1;
+    if (rows - (m0 + 1) * kBM <= 0) {
+        // the segment's last, unpaired m-block: both CTAs work on it with the operands swapped,
+        // so the MMA costs ceil(nrows/16)*16 columns instead of a half-empty 256-row tile
+        lead.type = type + 3;
+        peer = lead;
+        return;
+    }
+    peer.nrows = min(kBM, rows - (m0 + 1) * kBM);
+    peer.mb = lead.mb + 1;
     peer.row0 = lead.row0 + kBM;
+}
+
+// epilogue-warp arrivals on y_done[j] when all gemm1 tiles of chunk j are finished: 4 per (m-block,
+// n-tile); an m-block processed as a swapped tile is finished by both CTAs of the pair (8)
+__device__ __forceinline__ unsigned y_done_target(const SmemTail &S, const KParams &p, int j)
+{
+    return (unsigned)(((S.chunk_mb0[j + 1] - S.chunk_mb0[j]) + S.chunk_nswap[j]) * p.nt1 * kEpiWarps);
 }
 
 // ------------------------------------------------------------------------------------ phase A: dispatch
@@ -549,8 +566,7 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uin
                     const unsigned long long tw0 = trace_now(p);
                     ok = flag_wait_ge(&p.ctl->fix_done, (unsigned)p.nblk, p, 20);
                     for (int j = ready_upto + 1; ok && j <= chunk; ++j) {
-                        const unsigned target = (unsigned)((S.chunk_mb0[j + 1] - S.chunk_mb0[j]) * p.nt1 * kEpiWarps);
-                        ok = flag_wait_ge(&p.ctl->y_done[j], target, p, 21);
+                        ok = flag_wait_ge(&p.ctl->y_done[j], y_done_target(S, p, j), p, 21);
                     }
                     trace_ev(p, S, kEvWaitChunk, (unsigned)chunk, tw0, trace_now(p), 0u);
                 }
@@ -694,8 +710,8 @@ __device__ __forceinline__ void staged_store_32x32(uint32_t stg, int lane, const
 // Called by both CTAs of a pair with the same arguments.
 __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_t *stages, uint32_t tmem_base,
                                            const CUtensorMap *tm_xe, const CUtensorMap *tm_wgu,
-                                           const CUtensorMap *tm_h, const CUtensorMap *tm_wd, int budget,
-                                           PipeState &ps)
+                                           const CUtensorMap *tm_h, const CUtensorMap *tm_wd,
+                                           const CUtensorMap *tm_wgu64, int budget, PipeState &ps)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = cluster_ctarank();      // 0 = leader (issues the MMAs), 1 = peer
@@ -733,19 +749,19 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                         if (qc >= (unsigned)S.n_comb) more = true;
                         else {
                             const int ch = ((((int)qc * kCombTile / kRouteBlock) * kFine) / p.nblk) / (kFine / S.K);
-                            const unsigned target = (unsigned)((S.chunk_mb0[ch + 1] - S.chunk_mb0[ch]) * p.nt1 * kEpiWarps);
-                            more = ld_acquire_u32(&p.ctl->y_done[ch]) < target;
+                            more = ld_acquire_u32(&p.ctl->y_done[ch]) < y_done_target(S, p, ch);
                         }
                     }
                     g_next = more ? (int)atomicAdd(&p.ctl->q_gemm, 1u) : 0x7fffffff;
                     bool ok;
-                    if (tl.type == 0) {
+                    const bool two = tp.mb != tl.mb;         // a regular pair tile has two m-blocks
+                    if (tl.type == 0 || tl.type == 3) {
                         ok = flag_wait_ge(&p.xe_ready[tl.mb], 1u, p, 31);
-                        if (ok && tp.nrows > 0) ok = flag_wait_ge(&p.xe_ready[tp.mb], 1u, p, 31);
+                        if (ok && two) ok = flag_wait_ge(&p.xe_ready[tp.mb], 1u, p, 31);
                     } else {
                         const unsigned need = (unsigned)(p.nt0 * kEpiWarps);
                         ok = flag_wait_ge(&p.h_ready[tl.mb], need, p, 32);
-                        if (ok && tp.nrows > 0) ok = flag_wait_ge(&p.h_ready[tp.mb], need, p, 32);
+                        if (ok && two) ok = flag_wait_ge(&p.h_ready[tp.mb], need, p, 32);
                     }
                     if (!ok) break;
                     trace_ev(p, S, kEvGemmLoad, (unsigned)g, tp0, trace_now(p), 0u);
@@ -769,20 +785,33 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                 if (ti.type == 2) break;
                 fence_proxy_async();     // rows written with ordinary stores elsewhere, read by TMA here
                 const CUtensorMap *tma_a, *tma_b;
-                int brow;
+                int arow, brow, arow2 = -1;
+                const int nhalf = (((ti.nrows + 15) >> 4) << 4) >> 1;     // swapped tiles: rows per CTA on the N axis
                 if (ti.type == 0) {      // leader holds the gate rows of the n-tile, peer the up rows
                     tma_a = tm_xe; tma_b = tm_wgu;
+                    arow = ti.row0;
                     brow = ti.e * 2 * p.I + ti.n * kTN0 + (int)rank * p.I;
-                } else {                 // 256 output columns: leader the first 128 weight rows, peer the rest
+                } else if (ti.type == 1) {   // 256 output columns: leader the first 128 weight rows, peer the rest
                     tma_a = tm_h; tma_b = tm_wd;
+                    arow = ti.row0;
                     brow = ti.e * p.H + ti.n * 256 + (int)rank * 128;
+                } else if (ti.type == 3) {   // M axis: 64 gate rows then 64 up rows of this CTA's 64 h-columns
+                    tma_a = tm_wgu64; tma_b = tm_xe;
+                    arow = ti.e * 2 * p.I + ti.n * kTN0 + (int)rank * 64;
+                    arow2 = arow + p.I;
+                    brow = ti.row0 + (int)rank * nhalf;
+                } else {                     // M axis: this CTA's 128 of the n-tile's 256 out-columns
+                    tma_a = tm_wd; tma_b = tm_h;
+                    arow = ti.e * p.H + ti.n * 256 + (int)rank * 128;
+                    brow = ti.row0 + (int)rank * nhalf;
                 }
                 for (int kb = 0; kb < ti.nkb; ++kb) {
                     if (!mbar_wait(&S.empty[ps.stage], ps.stage_phase ^ 1u, p, 33)) { dead = true; break; }
                     uint8_t *sa = stages + ps.stage * kStageBytes;
                     const uint32_t lbar = mapa_u32(smem_u32(&S.full[ps.stage]), 0u);
                     if (rank == 0) mbar_arrive_expect_tx(&S.full[ps.stage], 2u * kStageBytes);
-                    tma_load_2d_pair(sa, tma_a, kb * kBK, ti.row0, lbar);
+                    tma_load_2d_pair(sa, tma_a, kb * kBK, arow, lbar);
+                    if (arow2 >= 0) tma_load_2d_pair(sa + kStageA / 2, tma_a, kb * kBK, arow2, lbar);
                     tma_load_2d_pair(sa + kStageA, tma_b, kb * kBK, brow, lbar);
                     ps.next_stage();
                 }
@@ -794,13 +823,14 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
         // ---------------- MMA issuer (leader only): one thread drives both SMs' tensor cores
         if (lane == 0) {
             bool dead = false;
-            const uint32_t idesc = umma_idesc_bf16(2 * kBM, 256u);
             while (!dead) {
                 if (!mbar_wait(&S.ti_full[ps.slot], ps.slot_phase, p, 40)) { dead = true; break; }
                 const TileInfo ti = S.ti[ps.slot];
                 mbar_arrive(&S.ti_empty[ps.slot]);
                 ps.next_slot();
                 if (ti.type == 2) break;
+                // regular tiles: 256 rows x 256 columns; swapped tiles: 256 weight rows x (rows rounded up to 16)
+                const uint32_t idesc = umma_idesc_bf16(2 * kBM, ti.type >= 3 ? (uint32_t)(((ti.nrows + 15) >> 4) << 4) : 256u);
                 if (!mbar_wait_cluster(&S.tmem_empty[ps.acc], ps.acc_phase ^ 1u, p, 41)) { dead = true; break; }
                 tc_fence_after();
                 const uint32_t d = tmem_base + (uint32_t)ps.acc * 256u;
@@ -828,6 +858,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
         const int q = warp & 3;                      // TMEM lane quadrant this warp may read
         const uint32_t stg = smem_u32(stages + kStages * kStageBytes) + (uint32_t)q * 2048u;
         bool dead = false;
+        uint32_t xg_phase = 0;
         while (!dead) {
             if (!mbar_wait_cluster(&S.ti_full[ps.slot], ps.slot_phase, p, 50)) { dead = true; }
             dead = __any_sync(0xffffffffu, dead);
@@ -844,7 +875,68 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
             const unsigned long long te0 = trace_now(p);
             const int rows_valid = ti.nrows - q * 32;          // rows of this warp's quadrant that exist
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)ps.acc * 256u;
-            if (rows_valid > 0) {
+            if (ti.type == 3) {
+                // swapped gemm0: lanes 0..63 hold the gate projection of this CTA's 64 h-columns, lanes
+                // 64..127 the up projection; TMEM columns are the m-block's rows.  The up warps hand
+                // their values to the gate warps through the staging buffer, 16 rows at a time.
+                const uint32_t xs = smem_u32(stages + kStages * kStageBytes);            // [64][16] fp32
+                const int col = ti.n * kTN0 + (int)rank * 64 + (q & 1) * 32 + lane;      // this thread's h-column
+                const int nch = (ti.nrows + 15) >> 4;
+                for (int c = 0; c < nch && !dead; ++c) {
+                    uint32_t v[16];
+                    tmem_ld_32x16(taddr + c * 16, v);
+                    tmem_ld_wait();
+                    if (q >= 2) {
+                        if (!mbar_wait(&S.xg_empty, xg_phase ^ 1u, p, 52)) dead = true;
+                        dead = __any_sync(0xffffffffu, dead);
+                        if (dead) break;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            st_shared_v4(xs + (uint32_t)(((q & 1) * 32 + lane) * 64 + i * 16),
+                                         make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&S.xg_full);
+                    } else {
+                        if (!mbar_wait(&S.xg_full, xg_phase, p, 53)) dead = true;
+                        dead = __any_sync(0xffffffffu, dead);
+                        if (dead) break;
+                        uint32_t u[16];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            const uint4 t4 = ld_shared_v4(xs + (uint32_t)(((q & 1) * 32 + lane) * 64 + i * 16));
+                            u[4 * i] = t4.x; u[4 * i + 1] = t4.y; u[4 * i + 2] = t4.z; u[4 * i + 3] = t4.w;
+                        }
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&S.xg_empty);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int tok = c * 16 + j;
+                            if (tok < ti.nrows)
+                                p.hbuf[(size_t)(ti.row0 + tok) * p.I + col] =
+                                    __float2bfloat16_rn(silu_mul(__uint_as_float(v[j]), __uint_as_float(u[j])));
+                        }
+                    }
+                    xg_phase ^= 1u;
+                }
+                if (dead) break;
+            } else if (ti.type == 4) {
+                // swapped gemm1: lane = one of this CTA's 128 out-columns, TMEM columns = the m-block's rows
+                const int col = ti.n * 256 + (int)rank * 128 + q * 32 + lane;
+                const int nch = (ti.nrows + 15) >> 4;
+                if (ti.n * 256 + (int)rank * 128 < p.H) {
+                    for (int c = 0; c < nch; ++c) {
+                        uint32_t v[16];
+                        tmem_ld_32x16(taddr + c * 16, v);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int tok = c * 16 + j;
+                            if (tok < ti.nrows)
+                                p.y[(size_t)(ti.row0 + tok) * p.H + col] = __float2bfloat16_rn(__uint_as_float(v[j]));
+                        }
+                    }
+                }
+            } else if (rows_valid > 0) {
                 if (ti.type == 0) {
                     __nv_bfloat16 *dst = p.hbuf + (size_t)(ti.row0 + q * 32) * p.I + (size_t)ti.n * kTN0;
 #pragma unroll 1
@@ -883,8 +975,10 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive_cluster(mapa_u32(smem_u32(&S.tmem_empty[ps.acc]), 0u));
-                if (ti.nrows > 0)
-                    red_release_add_u32(ti.type == 0 ? &p.h_ready[ti.mb] : &p.ctl->y_done[ti.chunk], 1u);
+                // a swapped gemm0 tile is stored by the two gate warps of each CTA (4 arrivals per
+                // m-block and n-tile, like a regular tile); a swapped gemm1 tile by all 8 warps
+                if (ti.type == 0 || (ti.type == 3 && q < 2)) red_release_add_u32(&p.h_ready[ti.mb], 1u);
+                else if (ti.type == 1 || ti.type == 4) red_release_add_u32(&p.ctl->y_done[ti.chunk], 1u);
                 if (q == 0) trace_ev(p, S, kEvGemmEpi, (unsigned)(ti.mb & 0xFFFFFF), te0, trace_now(p),
                                      (unsigned)(ti.type << 16 | ti.n));
             }
@@ -902,7 +996,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
 __global__ void __launch_bounds__(kThreads, 1)
 weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUtensorMap tm_xe,
                  const __grid_constant__ CUtensorMap tm_wgu, const __grid_constant__ CUtensorMap tm_h,
-                 const __grid_constant__ CUtensorMap tm_wd)
+                 const __grid_constant__ CUtensorMap tm_wd, const __grid_constant__ CUtensorMap tm_wgu64)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *stages = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -922,8 +1016,9 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
             mbar_init(&S.dv_full[i], 1); mbar_init(&S.dv_empty[i], 1);
             mbar_init(&S.cb_full[i], 1); mbar_init(&S.cb_empty[i], kCombWarps);
         }
+        mbar_init(&S.xg_full, 2); mbar_init(&S.xg_empty, 2);
         fence_mbar_init();
-        tma_prefetch_desc(&tm_xe); tma_prefetch_desc(&tm_wgu); tma_prefetch_desc(&tm_h); tma_prefetch_desc(&tm_wd);
+        tma_prefetch_desc(&tm_xe); tma_prefetch_desc(&tm_wgu); tma_prefetch_desc(&tm_h); tma_prefetch_desc(&tm_wd); tma_prefetch_desc(&tm_wgu64);
     }
     if (warp == 1) { tmem_alloc_pair(&S.tmem_base, kTmemCols); tmem_relinquish_pair(); }
     tc_fence_before();
@@ -1070,9 +1165,10 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
 #pragma unroll
             for (int f = 0; f < kFine; ++f) if (f / g == j) rows += cf[f];
             const int mbs = (rows + kBM - 1) / kBM;
-            int tot, ptot;
+            int tot, ptot, nodd;
             const int ex = block_excl_scan(mbs, S, tot);
             const int pex = block_excl_scan((mbs + 1) >> 1, S, ptot);
+            (void)block_excl_scan(mbs & 1, S, nodd);
             if (tid < EE) {
                 S.seg_mb0[j * EE + tid] = mb_base + ex;
                 S.seg_pt0[j * EE + tid] = pt_base + pex;
@@ -1083,6 +1179,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
                 S.chunk_mb0[j] = mb_base;
                 S.chunk_pt0[j] = pt_base;
                 S.chunk_tile0[j] = pt_base * (p.nt0 + p.nt1);
+                S.chunk_nswap[j] = nodd;
             }
             run_row += rows;
             mb_base += tot;
@@ -1153,14 +1250,14 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
         if (p.mode == kModeSerial) {
             dispatch_phase(p, S, stages);
             alive = grid_barrier(p, S, 2u * n_sm, 2);
-            if (alive) gemm_phase(p, S, stages, tmem_base, &tm_xe, &tm_wgu, &tm_h, &tm_wd, 0x7fffffff, ps);
+            if (alive) gemm_phase(p, S, stages, tmem_base, &tm_xe, &tm_wgu, &tm_h, &tm_wd, &tm_wgu64, 0x7fffffff, ps);
             alive = alive && grid_barrier(p, S, 3u * n_sm, 3);
             if (alive) combine_phase(p, S, stages);
         } else {
             const bool mover = (int)blockIdx.x < plan_c;      // role from c* and the block index
             if (mover) dispatch_phase(p, S, stages);
             const int budget = mover ? plan_steal : 0x7fffffff;
-            if (budget > 0 || p.elastic_steal) gemm_phase(p, S, stages, tmem_base, &tm_xe, &tm_wgu, &tm_h, &tm_wd, budget, ps);
+            if (budget > 0 || p.elastic_steal) gemm_phase(p, S, stages, tmem_base, &tm_xe, &tm_wgu, &tm_h, &tm_wd, &tm_wgu64, budget, ps);
             combine_phase(p, S, stages);
         }
     }

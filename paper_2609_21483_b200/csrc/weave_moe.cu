@@ -101,7 +101,7 @@ struct weave_moe {
     int last_cuda_error;
     void *trace;
     int trace_cap;
-    CUtensorMap tm_xe, tm_wgu, tm_h, tm_wd;
+    CUtensorMap tm_xe, tm_wgu, tm_h, tm_wd, tm_wgu64;
 };
 
 namespace {
@@ -113,11 +113,12 @@ int cuda_fail(weave_moe *h, cudaError_t e)
 }
 
 // bf16 matrix [rows][cols] row-major, box = 64 columns (128 bytes) x 128 rows, 128-byte swizzle
-int encode_map(EncodeTiledFn fn, CUtensorMap *m, const void *base, uint64_t rows, uint64_t cols, bool weights)
+int encode_map(EncodeTiledFn fn, CUtensorMap *m, const void *base, uint64_t rows, uint64_t cols, bool weights,
+               uint32_t box_rows = kBM)
 {
     cuuint64_t dims[2] = {cols, rows};
     cuuint64_t strides[1] = {cols * 2};
-    cuuint32_t box[2] = {kBK, kBM};
+    cuuint32_t box[2] = {kBK, box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -239,6 +240,7 @@ int weave_moe_create(const weave_moe_config *cfg, weave_moe_t *out)
     r |= encode_map(enc, &h->tm_wgu, cfg->gate_up, (uint64_t)EE * 2 * cfg->ffn, (uint64_t)cfg->hidden, true);
     r |= encode_map(enc, &h->tm_h, h->ws + L.hbuf, (uint64_t)L.p_max, (uint64_t)cfg->ffn, false);
     r |= encode_map(enc, &h->tm_wd, cfg->down, (uint64_t)EE * cfg->hidden, (uint64_t)cfg->ffn, true);
+    r |= encode_map(enc, &h->tm_wgu64, cfg->gate_up, (uint64_t)EE * 2 * cfg->ffn, (uint64_t)cfg->hidden, true, 64);
     if (r) { h->last_cuda_error = r; delete h; return WEAVE_ERR_CUDA; }
 
     e = cudaMemset(h->ws, 0, L.zero_end);
@@ -301,7 +303,7 @@ int weave_moe_forward(weave_moe_t h, const void *x, const float *logits, void *o
     p.trace = reinterpret_cast<uint4 *>(h->trace);
     p.trace_cap = h->trace_cap;
 
-    void *args[] = {&p, &h->tm_xe, &h->tm_wgu, &h->tm_h, &h->tm_wd};
+    void *args[] = {&p, &h->tm_xe, &h->tm_wgu, &h->tm_h, &h->tm_wd, &h->tm_wgu64};
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // one CTA per SM, in clusters of two neighbouring SMs (the GEMM phase's CTA pairs); cooperative,
     // so that all CTAs are co-resident for the in-kernel grid barrier and flag waits
@@ -588,6 +590,7 @@ int weave_moe_forward_static(int hidden, int ffn, int num_experts, int top_k, in
     r |= encode_map(sd->encode, &h.tm_wgu, gate_up, (uint64_t)EE * 2 * ffn, (uint64_t)hidden, true);
     r |= encode_map(sd->encode, &h.tm_h, h.ws + L.hbuf, (uint64_t)L.p_max, (uint64_t)ffn, false);
     r |= encode_map(sd->encode, &h.tm_wd, down, (uint64_t)EE * hidden, (uint64_t)ffn, true);
+    r |= encode_map(sd->encode, &h.tm_wgu64, gate_up, (uint64_t)EE * 2 * ffn, (uint64_t)hidden, true, 64);
     if (r) return WEAVE_ERR_CUDA;
 
     // the array keeps whatever the last call left behind: zero the control words, refill the tables
