@@ -260,25 +260,31 @@ __device__ __forceinline__ int block_excl_scan(int v, SmemTail &S, int &total)
 // ------------------------------------------------------------------------------------ phase R
 
 // One warp routes one token: the k largest logits (ties to the lowest expert index) in descending
-// order, gates = softmax over those k.  Lane l holds the logits of experts l, l+32, ...
-__device__ __forceinline__ void route_token(const KParams &p, int t, int tl, unsigned long long *r_mask, int *r_idx)
+// order, gates = softmax over those k.  Lane l holds the logits of experts l, l+32, ... (NS of them).
+template <int NS>
+__device__ __forceinline__ void load_logits(const KParams &p, int t, float (&v)[NS])
+{
+    const int lane = threadIdx.x & 31;
+#pragma unroll
+    for (int m = 0; m < NS; ++m) {
+        const int e = lane + 32 * m;
+        v[m] = e < p.E ? __ldg(p.logits + (size_t)t * p.E + e) : __int_as_float(0xff800000);
+    }
+}
+
+template <int NS>
+__device__ __forceinline__ void route_token(const KParams &p, int t, int tl, float (&v)[NS],
+                                            unsigned long long *r_mask, int *r_idx)
 {
     const int lane = threadIdx.x & 31;
     const float NEG_INF = __int_as_float(0xff800000);
-    float v[kMaxEE / 32];
     bool bad = false;
 #pragma unroll
-    for (int m = 0; m < kMaxEE / 32; ++m) {
-        int e = lane + 32 * m;
-        float x = NEG_INF;
-        if (e < p.E) {
-            x = __ldg(p.logits + (size_t)t * p.E + e);
-            if (!(fabsf(x) <= 3.402823466e38f)) {   // NaN or +-inf: flag it, keep indices in range
-                bad = true;
-                x = -3.402823466e38f;
-            }
+    for (int m = 0; m < NS; ++m) {
+        if (lane + 32 * m < p.E && !(fabsf(v[m]) <= 3.402823466e38f)) {   // NaN or +-inf: flag it, keep indices in range
+            bad = true;
+            v[m] = -3.402823466e38f;
         }
-        v[m] = x;
     }
     if (__any_sync(0xffffffffu, bad) && lane == 0) atomicCAS(&p.ctl->status, 0, kErrNonFinite);
 
@@ -288,7 +294,7 @@ __device__ __forceinline__ void route_token(const KParams &p, int t, int tl, uns
         float bv = NEG_INF;
         int be = 0x7fffffff;
 #pragma unroll
-        for (int m = 0; m < kMaxEE / 32; ++m)
+        for (int m = 0; m < NS; ++m)
             if (v[m] > bv) { bv = v[m]; be = lane + 32 * m; }   // strict '>' keeps the lower index
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
@@ -298,7 +304,7 @@ __device__ __forceinline__ void route_token(const KParams &p, int t, int tl, uns
         }
         if ((be & 31) == lane) {
 #pragma unroll
-            for (int m = 0; m < kMaxEE / 32; ++m)
+            for (int m = 0; m < NS; ++m)
                 if (m == (be >> 5)) v[m] = NEG_INF;             // taken
         }
         if (lane == j) { my_e = be; my_v = bv; }
@@ -312,6 +318,29 @@ __device__ __forceinline__ void route_token(const KParams &p, int t, int tl, uns
         p.gates[(size_t)t * p.k + lane] = __fdiv_rn(pj, sum);
         r_idx[tl * kMaxTopK + lane] = my_e;
         atomicOr(&r_mask[my_e], 1ull << tl);
+    }
+}
+
+// the tokens of one 64-token block that belong to this warp; the next token's logits are in flight
+// while the current one is ranked
+template <int NS>
+__device__ __forceinline__ void route_block_tokens(const KParams &p, int b, unsigned long long *r_mask, int *r_idx)
+{
+    const int warp = threadIdx.x >> 5;
+    float cur[NS], nxt[NS];
+    int tl = warp;
+    if (b * kRouteBlock + tl < p.T) load_logits<NS>(p, b * kRouteBlock + tl, cur);
+    for (; tl < kRouteBlock; tl += kThreads / 32) {
+        const int t = b * kRouteBlock + tl;
+        if (t >= p.T) break;
+        const int tn = t + kThreads / 32;
+        const bool more = (tl + kThreads / 32 < kRouteBlock) && tn < p.T;
+        if (more) load_logits<NS>(p, tn, nxt);
+        route_token<NS>(p, t, tl, cur, r_mask, r_idx);
+        if (more) {
+#pragma unroll
+            for (int m = 0; m < NS; ++m) cur[m] = nxt[m];
+        }
     }
 }
 
@@ -874,25 +903,29 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
             tc_fence_after();
             const unsigned long long te0 = trace_now(p);
             const int rows_valid = ti.nrows - q * 32;          // rows of this warp's quadrant that exist
+            bool acc_released = false;
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)ps.acc * 256u;
             if (ti.type == 3) {
                 // swapped gemm0: lanes 0..63 hold the gate projection of this CTA's 64 h-columns, lanes
                 // 64..127 the up projection; TMEM columns are the m-block's rows.  The up warps hand
                 // their values to the gate warps through the staging buffer, 16 rows at a time.
-                const uint32_t xs = smem_u32(stages + kStages * kStageBytes);            // [64][16] fp32
+                // each up warp (q = 2, 3) writes into its OWN 2 KB staging region, [32][16] fp32, and gate
+                // warp q - 2 reads it; a warp's region is never written by anybody else, so a warp that
+                // is still busy with the previous tile cannot be overrun
+                const uint32_t xs = smem_u32(stages + kStages * kStageBytes) + (uint32_t)(2 + (q & 1)) * 2048u;
                 const int col = ti.n * kTN0 + (int)rank * 64 + (q & 1) * 32 + lane;      // this thread's h-column
                 const int nch = (ti.nrows + 15) >> 4;
                 for (int c = 0; c < nch && !dead; ++c) {
                     uint32_t v[16];
                     tmem_ld_32x16(taddr + c * 16, v);
-                    tmem_ld_wait();
+                    tmem_ld_wait16(v);
                     if (q >= 2) {
                         if (!mbar_wait(&S.xg_empty, xg_phase ^ 1u, p, 52)) dead = true;
                         dead = __any_sync(0xffffffffu, dead);
                         if (dead) break;
 #pragma unroll
                         for (int i = 0; i < 4; ++i)
-                            st_shared_v4(xs + (uint32_t)(((q & 1) * 32 + lane) * 64 + i * 16),
+                            st_shared_v4(xs + (uint32_t)(lane * 64 + i * 16),
                                          make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&S.xg_full);
@@ -903,7 +936,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                         uint32_t u[16];
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
-                            const uint4 t4 = ld_shared_v4(xs + (uint32_t)(((q & 1) * 32 + lane) * 64 + i * 16));
+                            const uint4 t4 = ld_shared_v4(xs + (uint32_t)(lane * 64 + i * 16));
                             u[4 * i] = t4.x; u[4 * i + 1] = t4.y; u[4 * i + 2] = t4.z; u[4 * i + 3] = t4.w;
                         }
                         __syncwarp();
@@ -919,6 +952,13 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                     xg_phase ^= 1u;
                 }
                 if (dead) break;
+                // an up warp may reuse its staging region in the next tile only after the gate warps
+                // have read the last chunk
+                if (q >= 2) {
+                    if (!mbar_wait(&S.xg_empty, xg_phase ^ 1u, p, 54)) dead = true;
+                    dead = __any_sync(0xffffffffu, dead);
+                    if (dead) break;
+                }
             } else if (ti.type == 4) {
                 // swapped gemm1: lane = one of this CTA's 128 out-columns, TMEM columns = the m-block's rows
                 const int col = ti.n * 256 + (int)rank * 128 + q * 32 + lane;
@@ -927,7 +967,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                     for (int c = 0; c < nch; ++c) {
                         uint32_t v[16];
                         tmem_ld_32x16(taddr + c * 16, v);
-                        tmem_ld_wait();
+                        tmem_ld_wait16(v);
 #pragma unroll
                         for (int j = 0; j < 16; ++j) {
                             const int tok = c * 16 + j;
@@ -937,50 +977,72 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                     }
                 }
             } else if (rows_valid > 0) {
+                // TMEM loads run one (half-)chunk ahead of the conversion and the stores; the
+                // accumulator is handed back to the MMA issuer as soon as the last load has landed
                 if (ti.type == 0) {
                     __nv_bfloat16 *dst = p.hbuf + (size_t)(ti.row0 + q * 32) * p.I + (size_t)ti.n * kTN0;
-#pragma unroll 1
-                    for (int c = 0; c < kTN0 / 32; ++c) {
-                        uint32_t gr[32], ur[32];
-                        tmem_ld_32x32(taddr + c * 32, gr);
-                        tmem_ld_32x32(taddr + 128 + c * 32, ur);
-                        tmem_ld_wait();
-                        uint32_t o[16];
+                    uint32_t gr[2][16], ur[2][16], o[16];
+                    tmem_ld_32x16(taddr, gr[0]);
+                    tmem_ld_32x16(taddr + 128, ur[0]);
 #pragma unroll
-                        for (int i = 0; i < 16; ++i)
-                            o[i] = pack_bf16x2(silu_mul(__uint_as_float(gr[2 * i]), __uint_as_float(ur[2 * i])),
-                                               silu_mul(__uint_as_float(gr[2 * i + 1]), __uint_as_float(ur[2 * i + 1])));
-                        staged_store_32x32(stg, lane, o, dst + c * 32, (size_t)p.I, rows_valid);
+                    for (int hc = 0; hc < kTN0 / 16; ++hc) {
+                        tmem_ld_wait16(gr[hc & 1]);
+                        reg_fence16(ur[hc & 1]);
+                        if (hc + 1 < kTN0 / 16) {
+                            tmem_ld_32x16(taddr + (hc + 1) * 16, gr[(hc + 1) & 1]);
+                            tmem_ld_32x16(taddr + 128 + (hc + 1) * 16, ur[(hc + 1) & 1]);
+                        } else {
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive_cluster(mapa_u32(smem_u32(&S.tmem_empty[ps.acc]), 0u));
+                            acc_released = true;
+                        }
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            o[(hc & 1) * 8 + i] =
+                                pack_bf16x2(silu_mul(__uint_as_float(gr[hc & 1][2 * i]), __uint_as_float(ur[hc & 1][2 * i])),
+                                            silu_mul(__uint_as_float(gr[hc & 1][2 * i + 1]), __uint_as_float(ur[hc & 1][2 * i + 1])));
+                        if (hc & 1) staged_store_32x32(stg, lane, o, dst + (hc >> 1) * 32, (size_t)p.I, rows_valid);
                     }
                 } else {
                     __nv_bfloat16 *dst = p.y + (size_t)(ti.row0 + q * 32) * p.H + (size_t)ti.n * 256;
                     const int nc = min(256, p.H - ti.n * 256) / 32;   // the last n-tile may be half wide
-#pragma unroll 1
-                    for (int c = 0; c < nc; ++c) {
-                        uint32_t ar[32];
-                        tmem_ld_32x32(taddr + c * 32, ar);
-                        tmem_ld_wait();
-                        uint32_t o[16];
+                    uint32_t ar[2][32], o[16];
+                    tmem_ld_32x32(taddr, ar[0]);
 #pragma unroll
-                        for (int i = 0; i < 16; ++i)
-                            o[i] = pack_bf16x2(__uint_as_float(ar[2 * i]), __uint_as_float(ar[2 * i + 1]));
-                        staged_store_32x32(stg, lane, o, dst + c * 32, (size_t)p.H, rows_valid);
+                    for (int c = 0; c < 8; ++c) {
+                        if (c < nc) {
+                            tmem_ld_wait32(ar[c & 1]);
+                            if (c + 1 < nc) {
+                                tmem_ld_32x32(taddr + (c + 1) * 32, ar[(c + 1) & 1]);
+                            } else {
+                                tc_fence_before();
+                                __syncwarp();
+                                if (lane == 0) mbar_arrive_cluster(mapa_u32(smem_u32(&S.tmem_empty[ps.acc]), 0u));
+                                acc_released = true;
+                            }
+#pragma unroll
+                            for (int i = 0; i < 16; ++i)
+                                o[i] = pack_bf16x2(__uint_as_float(ar[c & 1][2 * i]), __uint_as_float(ar[c & 1][2 * i + 1]));
+                            staged_store_32x32(stg, lane, o, dst + c * 32, (size_t)p.H, rows_valid);
+                        }
                     }
                 }
             }
             // the accumulator may be overwritten by the next-but-one tile; the rows just stored are read
             // by TMA (gemm1) or by ordinary loads (combine) on other SMs once the counter says so
+            const unsigned long long te1 = trace_now(p);
             tc_fence_before();
             fence_proxy_async();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive_cluster(mapa_u32(smem_u32(&S.tmem_empty[ps.acc]), 0u));
+                if (!acc_released) mbar_arrive_cluster(mapa_u32(smem_u32(&S.tmem_empty[ps.acc]), 0u));
                 // a swapped gemm0 tile is stored by the two gate warps of each CTA (4 arrivals per
                 // m-block and n-tile, like a regular tile); a swapped gemm1 tile by all 8 warps
                 if (ti.type == 0 || (ti.type == 3 && q < 2)) red_release_add_u32(&p.h_ready[ti.mb], 1u);
                 else if (ti.type == 1 || ti.type == 4) red_release_add_u32(&p.ctl->y_done[ti.chunk], 1u);
                 if (q == 0) trace_ev(p, S, kEvGemmEpi, (unsigned)(ti.mb & 0xFFFFFF), te0, trace_now(p),
-                                     (unsigned)(ti.type << 16 | ti.n));
+                                     (unsigned)(ti.type << 16 | (int)min(65535ull, te1 - te0)));
             }
             ps.next_acc();
         }
@@ -1038,10 +1100,10 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
     for (int b = blockIdx.x; b < p.nblk; b += n_sm) {
         for (int e = tid; e < EE; e += kThreads) r_mask[e] = 0ull;
         __syncthreads();
-        for (int tl = warp; tl < kRouteBlock; tl += kThreads / 32) {
-            const int t = b * kRouteBlock + tl;
-            if (t < p.T) route_token(p, t, tl, r_mask, r_idx);
-        }
+        if (p.E <= 32) route_block_tokens<1>(p, b, r_mask, r_idx);
+        else if (p.E <= 64) route_block_tokens<2>(p, b, r_mask, r_idx);
+        else if (p.E <= 128) route_block_tokens<4>(p, b, r_mask, r_idx);
+        else route_block_tokens<8>(p, b, r_mask, r_idx);
         __syncthreads();
         // in-block rank of each (token, slot): tokens before it in the block that chose the same expert
         for (int pi = tid; pi < kRouteBlock * p.k; pi += kThreads) {

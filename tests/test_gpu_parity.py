@@ -58,11 +58,15 @@ def test_c3_skewed_routing_sampled():
     dev = to_dev(inp)
     moe, out0, _ = run_case(cfg, n_sample=24, inp=inp, dev_tensors=dev)
     bits = out0.view(torch.int16).clone()
-    for s in [(pk.SCHED_SERIAL, 0, 1, 0), (pk.SCHED_FIXED, 22, 1, 0), (pk.SCHED_FIXED, 30, 4, 5)]:
+    # chunking multiplies the (chunk, expert) segments and with them the unpaired, swapped-operand
+    # tiles; every schedule, repeated, must reproduce the same bits
+    for s in [(pk.SCHED_SERIAL, 0, 1, 0), (pk.SCHED_FIXED, 22, 1, 0), (pk.SCHED_FIXED, 30, 4, 5),
+              (pk.SCHED_FIXED, 8, 8, 1 << 20), (pk.SCHED_FIXED, 74, 2, 0)]:
         moe.set_schedule(*s)
-        out = moe.forward(dev[0], dev[1])
-        moe.check()
-        assert torch.equal(out.view(torch.int16), bits), f"schedule {s} changed the output bits"
+        for rep in range(3):
+            out = moe.forward(dev[0], dev[1])
+            moe.check()
+            assert torch.equal(out.view(torch.int16), bits), f"schedule {s} (run {rep}) changed the output bits"
     moe.close()
 
 
