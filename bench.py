@@ -219,6 +219,8 @@ def run_ours(args):
     out = torch.empty_like(x)
     out_h = torch.empty_like(x_h).pin_memory()
     moe = pk.WeaveMoE(gu, dn, cfg.E, cfg.k, cfg.S, max_tokens=cfg.T)
+    if args.sms:
+        moe.set_sm_count(args.sms)
     stream = torch.cuda.current_stream()
     sched = {"auto": (pk.SCHED_AUTO, 0, 1, 0), "serial": (pk.SCHED_SERIAL, 0, 1, 0)}
     geo = moe.geometry()
@@ -352,6 +354,7 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=0,
                     help="tokens in the CPU oracle's timed sample (0 = sized for --cpu-seconds of work)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--sms", type=int, default=0, help="SMs the kernel may occupy (0 = all; even)")
     ap.add_argument("--no-ablation", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -99,6 +99,12 @@ int weave_moe_destroy(weave_moe_t h);
  * next forward. */
 int weave_moe_set_schedule(weave_moe_t h, int mode, int c, int K, int steal);
 
+/* Number of SMs (= persistent CTAs) the kernel occupies from the next forward on: even, at least 4,
+ * at most the device's SM count rounded down to even (the default).  Leaves the other SMs to
+ * concurrent work (or to a profiler).  The cost tables keep being indexed by SM count, so the
+ * model's candidate c must stay below the new count. */
+int weave_moe_set_sm_count(weave_moe_t h, int n_sm);
+
 /* Hardware input of the cost model (Figure 7): bw[i] = bytes/us moved by i movement SMs,
  * tflops[i] = FLOP/us of i GEMM SMs, i in [0, n_sm] (host arrays of n_sm+1 floats, entry 0
  * ignored); eff_chunk[4] = Eq. 9's correction factor for K = 1,2,4,8; alpha = Section 3.1's

@@ -59,7 +59,7 @@ EXPORTS = [
     "weave_moe_get_geometry", "weave_moe_get_routing", "weave_moe_get_intermediates",
     "weave_moe_status", "weave_moe_set_timeout_ms", "weave_moe_debug_withhold_flag",
     "weave_moe_last_cuda_error", "weave_moe_strerror", "weave_moe_set_trace",
-    "weave_moe_forward_static", "weave_moe_static_scratch_bytes",
+    "weave_moe_forward_static", "weave_moe_static_scratch_bytes", "weave_moe_set_sm_count",
 ]
 
 
@@ -102,6 +102,8 @@ def load():
     lib.weave_moe_set_timeout_ms.argtypes = [vp, ci]
     lib.weave_moe_debug_withhold_flag.restype = ci
     lib.weave_moe_debug_withhold_flag.argtypes = [vp, ci]
+    lib.weave_moe_set_sm_count.restype = ci
+    lib.weave_moe_set_sm_count.argtypes = [vp, ci]
     lib.weave_moe_set_trace.restype = ci
     lib.weave_moe_set_trace.argtypes = [vp, vp, ci]
     lib.weave_moe_forward_static.restype = ci
@@ -297,6 +299,9 @@ class WeaveMoE:
         st = self.status()
         if st != WEAVE_OK:
             raise WeaveError(st, f"device status (wait id {self._lib.weave_moe_last_cuda_error(self._h)})")
+
+    def set_sm_count(self, n_sm: int):
+        _check(self._lib.weave_moe_set_sm_count(self._h, n_sm), "weave_moe_set_sm_count")
 
     def set_timeout_ms(self, ms: int):
         _check(self._lib.weave_moe_set_timeout_ms(self._h, ms), "weave_moe_set_timeout_ms")

@@ -1055,7 +1055,9 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
 
 // ------------------------------------------------------------------------------------ the kernel
 
-__global__ void __launch_bounds__(kThreads, 1)
+constexpr int kErrNoPairs = -2;     // reported as "unsupported device"
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUtensorMap tm_xe,
                  const __grid_constant__ CUtensorMap tm_wgu, const __grid_constant__ CUtensorMap tm_h,
                  const __grid_constant__ CUtensorMap tm_wd, const __grid_constant__ CUtensorMap tm_wgu64)
@@ -1067,6 +1069,14 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int n_sm = (int)gridDim.x;
     const int EE = p.EE;
+
+    // The GEMM phase addresses the neighbouring CTA's shared memory and barriers.  If a launch path
+    // ever drops the cluster shape, say so and leave before anything is sent to a peer that is
+    // not there (every CTA takes the same branch).
+    if (cluster_nctarank() != 2u) {
+        if (threadIdx.x == 0) atomicCAS(&p.ctl->status, 0, kErrNoPairs);
+        return;
+    }
 
     if (tid == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(&S.full[i], 1); mbar_init(&S.empty[i], 1); }

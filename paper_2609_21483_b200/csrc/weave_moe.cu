@@ -220,10 +220,7 @@ int weave_moe_create(const weave_moe_config *cfg, weave_moe_t *out)
         cudaLaunchConfig_t lc;
         memset(&lc, 0, sizeof(lc));
         lc.gridDim = dim3(h->n_cta); lc.blockDim = dim3(kThreads); lc.dynamicSmemBytes = (size_t)kSmemBytes;
-        cudaLaunchAttribute at[1];
-        at[0].id = cudaLaunchAttributeClusterDimension;
-        at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-        lc.attrs = at; lc.numAttrs = 1;
+        lc.attrs = nullptr; lc.numAttrs = 0;      // the cluster shape (2,1,1) is compiled into the kernel
         int ncl = 0;
         e = cudaOccupancyMaxActiveClusters(&ncl, (const void *)weave_moe_kernel, &lc);
         if (e != cudaSuccess || ncl * 2 < h->n_cta) { delete h; return WEAVE_ERR_UNSUPPORTED_DEVICE; }
@@ -305,22 +302,11 @@ int weave_moe_forward(weave_moe_t h, const void *x, const float *logits, void *o
 
     void *args[] = {&p, &h->tm_xe, &h->tm_wgu, &h->tm_h, &h->tm_wd, &h->tm_wgu64};
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // one CTA per SM, in clusters of two neighbouring SMs (the GEMM phase's CTA pairs); cooperative,
-    // so that all CTAs are co-resident for the in-kernel grid barrier and flag waits
-    cudaLaunchConfig_t lc;
-    memset(&lc, 0, sizeof(lc));
-    lc.gridDim = dim3(h->n_cta);
-    lc.blockDim = dim3(kThreads);
-    lc.dynamicSmemBytes = (size_t)kSmemBytes;
-    lc.stream = st;
-    cudaLaunchAttribute at[2];
-    at[0].id = cudaLaunchAttributeClusterDimension;
-    at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
-    at[1].id = cudaLaunchAttributeCooperative;
-    at[1].val.cooperative = 1;
-    lc.attrs = at;
-    lc.numAttrs = 2;
-    cudaError_t e = cudaLaunchKernelExC(&lc, (const void *)weave_moe_kernel, args);
+    // one CTA per SM; the kernel is compiled with a cluster shape of two neighbouring CTAs (the GEMM
+    // phase's CTA pairs); cooperative, so that all CTAs are co-resident for the in-kernel grid
+    // barrier and flag waits
+    cudaError_t e = cudaLaunchCooperativeKernel((const void *)weave_moe_kernel, dim3(h->n_cta), dim3(kThreads), args,
+                                                (size_t)kSmemBytes, st);
     if (e != cudaSuccess) return cuda_fail(h, e);
     h->last_T = T;
     h->last_stream = st;
@@ -456,6 +442,14 @@ int weave_moe_status(weave_moe_t h)
         h->last_cuda_error = ctl.timeout_where;   // where the first wait gave up (diagnostic)
     }
     return st;
+}
+
+int weave_moe_set_sm_count(weave_moe_t h, int n_sm)
+{
+    if (!h) return WEAVE_ERR_INVALID_ARG;
+    if (n_sm < 4 || (n_sm & 1) || n_sm > h->n_sm) return WEAVE_ERR_INVALID_ARG;
+    h->n_cta = n_sm;
+    return WEAVE_OK;
 }
 
 int weave_moe_set_timeout_ms(weave_moe_t h, int ms)

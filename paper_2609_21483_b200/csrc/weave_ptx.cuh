@@ -260,6 +260,12 @@ __device__ __forceinline__ uint32_t cluster_ctarank()
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
     return r;
 }
+__device__ __forceinline__ uint32_t cluster_nctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
 // shared::cluster address of the same variable in the CTA of the given rank
 __device__ __forceinline__ uint32_t mapa_u32(uint32_t cta_addr, uint32_t rank)
 {
