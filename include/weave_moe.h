@@ -159,8 +159,9 @@ int weave_moe_debug_withhold_flag(weave_moe_t h, int m_block);
  * tracing off.  Each CTA writes up to events_per_cta - 1 records {start ns, end ns (low 32 bits of
  * the global nanosecond timer), kind << 24 | id, extra} into its slice; the slice's last record
  * holds the number written.  Kinds: 1 routing, 2 set-up, 3 permutation fix-up, 4 dispatch tile,
- * 5 GEMM tile loads (extra = ns until its inputs were ready), 6 GEMM tile epilogue (id = m-block,
- * extra = type << 16 | n-tile), 7 combine tile, 8 wait for a chunk's gemm1, 9 grid barrier. */
+ * 5 GEMM tile scheduled (claim until its inputs were ready), 6 GEMM tile epilogue (id = m-block,
+ * extra = type << 16 | ns spent before the release), 7 combine tile, 8 wait for a chunk's gemm1,
+ * 9 grid barrier. */
 int weave_moe_set_trace(weave_moe_t h, void *buf, int events_per_cta);
 
 /* ---- for callers that cannot allocate ---------------------------------------------------------

@@ -715,24 +715,15 @@ __device__ __forceinline__ void linger_after_abort()
     while (globaltimer_ns() - t0 < 50000ull) __nanosleep(1000);
 }
 
-// One warp's 32 rows x 32 columns of bf16 (16 packed words per thread, thread = row) go through a
-// 2 KB staging buffer so that every global store instruction writes 8 rows x 64 contiguous bytes.
-// 16-byte chunk j of row r sits at r*64 + ((j ^ ((r >> 1) & 3)) << 4): conflict-free both ways.
-__device__ __forceinline__ void staged_store_32x32(uint32_t stg, int lane, const uint32_t (&o)[16],
-                                                   __nv_bfloat16 *dst_row0, size_t ld, int rows_valid)
+// Thread = row: 32 columns of bf16 (16 packed words) straight from registers as two 32-byte stores,
+// each a full sector.  No shared memory: during the GEMM phase its bandwidth belongs to the TMA
+// writes and the tensor core's operand reads, and a staged epilogue would queue behind them.
+__device__ __forceinline__ void direct_store_32(const uint32_t (&o)[16], __nv_bfloat16 *dst_row, bool valid)
 {
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-        st_shared_v4(stg + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4),
-                     make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]));
-    __syncwarp();
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int row = i * 8 + (lane >> 2), ch = lane & 3;
-        const uint4 v = ld_shared_v4(stg + row * 64 + ((ch ^ ((row >> 1) & 3)) << 4));
-        if (row < rows_valid) st_v4(dst_row0 + (size_t)row * ld + ch * 8, v);
+    if (valid) {
+        st_v8(dst_row, &o[0]);
+        st_v8(dst_row + 16, &o[8]);
     }
-    __syncwarp();
 }
 
 // budget = how many pair tiles this CTA pair may claim (the steal count for a movement pair).
@@ -885,7 +876,6 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
     } else if (warp >= 4) {
         // ---------------- epilogue (both CTAs): TMEM -> registers -> (SwiGLU) -> bf16 -> staged store
         const int q = warp & 3;                      // TMEM lane quadrant this warp may read
-        const uint32_t stg = smem_u32(stages + kStages * kStageBytes) + (uint32_t)q * 2048u;
         bool dead = false;
         uint32_t xg_phase = 0;
         while (!dead) {
@@ -980,17 +970,20 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                 // TMEM loads run one (half-)chunk ahead of the conversion and the stores; the
                 // accumulator is handed back to the MMA issuer as soon as the last load has landed
                 if (ti.type == 0) {
+                    // batches of 32 h-columns (32 gate + 32 up accumulator columns), double-buffered:
+                    // a TMEM load takes several hundred cycles while the tensor core is busy, so
+                    // the next batch is in flight while this one is converted and stored
                     __nv_bfloat16 *dst = p.hbuf + (size_t)(ti.row0 + q * 32) * p.I + (size_t)ti.n * kTN0;
-                    uint32_t gr[2][16], ur[2][16], o[16];
-                    tmem_ld_32x16(taddr, gr[0]);
-                    tmem_ld_32x16(taddr + 128, ur[0]);
+                    uint32_t gr[2][32], ur[2][32], o[16];
+                    tmem_ld_32x32(taddr, gr[0]);
+                    tmem_ld_32x32(taddr + 128, ur[0]);
 #pragma unroll
-                    for (int hc = 0; hc < kTN0 / 16; ++hc) {
-                        tmem_ld_wait16(gr[hc & 1]);
-                        reg_fence16(ur[hc & 1]);
-                        if (hc + 1 < kTN0 / 16) {
-                            tmem_ld_32x16(taddr + (hc + 1) * 16, gr[(hc + 1) & 1]);
-                            tmem_ld_32x16(taddr + 128 + (hc + 1) * 16, ur[(hc + 1) & 1]);
+                    for (int c = 0; c < kTN0 / 32; ++c) {
+                        tmem_ld_wait32(gr[c & 1]);
+                        reg_fence32(ur[c & 1]);
+                        if (c + 1 < kTN0 / 32) {
+                            tmem_ld_32x32(taddr + (c + 1) * 32, gr[(c + 1) & 1]);
+                            tmem_ld_32x32(taddr + 128 + (c + 1) * 32, ur[(c + 1) & 1]);
                         } else {
                             tc_fence_before();
                             __syncwarp();
@@ -998,23 +991,23 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                             acc_released = true;
                         }
 #pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            o[(hc & 1) * 8 + i] =
-                                pack_bf16x2(silu_mul(__uint_as_float(gr[hc & 1][2 * i]), __uint_as_float(ur[hc & 1][2 * i])),
-                                            silu_mul(__uint_as_float(gr[hc & 1][2 * i + 1]), __uint_as_float(ur[hc & 1][2 * i + 1])));
-                        if (hc & 1) staged_store_32x32(stg, lane, o, dst + (hc >> 1) * 32, (size_t)p.I, rows_valid);
+                        for (int i = 0; i < 16; ++i)
+                            o[i] = pack_bf16x2(silu_mul(__uint_as_float(gr[c & 1][2 * i]), __uint_as_float(ur[c & 1][2 * i])),
+                                               silu_mul(__uint_as_float(gr[c & 1][2 * i + 1]), __uint_as_float(ur[c & 1][2 * i + 1])));
+                        direct_store_32(o, dst + (size_t)lane * p.I + c * 32, lane < rows_valid);
                     }
                 } else {
+                    // batches of 64 out-columns, double-buffered
                     __nv_bfloat16 *dst = p.y + (size_t)(ti.row0 + q * 32) * p.H + (size_t)ti.n * 256;
-                    const int nc = min(256, p.H - ti.n * 256) / 32;   // the last n-tile may be half wide
-                    uint32_t ar[2][32], o[16];
-                    tmem_ld_32x32(taddr, ar[0]);
+                    const int nb = min(256, p.H - ti.n * 256) / 64;   // the last n-tile may be half wide
+                    uint32_t ar[2][64], o[16];
+                    tmem_ld_32x64(taddr, ar[0]);
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        if (c < nc) {
-                            tmem_ld_wait32(ar[c & 1]);
-                            if (c + 1 < nc) {
-                                tmem_ld_32x32(taddr + (c + 1) * 32, ar[(c + 1) & 1]);
+                    for (int c = 0; c < 4; ++c) {
+                        if (c < nb) {
+                            tmem_ld_wait64(ar[c & 1]);
+                            if (c + 1 < nb) {
+                                tmem_ld_32x64(taddr + (c + 1) * 64, ar[(c + 1) & 1]);
                             } else {
                                 tc_fence_before();
                                 __syncwarp();
@@ -1022,9 +1015,13 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                                 acc_released = true;
                             }
 #pragma unroll
-                            for (int i = 0; i < 16; ++i)
-                                o[i] = pack_bf16x2(__uint_as_float(ar[c & 1][2 * i]), __uint_as_float(ar[c & 1][2 * i + 1]));
-                            staged_store_32x32(stg, lane, o, dst + c * 32, (size_t)p.H, rows_valid);
+                            for (int hh = 0; hh < 2; ++hh) {
+#pragma unroll
+                                for (int i = 0; i < 16; ++i)
+                                    o[i] = pack_bf16x2(__uint_as_float(ar[c & 1][hh * 32 + 2 * i]),
+                                                       __uint_as_float(ar[c & 1][hh * 32 + 2 * i + 1]));
+                                direct_store_32(o, dst + (size_t)lane * p.H + c * 64 + hh * 32, lane < rows_valid);
+                            }
                         }
                     }
                 }
