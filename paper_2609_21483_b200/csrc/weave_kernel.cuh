@@ -272,75 +272,112 @@ __device__ __forceinline__ void load_logits(const KParams &p, int t, float (&v)[
     }
 }
 
+// fp32 -> uint32 that orders like the float (finite values; -0 has been folded into +0)
+__device__ __forceinline__ unsigned float_order_key(float v)
+{
+    const unsigned u = __float_as_uint(v);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float float_from_order_key(unsigned k)
+{
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+
+// Two tokens per warp at a time: the two selections are independent instruction streams, so the
+// warp-reduction latencies of one hide behind the other.  `nt` (1 or 2) tokens are valid.
 template <int NS>
-__device__ __forceinline__ void route_token(const KParams &p, int t, int tl, float (&v)[NS],
-                                            unsigned long long *r_mask, int *r_idx)
+__device__ __forceinline__ void route_tokens2(const KParams &p, const int (&t)[2], const int (&tl)[2], int nt,
+                                              float (&v)[2][NS], unsigned long long *r_mask, int *r_idx)
 {
     const int lane = threadIdx.x & 31;
-    const float NEG_INF = __int_as_float(0xff800000);
+    // keys: 0 = absent / already taken; every finite logit maps to a key >= 1 that orders like
+    // the float, with -0.0 == +0.0 (the comparison rule of the routing definition)
+    unsigned key[2][NS];
     bool bad = false;
 #pragma unroll
-    for (int m = 0; m < NS; ++m) {
-        if (lane + 32 * m < p.E && !(fabsf(v[m]) <= 3.402823466e38f)) {   // NaN or +-inf: flag it, keep indices in range
-            bad = true;
-            v[m] = -3.402823466e38f;
+    for (int u = 0; u < 2; ++u) {
+#pragma unroll
+        for (int m = 0; m < NS; ++m) {
+            key[u][m] = 0u;
+            if (u < nt && lane + 32 * m < p.E) {
+                float x = v[u][m];
+                if (!(fabsf(x) <= 3.402823466e38f)) {   // NaN or +-inf: flag it, keep indices in range
+                    bad = true;
+                    x = -3.402823466e38f;
+                }
+                x = __fadd_rn(x, 0.0f);                  // folds -0 into +0, leaves everything else alone
+                key[u][m] = float_order_key(x);
+            }
         }
     }
     if (__any_sync(0xffffffffu, bad) && lane == 0) atomicCAS(&p.ctl->status, 0, kErrNonFinite);
 
-    int my_e = 0;
-    float my_v = 0.f;
+    int my_e[2] = {0, 0};
+    unsigned my_key[2] = {0u, 0u};
     for (int j = 0; j < p.k; ++j) {
-        float bv = NEG_INF;
-        int be = 0x7fffffff;
+        unsigned bk[2], wk[2];
+        int be[2], we[2];
 #pragma unroll
-        for (int m = 0; m < NS; ++m)
-            if (v[m] > bv) { bv = v[m]; be = lane + 32 * m; }   // strict '>' keeps the lower index
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            float ov = __shfl_xor_sync(0xffffffffu, bv, o);
-            int oe = __shfl_xor_sync(0xffffffffu, be, o);
-            if (ov > bv || (ov == bv && oe < be)) { bv = ov; be = oe; }
-        }
-        if ((be & 31) == lane) {
+        for (int u = 0; u < 2; ++u) {
+            bk[u] = 0u;
+            be[u] = 0x7fffffff;
 #pragma unroll
             for (int m = 0; m < NS; ++m)
-                if (m == (be >> 5)) v[m] = NEG_INF;             // taken
+                if (key[u][m] > bk[u]) { bk[u] = key[u][m]; be[u] = lane + 32 * m; }   // strict '>' keeps the lower index
         }
-        if (lane == j) { my_e = be; my_v = bv; }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) wk[u] = __reduce_max_sync(0xffffffffu, bk[u]);          // largest logit
+#pragma unroll
+        for (int u = 0; u < 2; ++u)                                                          // lowest index with it
+            we[u] = (int)__reduce_min_sync(0xffffffffu, bk[u] == wk[u] ? (unsigned)be[u] : 0x7fffffffu);
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            if ((we[u] & 31) == lane) {
+#pragma unroll
+                for (int m = 0; m < NS; ++m)
+                    if (m == (we[u] >> 5)) key[u][m] = 0u;                                   // taken
+            }
+            if (lane == j) { my_e[u] = we[u]; my_key[u] = wk[u]; }
+        }
     }
-    const float vmax = __shfl_sync(0xffffffffu, my_v, 0);
-    const float pj = lane < p.k ? expf(my_v - vmax) : 0.f;
-    float sum = 0.f;
-    for (int j = 0; j < p.k; ++j) sum += __shfl_sync(0xffffffffu, pj, j);   // slot order
-    if (lane < p.k) {
-        p.topk_idx[(size_t)t * p.k + lane] = my_e;
-        p.gates[(size_t)t * p.k + lane] = __fdiv_rn(pj, sum);
-        r_idx[tl * kMaxTopK + lane] = my_e;
-        atomicOr(&r_mask[my_e], 1ull << tl);
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        if (u < nt) {
+            const float my_v = float_from_order_key(my_key[u]);
+            const float vmax = __shfl_sync(0xffffffffu, my_v, 0);
+            const float pj = lane < p.k ? expf(my_v - vmax) : 0.f;
+            float sum = 0.f;
+            for (int j = 0; j < p.k; ++j) sum += __shfl_sync(0xffffffffu, pj, j);   // slot order
+            if (lane < p.k) {
+                p.topk_idx[(size_t)t[u] * p.k + lane] = my_e[u];
+                p.gates[(size_t)t[u] * p.k + lane] = __fdiv_rn(pj, sum);
+                r_idx[tl[u] * kMaxTopK + lane] = my_e[u];
+                atomicOr(&r_mask[my_e[u]], 1ull << tl[u]);
+            }
+        }
     }
 }
 
-// the tokens of one 64-token block that belong to this warp; the next token's logits are in flight
-// while the current one is ranked
+// the tokens of one 64-token block that belong to this warp (tl = warp, warp + 8, ...), two at a time
 template <int NS>
 __device__ __forceinline__ void route_block_tokens(const KParams &p, int b, unsigned long long *r_mask, int *r_idx)
 {
     const int warp = threadIdx.x >> 5;
-    float cur[NS], nxt[NS];
-    int tl = warp;
-    if (b * kRouteBlock + tl < p.T) load_logits<NS>(p, b * kRouteBlock + tl, cur);
-    for (; tl < kRouteBlock; tl += kThreads / 32) {
-        const int t = b * kRouteBlock + tl;
-        if (t >= p.T) break;
-        const int tn = t + kThreads / 32;
-        const bool more = (tl + kThreads / 32 < kRouteBlock) && tn < p.T;
-        if (more) load_logits<NS>(p, tn, nxt);
-        route_token<NS>(p, t, tl, cur, r_mask, r_idx);
-        if (more) {
+    constexpr int kStep = kThreads / 32;
+    for (int tl0 = warp; tl0 < kRouteBlock; tl0 += 2 * kStep) {
+        int t[2], tl[2];
+        tl[0] = tl0; tl[1] = tl0 + kStep;
+        t[0] = b * kRouteBlock + tl[0]; t[1] = b * kRouteBlock + tl[1];
+        if (t[0] >= p.T) break;
+        const int nt = (tl[1] < kRouteBlock && t[1] < p.T) ? 2 : 1;
+        float v[2][NS];
+        load_logits<NS>(p, t[0], v[0]);
+        if (nt == 2) load_logits<NS>(p, t[1], v[1]);
+        else {
 #pragma unroll
-            for (int m = 0; m < NS; ++m) cur[m] = nxt[m];
+            for (int m = 0; m < NS; ++m) v[1][m] = 0.f;
         }
+        route_tokens2<NS>(p, t, tl, nt, v, r_mask, r_idx);
     }
 }
 
@@ -466,7 +503,7 @@ __device__ __forceinline__ unsigned y_done_target(const SmemTail &S, const KPara
 // writes each full buffer to its (contiguous) destination rows with one bulk store.  About 96 KB
 // of loads and as much of stores are in flight per SM.  The m-block's ready flag is released once
 // its last store has completed.
-__device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, uint8_t *stages)
+__device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, uint8_t *stages, int max_tiles)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     fence_proxy_async();      // the buffers held routing scratch written with ordinary stores
@@ -480,7 +517,7 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
         bool ok = true;
         if (lane == 0) ok = flag_wait_ge(&p.ctl->fix_done, (unsigned)p.nblk, p, 10);
         ok = __shfl_sync(0xffffffffu, ok, 0);
-        while (ok) {
+        for (int taken = 0; ok && taken < max_tiles; ++taken) {
             int mb = 0;
             if (lane == 0) mb = (int)atomicAdd(&p.ctl->q_disp, 1u);
             mb = __shfl_sync(0xffffffffu, mb, 0);
@@ -1317,14 +1354,19 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
     PipeState ps;
     if (alive) {
         if (p.mode == kModeSerial) {
-            dispatch_phase(p, S, stages);
+            dispatch_phase(p, S, stages, 0x7fffffff);
             alive = grid_barrier(p, S, 2u * n_sm, 2);
             if (alive) gemm_phase(p, S, stages, tmem_base, &tm_xe, &tm_wgu, &tm_h, &tm_wd, &tm_wgu64, 0x7fffffff, ps);
             alive = alive && grid_barrier(p, S, 3u * n_sm, 3);
             if (alive) combine_phase(p, S, stages);
         } else {
             const bool mover = (int)blockIdx.x < plan_c;      // role from c* and the block index
-            if (mover) dispatch_phase(p, S, stages);
+            // movement CTAs work through the dispatch queue; every GEMM CTA first dispatches one
+            // m-block too, so that the first wave of GEMM tiles does not wait for a handful of movers
+            // (the mirror image of the final combine on all SMs); the forced "no temporal
+            // scheduling" ablation keeps the two groups apart
+            const int dmax = mover ? 0x7fffffff : (p.elastic_steal ? 1 : 0);
+            if (dmax > 0) dispatch_phase(p, S, stages, dmax);
             const int budget = mover ? plan_steal : 0x7fffffff;
             if (budget > 0 || p.elastic_steal) gemm_phase(p, S, stages, tmem_base, &tm_xe, &tm_wgu, &tm_h, &tm_wd, &tm_wgu64, budget, ps);
             combine_phase(p, S, stages);
