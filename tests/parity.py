@@ -81,3 +81,44 @@ def run_case(cfg: wl.MoEConfig, sched=None, n_sample=None, layer=0, inp=None, de
         l2 = check_values(bf16_to_np(out[torch.from_numpy(toks).long().to(out.device)]),
                           oracle_rows(inp, toks), cfg.name)
     return moe, out, l2
+
+
+def stream_weights_to_dev(cfg: wl.MoEConfig, dev="cuda"):
+    """Device weights of a layer too large to build on the host in one piece: generated and copied
+    expert by expert (the generator is counter-based, so the values equal make_weights())."""
+    EE = cfg.E + cfg.S
+    gu = torch.empty((EE, 2 * cfg.I, cfg.H), dtype=torch.bfloat16, device=dev)
+    dn = torch.empty((EE, cfg.H, cfg.I), dtype=torch.bfloat16, device=dev)
+    for e in range(EE):
+        g, d = wl.expert_weights(cfg, e)
+        gu[e].copy_(torch.from_numpy(g.view(np.int16)).view(torch.bfloat16))
+        dn[e].copy_(torch.from_numpy(d.view(np.int16)).view(torch.bfloat16))
+    return gu, dn
+
+
+def run_case_streamed(cfg: wl.MoEConfig, n_sample: int, sched=None):
+    """Like run_case for shapes whose weights do not fit comfortably on the host: the oracle gets
+    zero-initialised weight arrays (untouched pages cost nothing) in which only the experts of the
+    sampled tokens are filled in."""
+    x_h, lg_h = wl.make_x(cfg), wl.make_logits(cfg)
+    x = torch.from_numpy(x_h.view(np.int16)).view(torch.bfloat16).cuda()
+    lg = torch.from_numpy(lg_h).cuda()
+    gu, dn = stream_weights_to_dev(cfg)
+    moe = WeaveMoE(gu, dn, cfg.E, cfg.k, cfg.S, max_tokens=cfg.T)
+    if sched is not None:
+        moe.set_schedule(*sched)
+    out = moe.forward(x, lg)
+    moe.check()
+    inp = wl.LayerInputs(cfg, x_h, lg_h, None, None)
+    check_routing(moe, inp)
+    toks = wl.stratified_token_sample(cfg.T, n_sample, seed=cfg.cfg_id)
+    idx, _ = oracle.route(lg_h[toks], cfg.k)
+    need = sorted(set(idx.ravel().tolist()) | set(range(cfg.E, cfg.E + cfg.S)))
+    EE = cfg.E + cfg.S
+    gu_h = np.zeros((EE, 2 * cfg.I, cfg.H), np.uint16)
+    dn_h = np.zeros((EE, cfg.H, cfg.I), np.uint16)
+    for e in need:
+        gu_h[e], dn_h[e] = wl.expert_weights(cfg, e)
+    ref = oracle.moe_tokens(x_h, lg_h, gu_h, dn_h, cfg.k, toks, cfg.S)
+    l2 = check_values(bf16_to_np(out[torch.from_numpy(toks).long().to(out.device)]), ref, cfg.name)
+    return moe, out, l2

@@ -8,7 +8,7 @@ import torch
 import oracle
 import workloads as wl
 import paper_2609_21483_b200 as pk
-from parity import bf16_to_np, check_routing, check_values, oracle_rows, run_case, to_dev
+from parity import bf16_to_np, check_routing, check_values, oracle_rows, run_case, run_case_streamed, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -93,6 +93,14 @@ def test_c5_qwen3_235b_shaped_two_layers_sampled():
             dev = (x, torch.from_numpy(inp.logits).cuda()) + dev_w
         moe, _, _ = run_case(cfg, n_sample=6, inp=inp, dev_tensors=dev, moe=moe)
         plans.append(moe.plan())
+    moe.close()
+
+
+@pytest.mark.parametrize("name", ["t1_dsv3_T2048", "t1_phi35_T2048", "t1_qwen35_35b_T2048", "t1_dsv2_T2048"])
+def test_remaining_table1_shapes_sampled(name):
+    """The Table 1 rows that are not among the five configs of record (256 experts, H = 7168 / 5120,
+    I = 512 ... 6400), mildly skewed routing, four sampled tokens each."""
+    moe, _, _ = run_case_streamed(wl.CONFIGS[name], n_sample=4)
     moe.close()
 
 

@@ -69,3 +69,22 @@ def test_token_sample_is_stratified():
     s = wl.stratified_token_sample(4096, 64, seed=1)
     assert s[0] == 0 and s[-1] == 4095 and len(set(s)) == len(s) and len(s) >= 60
     assert np.diff(s).max() < 3 * 4096 // 62
+
+
+def test_expert_weights_equal_the_slices_of_the_full_tensors():
+    cfg = wl.MoEConfig("slice", 77, T=8, H=128, I=256, E=5, k=2, S=1)
+    gu, dn = wl.make_weights(cfg)
+    for e in (0, 3, 5):
+        g, d = wl.expert_weights(cfg, e)
+        np.testing.assert_array_equal(g, gu[e])
+        np.testing.assert_array_equal(d, dn[e])
+
+
+def test_table1_bench_configs_cover_every_row_and_sequence_length():
+    t1 = _table1()
+    names = {"DSv3": "dsv3", "Phi-3.5-MoE": "phi35", "Qwen3-30B": "qwen3_30b", "Qwen3.5-35B": "qwen35_35b",
+             "DSv2-Lite": "dsv2lite", "DSv2": "dsv2"}
+    for row, short in names.items():
+        for T in (2048, 4096, 8192):
+            c = wl.CONFIGS[f"t1_{short}_T{T}"]
+            assert (c.E, c.k, c.H, c.I) == t1[row] and c.T == T

@@ -45,6 +45,9 @@ def _load():
             fn.restype = None
             fn.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_uint64,
                            ctypes.c_double, ctypes.c_double]
+        lib.wl_normal_bf16_range.restype = None
+        lib.wl_normal_bf16_range.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_uint64,
+                                             ctypes.c_double, ctypes.c_double]
         lib.wl_add_row_bias_f32.restype = None
         lib.wl_add_row_bias_f32.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
                                             ctypes.c_void_p]
@@ -93,6 +96,15 @@ CONFIGS: Dict[str, MoEConfig] = {
     "c5_qwen3_235b": MoEConfig("c5_qwen3_235b", 5, T=16384, H=4096, I=1536, E=128, k=8,
                                zipf_range=(0.8, 1.6), layers=24),
 }
+
+# The other shapes of the paper's Table 1 (Qwen3-30B and DSv2-Lite are C3 / C4 above), at the
+# paper's sequence lengths 2048 / 4096 / 8192, with a mild load skew (the paper's routing comes from
+# trained routers on real prompts; a flat N(0,1) router would be unrealistically balanced).
+for _i, (_n, _E, _k, _H, _I) in enumerate([("dsv3", 256, 8, 7168, 2048), ("phi35", 16, 2, 4096, 6400),
+                                           ("qwen35_35b", 256, 8, 2048, 512), ("dsv2", 160, 6, 5120, 1536),
+                                           ("qwen3_30b", 128, 8, 2048, 768), ("dsv2lite", 64, 6, 2048, 1408)]):
+    for _T in (2048, 4096, 8192):
+        CONFIGS[f"t1_{_n}_T{_T}"] = MoEConfig(f"t1_{_n}_T{_T}", 10 + _i, T=_T, H=_H, I=_I, E=_E, k=_k, zipf_s=0.5)
 
 _T_X, _T_LOGITS, _T_GATE_UP, _T_DOWN, _T_PERM, _T_SKEW = 1, 2, 3, 4, 5, 6
 
@@ -165,6 +177,18 @@ def make_weights(cfg: MoEConfig):
     gu = normal_bf16(EE * 2 * cfg.I * cfg.H, tensor_seed(cfg, 0, _T_GATE_UP), 0.0, 0.02)
     dn = normal_bf16(EE * cfg.H * cfg.I, tensor_seed(cfg, 0, _T_DOWN), 0.0, 0.02)
     return gu.reshape(EE, 2 * cfg.I, cfg.H), dn.reshape(EE, cfg.H, cfg.I)
+
+
+def expert_weights(cfg: MoEConfig, e: int):
+    """(gate_up[e] [2I,H], down[e] [H,I]) of one expert: the same values make_weights() puts at index
+    e, produced without materialising the other experts (the streams are counter-based)."""
+    lib = _load()
+    n_gu, n_dn = 2 * cfg.I * cfg.H, cfg.H * cfg.I
+    gu = np.empty(n_gu, dtype=np.uint16)
+    dn = np.empty(n_dn, dtype=np.uint16)
+    lib.wl_normal_bf16_range(gu.ctypes.data, e * n_gu, n_gu, tensor_seed(cfg, 0, _T_GATE_UP), 0.0, 0.02)
+    lib.wl_normal_bf16_range(dn.ctypes.data, e * n_dn, n_dn, tensor_seed(cfg, 0, _T_DOWN), 0.0, 0.02)
+    return gu.reshape(2 * cfg.I, cfg.H), dn.reshape(cfg.H, cfg.I)
 
 
 @dataclass

@@ -47,6 +47,21 @@ static inline uint16_t f32_to_bf16_rne(float f)
     return (uint16_t)(u >> 16);
 }
 
+/* elements [start, start+n) of the bf16 stream (start must be even): lets a caller produce a huge
+ * tensor piece by piece, or only the pieces it needs */
+void wl_normal_bf16_range(uint16_t *out, int64_t start, int64_t n, uint64_t seed, double mean, double std)
+{
+    uint64_t sh = sm64(seed);
+    int64_t p0 = start / 2, npairs = (n + 1) / 2;
+#pragma omp parallel for schedule(static)
+    for (int64_t p = 0; p < npairs; ++p) {
+        double z0, z1;
+        normal_pair(sh, (uint64_t)(p0 + p), &z0, &z1);
+        out[2 * p] = f32_to_bf16_rne((float)(mean + std * z0));
+        if (2 * p + 1 < n) out[2 * p + 1] = f32_to_bf16_rne((float)(mean + std * z1));
+    }
+}
+
 /* out[i] = mean + std * z_i, i in [0,n), stored as fp32 */
 void wl_normal_f32(float *out, int64_t n, uint64_t seed, double mean, double std)
 {
