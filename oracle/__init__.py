@@ -43,6 +43,13 @@ def _load():
         lib.oracle_moe_layer.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci] + [vp] * 10
         lib.oracle_moe_tokens.restype = ci
         lib.oracle_moe_tokens.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, vp, ci, vp]
+        i64p = ctypes.POINTER(ctypes.c_int64)
+        lib.oracle_ep_descriptors.restype = ci
+        lib.oracle_ep_descriptors.argtypes = [vp, ci, ci, ci, ci, ci, i64p, i64p, i64p]
+        lib.oracle_permute_ep.restype = ci
+        lib.oracle_permute_ep.argtypes = [vp, ci, ci, ci, ci, ci, vp, vp, vp, vp]
+        lib.oracle_moe_tokens_ep.restype = ci
+        lib.oracle_moe_tokens_ep.argtypes = [vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci, vp, ci, vp]
         lib.oracle_num_threads.restype = ci
         _lib = lib
     return _lib
@@ -177,4 +184,52 @@ def moe_tokens(x, logits, gate_up, down, k: int, tokens, S: int = 0,
                                    int(acc_double), _p(tokens), tokens.shape[0], _p(out))
     if rc:
         raise ValueError(f"oracle_moe_tokens failed: {rc}")
+    return out
+
+
+# ---------------------------------------------------------------------------- one EP rank's share
+
+def ep_descriptors(idx: np.ndarray, E: int, ep_rank: int, ep_size: int):
+    """(X_local, X_in, X_in_uniq) of Section 3.1 for one rank."""
+    idx = _c(idx, np.int32)
+    T, k = idx.shape
+    a, b, c = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
+    rc = _load().oracle_ep_descriptors(_p(idx), T, E, k, ep_rank, ep_size, ctypes.byref(a), ctypes.byref(b),
+                                       ctypes.byref(c))
+    if rc:
+        raise ValueError(f"oracle_ep_descriptors failed: {rc}")
+    return a.value, b.value, c.value
+
+
+def routing_ep(logits: np.ndarray, k: int, ep_rank: int, ep_size: int) -> Routing:
+    """Global routing, permutation restricted to the rank's experts (row -1 for the other slots)."""
+    idx, gates = route(logits, k)
+    T, E = logits.shape
+    counts = np.empty(E, np.int32)
+    offsets = np.empty(E + 1, np.int32)
+    row_of = np.empty((T, k), np.int32)
+    token_of = np.full(T * k, -1, np.int32)
+    rc = _load().oracle_permute_ep(_p(idx), T, E, k, ep_rank, ep_size, _p(counts), _p(offsets), _p(row_of),
+                                   _p(token_of))
+    if rc:
+        raise ValueError(f"oracle_permute_ep failed: {rc}")
+    return Routing(idx, gates, counts, offsets, row_of, token_of[:int(offsets[-1])].copy())
+
+
+def moe_tokens_ep(x, logits, gate_up, down, k: int, tokens, ep_rank: int, ep_size: int,
+                  acc_double: bool = False) -> np.ndarray:
+    """Partial output rows [n,H] of the listed tokens for one rank (sum over its local experts)."""
+    x = _c(x, np.uint16)
+    logits = _c(logits, np.float32)
+    gate_up = _c(gate_up, np.uint16)
+    down = _c(down, np.uint16)
+    tokens = _c(tokens, np.int32)
+    T, H = x.shape
+    E = logits.shape[1]
+    I = gate_up.shape[1] // 2
+    out = np.empty((tokens.shape[0], H), np.float32)
+    rc = _load().oracle_moe_tokens_ep(_p(x), _p(logits), _p(gate_up), _p(down), H, I, E, k, ep_rank, ep_size,
+                                      int(acc_double), _p(tokens), tokens.shape[0], _p(out))
+    if rc:
+        raise ValueError(f"oracle_moe_tokens_ep failed: {rc}")
     return out

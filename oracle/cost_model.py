@@ -62,6 +62,16 @@ def workloads(T: int, P: int, H: int, I: int):
     return w_comp, w_disp, w_comb
 
 
+def workloads_ep(x_local: int, x_in: int, x_in_uniq: int, H: int, I: int):
+    """Eq. 1-3 literally, for one expert-parallel rank: W_comp = (X_local + X_in) * 6HI,
+    W_dispatch = X_in^uniq * B (each unique remote token is pulled once), W_combine = X_in * B."""
+    B = f32(2 * H)
+    w_comp = f32(x_local + x_in) * f32(6.0) * f32(H) * f32(I)
+    w_disp = f32(x_in_uniq) * B
+    w_comb = f32(x_in) * B
+    return w_comp, w_disp, w_comb
+
+
 def t_total(tab: CostTables, c: int, ki: int, w_comp, w_disp, w_comb) -> np.float32:
     """Eq. 15 with Eq. 9 (T_comp), Eq. 5 (T_comm) and Eq. 10 (T_tail)."""
     K = f32(K_CANDIDATES[ki])
@@ -98,11 +108,12 @@ def n_steal(tab: CostTables, c: int, w_comp, w_disp, w_comb, n_tiles: int) -> in
     return max(0, min(ns, n_tiles))
 
 
-def plan(tab: CostTables, T: int, P: int, H: int, I: int, n_tiles_of_K: Sequence[int]) -> Plan:
+def plan(tab: CostTables, T: int, P: int, H: int, I: int, n_tiles_of_K: Sequence[int], w=None) -> Plan:
     """Eq. 16: argmin over the (c,K) grid, ties to the smaller c and then the smaller K;
     then the steal count at (c*,K*).  n_tiles_of_K[ki] = number of GEMM tiles of the
-    layer when it is cut into K_CANDIDATES[ki] chunks."""
-    w_comp, w_disp, w_comb = workloads(T, P, H, I)
+    layer when it is cut into K_CANDIDATES[ki] chunks.  w = (W_comp, W_disp, W_comb) overrides the
+    single-GPU workload terms (used with workloads_ep)."""
+    w_comp, w_disp, w_comb = w if w is not None else workloads(T, P, H, I)
     best = None
     for c in candidates(tab):
         for ki in range(len(K_CANDIDATES)):

@@ -295,6 +295,108 @@ int oracle_moe_tokens(const uint16_t *x, const float *logits, const uint16_t *ga
     return rc;
 }
 
+/* ------------------------------------------------------------------ one expert-parallel rank's share */
+
+/*
+ * Expert parallelism (the paper's Section 2.1 / 3.1 setting) as seen by one rank r of R: the rank
+ * hosts experts [r*E/R, (r+1)*E/R) and owns the tokens of shard r, where shard s = tokens
+ * [s*Ts, min(T,(s+1)*Ts)), Ts = ceil(T/R).  Routing is global (all E experts, gates normalised
+ * over all k selected experts).  The rank computes, for every token, the partial sum over the
+ * token's experts that live on this rank (the per-pair results a real system would send back to
+ * the token's owner); tokens without a local expert get zeros.  Summing the partial outputs of all
+ * R ranks gives the full layer.
+ *
+ * Workload descriptors of Section 3.1:
+ *   x_local      pairs (token, local expert) whose token is in the rank's own shard
+ *   x_in         pairs whose token belongs to another rank ("remote tokens routed to local experts")
+ *   x_in_uniq    distinct remote tokens with at least one local expert (each is transferred once)
+ */
+int oracle_ep_descriptors(const int32_t *idx, int T, int E, int k, int ep_rank, int ep_size,
+                          int64_t *x_local, int64_t *x_in, int64_t *x_in_uniq)
+{
+    if (ep_size < 1 || ep_rank < 0 || ep_rank >= ep_size || E % ep_size) return -2;
+    const int el = ep_rank * (E / ep_size), eh = el + E / ep_size;
+    const int Ts = (T + ep_size - 1) / ep_size;
+    int64_t xl = 0, xi = 0, xu = 0;
+    for (int t = 0; t < T; ++t) {
+        const int own = (t / Ts) == ep_rank;
+        int n = 0;
+        for (int j = 0; j < k; ++j) {
+            int e = idx[(size_t)t * k + j];
+            if (e >= el && e < eh) ++n;
+        }
+        if (own) xl += n; else { xi += n; if (n) ++xu; }
+    }
+    *x_local = xl; *x_in = xi; *x_in_uniq = xu;
+    return 0;
+}
+
+/* counts / offsets / permutation restricted to the rank's experts: other experts have count 0,
+ * slots that point to them get row -1; rows of a local expert are its tokens in ascending order. */
+int oracle_permute_ep(const int32_t *idx, int T, int E, int k, int ep_rank, int ep_size,
+                      int32_t *counts, int32_t *offsets, int32_t *row_of, int32_t *token_of)
+{
+    if (ep_size < 1 || ep_rank < 0 || ep_rank >= ep_size || E % ep_size) return -2;
+    const int el = ep_rank * (E / ep_size), eh = el + E / ep_size;
+    for (int e = 0; e < E; ++e) counts[e] = 0;
+    for (int t = 0; t < T; ++t)
+        for (int j = 0; j < k; ++j) {
+            int e = idx[(size_t)t * k + j];
+            if (e < 0 || e >= E) return -1;
+            if (e >= el && e < eh) counts[e] += 1;
+        }
+    offsets[0] = 0;
+    for (int e = 0; e < E; ++e) offsets[e + 1] = offsets[e] + counts[e];
+    int32_t *cursor = (int32_t *)malloc(sizeof(int32_t) * (size_t)E);
+    if (!cursor) return -3;
+    for (int e = 0; e < E; ++e) cursor[e] = offsets[e];
+    for (int t = 0; t < T; ++t)
+        for (int j = 0; j < k; ++j) {
+            int e = idx[(size_t)t * k + j];
+            if (e >= el && e < eh) {
+                int r = cursor[e]++;
+                row_of[(size_t)t * k + j] = r;
+                token_of[r] = t;
+            } else {
+                row_of[(size_t)t * k + j] = -1;
+            }
+        }
+    free(cursor);
+    return 0;
+}
+
+/* partial output rows of the listed tokens for rank ep_rank (see above); out [n][H] fp32 */
+int oracle_moe_tokens_ep(const uint16_t *x, const float *logits, const uint16_t *gate_up,
+                         const uint16_t *down, int H, int I, int E, int k, int ep_rank, int ep_size,
+                         int acc_double, const int32_t *tokens, int n, float *out)
+{
+    if (k < 1 || k > E || k > 64) return -2;
+    if (ep_size < 1 || ep_rank < 0 || ep_rank >= ep_size || E % ep_size) return -2;
+    const int el = ep_rank * (E / ep_size), eh = el + E / ep_size;
+    float *xr = (float *)malloc(sizeof(float) * (size_t)H);
+    float *hb = (float *)malloc(sizeof(float) * (size_t)I);
+    float *y = (float *)malloc(sizeof(float) * (size_t)H);
+    if (!xr || !hb || !y) { free(xr); free(hb); free(y); return -3; }
+    int rc = 0;
+    for (int i = 0; i < n && !rc; ++i) {
+        int t = tokens[i];
+        int32_t idx[64];
+        float gate[64];
+        if (route_token(logits + (size_t)t * E, E, k, idx, gate)) { rc = -1; break; }
+        for (int h = 0; h < H; ++h) xr[h] = bf16_to_f32(x[(size_t)t * H + h]);
+        for (int h = 0; h < H; ++h) out[(size_t)i * H + h] = 0.0f;
+        for (int j = 0; j < k; ++j) {                 /* slot order, local experts only */
+            int e = idx[j];
+            if (e < el || e >= eh) continue;
+            expert_ffn_row(xr, gate_up + (size_t)e * 2 * I * H, down + (size_t)e * H * I, H, I,
+                           acc_double, 1, hb, y);
+            for (int h = 0; h < H; ++h) out[(size_t)i * H + h] += gate[j] * y[h];
+        }
+    }
+    free(xr); free(hb); free(y);
+    return rc;
+}
+
 int oracle_num_threads(void)
 {
     int n = 1;
