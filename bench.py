@@ -242,6 +242,8 @@ def run_ours(args):
     moe = pk.WeaveMoE(gu, dn, cfg.E, cfg.k, cfg.S, max_tokens=cfg.T)
     if args.sms:
         moe.set_sm_count(args.sms)
+    if args.ep > 1:
+        moe.set_expert_parallel(args.ep_rank, args.ep)
     stream = torch.cuda.current_stream()
     sched = {"auto": (pk.SCHED_AUTO, 0, 1, 0), "serial": (pk.SCHED_SERIAL, 0, 1, 0)}
     geo = moe.geometry()
@@ -322,6 +324,12 @@ def run_ours(args):
 
     peaks = load_peaks()
     work = layer_work(cfg)
+    ep_desc = None
+    if args.ep > 1:
+        # the rank computes only its own pairs: scale the algorithmic work by its share of the pairs
+        ep_desc = moe.ep_descriptors()
+        share = (ep_desc["x_local"] + ep_desc["x_in"]) / float(cfg.P)
+        work = {k: v * share for k, v in work.items()}
     layer_s = sec_max / args.steps / L
     # the burst bf16 peak for a kernel timed more or less alone, the sustained one when the timed
     # region is a long back-to-back run under the power cap (the 24-layer stack, or >= 0.5 s)
@@ -337,7 +345,7 @@ def run_ours(args):
     traffic = NCU_DRAM_BYTES_PER_LAUNCH.get(cfg.name)
 
     cpu_base = None
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and args.ep <= 1:
         import oracle
         oracle.build()
         lg0 = logits_h[0].numpy()
@@ -376,6 +384,9 @@ def run_ours(args):
         "gpu_launches": args.steps * L,
         "clocks": clocks,
         "plan": plans[0] if plans else None,
+        "expert_parallel": ({"ep_size": args.ep, "ep_rank": args.ep_rank, **ep_desc,
+                             "note": "work and roofline scaled by this rank's share of the token-expert pairs (last layer's routing)"}
+                            if ep_desc else None),
         "ablation": ablation,
         "cpu_baseline": cpu_base,
         "paper_context": "paper reports 2.89x geomean MoE-layer speedup over 5 systems on 4xH100 (EP=4); no 1-GPU or B200 number",
@@ -397,6 +408,8 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=0,
                     help="tokens in the CPU oracle's timed sample (0 = sized for --cpu-seconds of work)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--ep", type=int, default=1, help="model one rank of an expert-parallel group of this size")
+    ap.add_argument("--ep-rank", type=int, default=0)
     ap.add_argument("--sms", type=int, default=0, help="SMs the kernel may occupy (0 = all; even)")
     ap.add_argument("--no-ablation", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -99,6 +99,24 @@ int weave_moe_destroy(weave_moe_t h);
  * next forward. */
 int weave_moe_set_schedule(weave_moe_t h, int mode, int c, int K, int steal);
 
+/* One expert-parallel rank's share of the layer (the paper's setting, Sections 2.1 and 3.1, modelled
+ * on one GPU): with ep_size > 1 the handle acts as rank ep_rank of ep_size.  It hosts experts
+ * [ep_rank*E/ep_size, (ep_rank+1)*E/ep_size) (weights of all E experts are still passed; the others
+ * are not touched) and owns token shard ep_rank, shard s = tokens [s*Ts, (s+1)*Ts), Ts =
+ * ceil(T/ep_size); the other shards play the remote ranks' tokens, held in local HBM.  Routing stays
+ * global (gates normalised over all k experts).  Every remote token with at least one expert here
+ * is copied once into a staging buffer and all its local experts read that copy (dispatch-side
+ * deduplication, Section 4); out[t] = the partial sum over t's experts hosted here (zero if none) -
+ * summing the outputs of all ranks gives the full layer.  row_of is -1 for slots whose expert
+ * lives elsewhere.  The cost model then uses Eq. 1-3 literally (X_local, X_in, X_in^uniq).
+ * Needs E % ep_size == 0 and no shared experts.  ep_size = 1 switches it off (the default). */
+int weave_moe_set_expert_parallel(weave_moe_t h, int ep_rank, int ep_size);
+
+/* The workload descriptors of Section 3.1 counted by the most recent forward in expert-parallel
+ * mode: pairs with an own-shard token, pairs with a remote token, distinct remote tokens.
+ * Synchronises the last stream. */
+int weave_moe_get_ep_descriptors(weave_moe_t h, long long *x_local, long long *x_in, long long *x_in_uniq);
+
 /* Number of SMs (= persistent CTAs) the kernel occupies from the next forward on: even, at least 4,
  * at most the device's SM count rounded down to even (the default).  Leaves the other SMs to
  * concurrent work (or to a profiler).  The cost tables keep being indexed by SM count, so the

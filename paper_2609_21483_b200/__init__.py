@@ -60,6 +60,7 @@ EXPORTS = [
     "weave_moe_status", "weave_moe_set_timeout_ms", "weave_moe_debug_withhold_flag",
     "weave_moe_last_cuda_error", "weave_moe_strerror", "weave_moe_set_trace",
     "weave_moe_forward_static", "weave_moe_static_scratch_bytes", "weave_moe_set_sm_count",
+    "weave_moe_set_expert_parallel", "weave_moe_get_ep_descriptors",
 ]
 
 
@@ -102,6 +103,10 @@ def load():
     lib.weave_moe_set_timeout_ms.argtypes = [vp, ci]
     lib.weave_moe_debug_withhold_flag.restype = ci
     lib.weave_moe_debug_withhold_flag.argtypes = [vp, ci]
+    lib.weave_moe_set_expert_parallel.restype = ci
+    lib.weave_moe_set_expert_parallel.argtypes = [vp, ci, ci]
+    lib.weave_moe_get_ep_descriptors.restype = ci
+    lib.weave_moe_get_ep_descriptors.argtypes = [vp] + [ctypes.POINTER(ctypes.c_longlong)] * 3
     lib.weave_moe_set_sm_count.restype = ci
     lib.weave_moe_set_sm_count.argtypes = [vp, ci]
     lib.weave_moe_set_trace.restype = ci
@@ -299,6 +304,16 @@ class WeaveMoE:
         st = self.status()
         if st != WEAVE_OK:
             raise WeaveError(st, f"device status (wait id {self._lib.weave_moe_last_cuda_error(self._h)})")
+
+    def set_expert_parallel(self, ep_rank: int, ep_size: int):
+        """Act as rank ep_rank of ep_size (see weave_moe_set_expert_parallel); ep_size = 1 = off."""
+        _check(self._lib.weave_moe_set_expert_parallel(self._h, ep_rank, ep_size), "weave_moe_set_expert_parallel")
+
+    def ep_descriptors(self):
+        v = [ctypes.c_longlong() for _ in range(3)]
+        _check(self._lib.weave_moe_get_ep_descriptors(self._h, *[ctypes.byref(a) for a in v]),
+               "weave_moe_get_ep_descriptors")
+        return {"x_local": v[0].value, "x_in": v[1].value, "x_in_uniq": v[2].value}
 
     def set_sm_count(self, n_sm: int):
         _check(self._lib.weave_moe_set_sm_count(self._h, n_sm), "weave_moe_set_sm_count")

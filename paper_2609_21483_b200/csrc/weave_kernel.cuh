@@ -59,14 +59,19 @@ struct Ctl {
     unsigned abort;       // set by the first wait that gives up; every wait polls it
     unsigned pad0;
     unsigned y_done[kFine];  // per chunk: epilogue-warp arrivals of finished gemm1 tiles
+    unsigned q_pull;      // expert-parallel share: next block of remote tokens to stage
+    unsigned pull_done;   // ... blocks staged
+    unsigned x_local, x_in, x_in_uniq;   // ... the workload descriptors of Section 3.1, counted while routing
+    unsigned pad1[3];
     // ---- not re-zeroed: results for the host
     int status;
     int timeout_where;
     int plan_c, plan_K, plan_steal;
     float plan_t;
     int plan_nmb, plan_ngemm;
+    unsigned ep_x_local, ep_x_in, ep_x_in_uniq;
 };
-constexpr int kCtlZeroWords = 16;
+constexpr int kCtlZeroWords = 24;
 
 struct KParams {
     int T, H, I, E, S, k, EE;
@@ -74,6 +79,11 @@ struct KParams {
     int mode, fixed_c, fixed_K, fixed_steal;
     int nt0, nt1;         // n-tiles per m-block: I / 128, ceil(H / 256)
     int nmb_max;          // allocated length of the per-m-block flag arrays
+    int ep_rank, ep_size; // expert-parallel share (ep_size <= 1: off): this rank hosts experts
+                          // [ep_rank*E/ep_size, (ep_rank+1)*E/ep_size) and owns token shard ep_rank
+    int ep_tshard;        // tokens per shard = ceil(T / ep_size)
+    __nv_bfloat16 *xs;    // [T][H] staging of remote tokens (each unique one is copied once)
+    unsigned long long *uniq_mask;   // [nblk] remote tokens of the block that have a local expert
     int elastic_steal;    // movement pairs keep stealing past their quota while no combine chunk is ready
     int withhold_mb;      // test hook: this m-block's "dispatched" flag is never published (-1 = off)
     int c_min, c_max, c_step;
@@ -117,8 +127,11 @@ struct MvDesc {
     int a;      // dispatch: first destination row        combine: token
     int b;      // dispatch: rows in the buffer            combine: first column
     int c;      // dispatch: m-block                       combine: columns
-    int d;      // dispatch: 1 = last buffer of its tile;  2 = no more work (both phases)
+    int d;      // dispatch: 1 = last buffer of its tile;  2 = no more work (both phases);
+                // 3 / 4 = staging of remote tokens (rows go to xs[tok[i]]; 4 = last buffer of the block)
+    int n;      // combine: rows gathered (0: the token has no expert here, the piece is zero)
     float g[kMaxTopK + 8];   // combine: weight of each gathered row
+    int tok[32];             // staging: destination token of each row in the buffer
 };
 constexpr int kMvBuf = kStageBytes;     // 32 KB
 constexpr int kCombWarps = 6;           // warps 2..7 reduce
@@ -287,9 +300,11 @@ __device__ __forceinline__ float float_from_order_key(unsigned k)
 // warp-reduction latencies of one hide behind the other.  `nt` (1 or 2) tokens are valid.
 template <int NS>
 __device__ __forceinline__ void route_tokens2(const KParams &p, const int (&t)[2], const int (&tl)[2], int nt,
-                                              float (&v)[2][NS], unsigned long long *r_mask, int *r_idx)
+                                              float (&v)[2][NS], unsigned long long *r_mask, int *r_idx, int *r_cnt)
 {
     const int lane = threadIdx.x & 31;
+    const int e_lo = p.ep_size > 1 ? p.ep_rank * (p.E / p.ep_size) : 0;
+    const int e_hi = p.ep_size > 1 ? e_lo + p.E / p.ep_size : p.E;
     // keys: 0 = absent / already taken; every finite logit maps to a key >= 1 that orders like
     // the float, with -0.0 == +0.0 (the comparison rule of the routing definition)
     unsigned key[2][NS];
@@ -348,11 +363,21 @@ __device__ __forceinline__ void route_tokens2(const KParams &p, const int (&t)[2
             const float pj = lane < p.k ? expf(my_v - vmax) : 0.f;
             float sum = 0.f;
             for (int j = 0; j < p.k; ++j) sum += __shfl_sync(0xffffffffu, pj, j);   // slot order
+            // expert-parallel share: only the experts hosted here get rows; the gates stay normalised
+            // over all k selected experts
+            const bool local = lane < p.k && my_e[u] >= e_lo && my_e[u] < e_hi;
             if (lane < p.k) {
                 p.topk_idx[(size_t)t[u] * p.k + lane] = my_e[u];
                 p.gates[(size_t)t[u] * p.k + lane] = __fdiv_rn(pj, sum);
-                r_idx[tl[u] * kMaxTopK + lane] = my_e[u];
-                atomicOr(&r_mask[my_e[u]], 1ull << tl[u]);
+                r_idx[tl[u] * kMaxTopK + lane] = local ? my_e[u] : -1;
+                if (local) atomicOr(&r_mask[my_e[u]], 1ull << tl[u]);
+            }
+            if (p.ep_size > 1) {
+                const int nloc = __popc(__ballot_sync(0xffffffffu, local));
+                if (lane == 0 && nloc) {
+                    if (t[u] / p.ep_tshard == p.ep_rank) atomicAdd(&r_cnt[0], nloc);
+                    else { atomicAdd(&r_cnt[1], nloc); atomicOr(&r_mask[kMaxEE], 1ull << tl[u]); }
+                }
             }
         }
     }
@@ -360,7 +385,8 @@ __device__ __forceinline__ void route_tokens2(const KParams &p, const int (&t)[2
 
 // the tokens of one 64-token block that belong to this warp (tl = warp, warp + 8, ...), two at a time
 template <int NS>
-__device__ __forceinline__ void route_block_tokens(const KParams &p, int b, unsigned long long *r_mask, int *r_idx)
+__device__ __forceinline__ void route_block_tokens(const KParams &p, int b, unsigned long long *r_mask, int *r_idx,
+                                                   int *r_cnt)
 {
     const int warp = threadIdx.x >> 5;
     constexpr int kStep = kThreads / 32;
@@ -377,7 +403,7 @@ __device__ __forceinline__ void route_block_tokens(const KParams &p, int b, unsi
 #pragma unroll
             for (int m = 0; m < NS; ++m) v[1][m] = 0.f;
         }
-        route_tokens2<NS>(p, t, tl, nt, v, r_mask, r_idx);
+        route_tokens2<NS>(p, t, tl, nt, v, r_mask, r_idx, r_cnt);
     }
 }
 
@@ -517,6 +543,57 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
         bool ok = true;
         if (lane == 0) ok = flag_wait_ge(&p.ctl->fix_done, (unsigned)p.nblk, p, 10);
         ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (p.ep_size > 1) {
+            // expert-parallel share: first every remote token that has an expert here is copied ONCE
+            // into the staging buffer xs (the dispatch-side deduplication of the paper's Section 4);
+            // the rows of all its local experts are then gathered from that copy.  One tile per
+            // 64-token routing block, taken by whoever comes first.
+            while (ok) {
+                int blk = 0;
+                if (lane == 0) blk = (int)atomicAdd(&p.ctl->q_pull, 1u);
+                blk = __shfl_sync(0xffffffffu, blk, 0);
+                if (blk >= p.nblk) break;
+                const unsigned long long um = __ldcg(p.uniq_mask + blk);
+                const int n = __popcll(um);
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int bit = lane + 32 * hh;
+                    if ((um >> bit) & 1ull) S.tok[__popcll(um & ((1ull << bit) - 1ull))] = blk * kRouteBlock + bit;
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    if (n == 0) {
+                        red_release_add_u32(&p.ctl->pull_done, 1u);
+                    } else {
+                        const int Rp = min(R, 32);
+                        for (int r0 = 0; r0 < n; r0 += Rp) {
+                            const int nr = min(Rp, n - r0);
+                            if (!mbar_wait(&S.dv_empty[b], ph ^ 1u, p, 14)) { ok = false; break; }
+                            S.mv[b].a = 0; S.mv[b].b = nr; S.mv[b].c = blk; S.mv[b].d = (r0 + nr >= n) ? 4 : 3;
+                            for (int i = 0; i < nr; ++i) S.mv[b].tok[i] = S.tok[r0 + i];
+                            mbar_arrive_expect_tx(&S.dv_full[b], (uint32_t)nr * rowb);
+                            const uint32_t dst = smem_u32(stages + b * kMvBuf);
+                            for (int i = 0; i < nr; ++i)
+                                bulk_load(dst + (uint32_t)i * rowb, p.x + (size_t)S.tok[r0 + i] * p.H, rowb, &S.dv_full[b]);
+                            if (++b == kStages) { b = 0; ph ^= 1u; }
+                        }
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                __syncwarp();
+            }
+            // rows may be gathered from xs only when every block has been staged: have the storer
+            // complete and publish what it still holds back (d = 5), then wait for everybody's blocks
+            if (lane == 0 && ok) {
+                if (mbar_wait(&S.dv_empty[b], ph ^ 1u, p, 16)) {
+                    S.mv[b].d = 5;
+                    mbar_arrive(&S.dv_full[b]);
+                    if (++b == kStages) { b = 0; ph ^= 1u; }
+                } else ok = false;
+            }
+            if (lane == 0 && ok && max_tiles > 0) ok = flag_wait_ge(&p.ctl->pull_done, (unsigned)p.nblk, p, 15);
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+        }
         for (int taken = 0; ok && taken < max_tiles; ++taken) {
             int mb = 0;
             if (lane == 0) mb = (int)atomicAdd(&p.ctl->q_disp, 1u);
@@ -533,8 +610,12 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
                     S.mv[b].a = row0 + r0; S.mv[b].b = nr; S.mv[b].c = mb; S.mv[b].d = (r0 + nr >= nrows) ? 1 : 0;
                     mbar_arrive_expect_tx(&S.dv_full[b], (uint32_t)nr * rowb);
                     const uint32_t dst = smem_u32(stages + b * kMvBuf);
-                    for (int i = 0; i < nr; ++i)
-                        bulk_load(dst + (uint32_t)i * rowb, p.x + (size_t)S.tok[r0 + i] * p.H, rowb, &S.dv_full[b]);
+                    for (int i = 0; i < nr; ++i) {
+                        const int tk = S.tok[r0 + i];
+                        // a remote token (another rank's shard) is read from its staged copy
+                        const __nv_bfloat16 *src = (p.ep_size > 1 && tk / p.ep_tshard != p.ep_rank) ? p.xs : p.x;
+                        bulk_load(dst + (uint32_t)i * rowb, src + (size_t)tk * p.H, rowb, &S.dv_full[b]);
+                    }
                     if (++b == kStages) { b = 0; ph ^= 1u; }
                 }
             }
@@ -555,7 +636,7 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
             int b = 0, n = 0;
             uint32_t ph = 0;
             int prev_buf = -1;
-            int pe_idx[kPend], pe_mb[kPend], pe_rows[kPend];      // tile ends not yet published
+            int pe_idx[kPend], pe_mb[kPend], pe_rows[kPend];      // tile ends not yet published (mb < 0: a staged block)
             unsigned long long pe_t0[kPend];
             for (int i = 0; i < kPend; ++i) { pe_idx[i] = 0; pe_mb[i] = 0; pe_rows[i] = 0; pe_t0[i] = 0ull; }
             int pe_head = 0, pe_tail = 0;
@@ -563,11 +644,13 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
                 bool fenced = false;
                 while (pe_head != pe_tail && pe_idx[pe_head % kPend] <= done_idx) {
                     const int s8 = pe_head % kPend;
-                    if (pe_mb[s8] != p.withhold_mb) {
-                        if (!fenced) { fence_proxy_async(); __threadfence(); fenced = true; }
-                        st_release_u32(&p.xe_ready[pe_mb[s8]], 1u);
+                    if (!fenced) { fence_proxy_async(); __threadfence(); fenced = true; }
+                    if (pe_mb[s8] < 0) {
+                        red_release_add_u32(&p.ctl->pull_done, 1u);      // a block of remote tokens is staged
+                    } else {
+                        if (pe_mb[s8] != p.withhold_mb) st_release_u32(&p.xe_ready[pe_mb[s8]], 1u);
+                        trace_ev(p, S, kEvDispatch, (unsigned)pe_mb[s8], pe_t0[s8], trace_now(p), (unsigned)pe_rows[s8]);
                     }
-                    trace_ev(p, S, kEvDispatch, (unsigned)pe_mb[s8], pe_t0[s8], trace_now(p), (unsigned)pe_rows[s8]);
                     ++pe_head;
                 }
             };
@@ -576,14 +659,27 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
                 if (!mbar_wait(&S.dv_full[b], ph, p, 13)) break;
                 const int da = S.mv[b].a, db = S.mv[b].b, dc = S.mv[b].c, dd = S.mv[b].d;
                 if (dd == 2) break;
-                bulk_store(p.xe + (size_t)da * p.H, smem_u32(stages + b * kMvBuf), (uint32_t)db * rowb);
+                if (dd == 5) {      // flush: everything stored so far becomes visible and is published
+                    bulk_wait<0>();
+                    if (prev_buf >= 0) { mbar_arrive(&S.dv_empty[prev_buf]); prev_buf = -1; }
+                    publish_upto(n);
+                    mbar_arrive(&S.dv_empty[b]);
+                    if (++b == kStages) { b = 0; ph ^= 1u; }
+                    continue;
+                }
+                if (dd >= 3) {      // staged remote tokens: one store per row, to the token's own slot of xs
+                    for (int i = 0; i < db; ++i)
+                        bulk_store(p.xs + (size_t)S.mv[b].tok[i] * p.H, smem_u32(stages + b * kMvBuf) + (uint32_t)i * rowb, rowb);
+                } else {
+                    bulk_store(p.xe + (size_t)da * p.H, smem_u32(stages + b * kMvBuf), (uint32_t)db * rowb);
+                }
                 bulk_commit();
                 if (prev_buf >= 0) { bulk_wait_read<1>(); mbar_arrive(&S.dv_empty[prev_buf]); }
                 prev_buf = b;
-                if (dd == 1) {
+                if (dd == 1 || dd == 4) {
                     if (pe_tail - pe_head == kPend) { bulk_wait<0>(); publish_upto(n); }
                     const int s8 = pe_tail % kPend;
-                    pe_idx[s8] = n; pe_mb[s8] = dc; pe_rows[s8] = db; pe_t0[s8] = tile_t0;
+                    pe_idx[s8] = n; pe_mb[s8] = dd == 4 ? -1 : dc; pe_rows[s8] = db; pe_t0[s8] = tile_t0;
                     ++pe_tail;
                     tile_t0 = trace_now(p);
                 }
@@ -654,12 +750,18 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uin
                         const int w = min(W, p.H - col0);
                         if (!mbar_wait(&S.cb_empty[b], ph ^ 1u, p, 22)) { ok = false; break; }
                         S.mv[b].a = t0 + tt; S.mv[b].b = col0; S.mv[b].c = w; S.mv[b].d = 0;
-                        for (int j = 0; j < kk; ++j) S.mv[b].g[j] = S.cgate[tt][j];
-                        mbar_arrive_expect_tx(&S.cb_full[b], (uint32_t)(kk * w * 2));
-                        const uint32_t dst = smem_u32(stages + b * kMvBuf);
+                        int nv = 0;      // slots whose expert lives on another rank have row -1 and are skipped
                         for (int j = 0; j < kk; ++j)
-                            bulk_load(dst + (uint32_t)(j * w * 2), p.y + (size_t)S.crow[tt][j] * p.H + col0,
-                                      (uint32_t)(w * 2), &S.cb_full[b]);
+                            if (S.crow[tt][j] >= 0) S.mv[b].g[nv++] = S.cgate[tt][j];
+                        S.mv[b].n = nv;
+                        if (nv > 0) mbar_arrive_expect_tx(&S.cb_full[b], (uint32_t)(nv * w * 2));
+                        else mbar_arrive(&S.cb_full[b]);
+                        const uint32_t dst = smem_u32(stages + b * kMvBuf);
+                        int q2 = 0;
+                        for (int j = 0; j < kk; ++j)
+                            if (S.crow[tt][j] >= 0)
+                                bulk_load(dst + (uint32_t)((q2++) * w * 2), p.y + (size_t)S.crow[tt][j] * p.H + col0,
+                                          (uint32_t)(w * 2), &S.cb_full[b]);
                         if (++b == kStages) { b = 0; ph ^= 1u; }
                     }
                 }
@@ -685,14 +787,14 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uin
             if (!ok) break;
             const MvDesc &d = S.mv[b];
             if (d.d == 2) break;
-            const int w = d.c, nv = w >> 3;
+            const int w = d.c, nv = w >> 3, nrow = d.n;
             const uint32_t src = smem_u32(stages + b * kMvBuf);
             __nv_bfloat16 *dst = p.out + (size_t)d.a * p.H + d.b;
             for (int v = ctid; v < nv; v += kCombWarps * 32) {
                 float a0[8];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) a0[i] = 0.f;
-                for (int j = 0; j < kk; ++j) {
+                for (int j = 0; j < nrow; ++j) {
                     const uint4 q4 = ld_shared_v4(src + (uint32_t)(j * w * 2 + v * 16));
                     const float gw = d.g[j];
                     a0[0] = fmaf(gw, bf16lo_to_f32(q4.x), a0[0]); a0[1] = fmaf(gw, bf16hi_to_f32(q4.x), a0[1]);
@@ -1136,27 +1238,36 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
     const unsigned long long tk0 = trace_now(p);
 
     // routing scratch lives in the (not yet used) stage buffers
-    unsigned long long *r_mask = reinterpret_cast<unsigned long long *>(stages);          // [256]
-    int *r_idx = reinterpret_cast<int *>(stages + 2048);                                   // [64][16]
-    int *r_base = reinterpret_cast<int *>(stages + 2048 + kRouteBlock * kMaxTopK * 4);     // [256]
+    unsigned long long *r_mask = reinterpret_cast<unsigned long long *>(stages);          // [256] + 1 (remote tokens)
+    int *r_idx = reinterpret_cast<int *>(stages + 2048 + 64);                              // [64][16]
+    int *r_base = reinterpret_cast<int *>(stages + 2048 + 64 + kRouteBlock * kMaxTopK * 4);    // [256]
+    int *r_cnt = r_base + kMaxEE;                                                          // [2] local / remote pairs
 
     // ================= phase R: routing
     for (int b = blockIdx.x; b < p.nblk; b += n_sm) {
         for (int e = tid; e < EE; e += kThreads) r_mask[e] = 0ull;
+        if (tid == 0) { r_mask[kMaxEE] = 0ull; r_cnt[0] = 0; r_cnt[1] = 0; }
         __syncthreads();
-        if (p.E <= 32) route_block_tokens<1>(p, b, r_mask, r_idx);
-        else if (p.E <= 64) route_block_tokens<2>(p, b, r_mask, r_idx);
-        else if (p.E <= 128) route_block_tokens<4>(p, b, r_mask, r_idx);
-        else route_block_tokens<8>(p, b, r_mask, r_idx);
+        if (p.E <= 32) route_block_tokens<1>(p, b, r_mask, r_idx, r_cnt);
+        else if (p.E <= 64) route_block_tokens<2>(p, b, r_mask, r_idx, r_cnt);
+        else if (p.E <= 128) route_block_tokens<4>(p, b, r_mask, r_idx, r_cnt);
+        else route_block_tokens<8>(p, b, r_mask, r_idx, r_cnt);
         __syncthreads();
         // in-block rank of each (token, slot): tokens before it in the block that chose the same expert
         for (int pi = tid; pi < kRouteBlock * p.k; pi += kThreads) {
             const int tl = pi / p.k, j = pi - tl * p.k;
             const int t = b * kRouteBlock + tl;
             if (t < p.T) {
-                const int e = r_idx[tl * kMaxTopK + j];
-                p.row_of[(size_t)t * p.k + j] = __popcll(r_mask[e] & ((1ull << tl) - 1ull));
+                const int e = r_idx[tl * kMaxTopK + j];     // -1: the expert lives on another rank
+                p.row_of[(size_t)t * p.k + j] = e >= 0 ? __popcll(r_mask[e] & ((1ull << tl) - 1ull)) : -1;
             }
+        }
+        if (p.ep_size > 1 && tid == 0) {
+            const unsigned long long um = r_mask[kMaxEE];
+            p.uniq_mask[b] = um;
+            if (r_cnt[0]) atomicAdd(&p.ctl->x_local, (unsigned)r_cnt[0]);
+            if (r_cnt[1]) atomicAdd(&p.ctl->x_in, (unsigned)r_cnt[1]);
+            if (um) atomicAdd(&p.ctl->x_in_uniq, (unsigned)__popcll(um));
         }
         const int ntok = min(kRouteBlock, p.T - b * kRouteBlock);
         const int f = (b * kFine) / p.nblk;
@@ -1218,14 +1329,26 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
     __syncthreads();     // red_i is reused by the arg-min below
 
     const int P = p.T * (p.k + p.S);
+    const unsigned ep_xl = alive ? __ldcg(&p.ctl->x_local) : 0u, ep_xi = alive ? __ldcg(&p.ctl->x_in) : 0u,
+                   ep_xu = alive ? __ldcg(&p.ctl->x_in_uniq) : 0u;
+    if (blockIdx.x == 0 && tid == 0) { p.ctl->ep_x_local = ep_xl; p.ctl->ep_x_in = ep_xi; p.ctl->ep_x_in_uniq = ep_xu; }
     int plan_c, plan_ki, plan_steal;
     float plan_t = 0.f;
     if (p.mode == kModeAuto) {
         // Eq. 1-3 (single-GPU reading: every pair moves through HBM), then Eq. 16 over the grid
         const float B = (float)(2 * p.H);
-        const float w_comp = __fmul_rn(__fmul_rn(__fmul_rn((float)P, 6.0f), (float)p.H), (float)p.I);
-        const float w_disp = __fmul_rn((float)(p.T + P), B);
-        const float w_comb = __fmul_rn((float)(P + p.T), B);
+        float w_comp, w_disp, w_comb;
+        if (p.ep_size > 1) {
+            // Eq. 1-3 literally: X_local + X_in pairs are computed here, each unique remote token is
+            // pulled once, one result goes back per remote pair
+            w_comp = __fmul_rn(__fmul_rn(__fmul_rn((float)(ep_xl + ep_xi), 6.0f), (float)p.H), (float)p.I);
+            w_disp = __fmul_rn((float)ep_xu, B);
+            w_comb = __fmul_rn((float)ep_xi, B);
+        } else {
+            w_comp = __fmul_rn(__fmul_rn(__fmul_rn((float)P, 6.0f), (float)p.H), (float)p.I);
+            w_disp = __fmul_rn((float)(p.T + P), B);
+            w_comb = __fmul_rn((float)(P + p.T), B);
+        }
         const int ci = tid >> 2, ki = tid & 3;
         const int cc = p.c_min + ci * p.c_step;
         float t = __int_as_float(0x7f800000);
@@ -1330,9 +1453,12 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
                 const int t = b * kRouteBlock + tl;
                 if (t < p.T) {
                     const int e = __ldcg(p.topk_idx + (size_t)t * p.k + j);
-                    const int r = __ldcg(p.row_of + (size_t)t * p.k + j) + r_base[e];
-                    p.row_of[(size_t)t * p.k + j] = r;
-                    p.token_of[r] = t;
+                    const int rk = __ldcg(p.row_of + (size_t)t * p.k + j);
+                    if (rk >= 0) {
+                        const int r = rk + r_base[e];
+                        p.row_of[(size_t)t * p.k + j] = r;
+                        p.token_of[r] = t;
+                    }
                 }
             }
             for (int pi = tid; pi < kRouteBlock * p.S; pi += kThreads) {

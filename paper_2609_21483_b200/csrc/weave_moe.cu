@@ -22,7 +22,7 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 struct Layout {
     size_t ctl, fcnt, xe_ready, h_ready, zero_end;       // [0, zero_end) is zeroed at create / recovery
-    size_t hist, topk, gates, row_of, token_of, counts, offsets, bw, tf;
+    size_t hist, topk, gates, row_of, token_of, counts, offsets, bw, tf, uniq_mask, xs;
     size_t xe, hbuf, y, st_x, st_logits, st_out, total;
     int nmb_max, nblk_max, p_max;
 };
@@ -68,6 +68,8 @@ Layout make_layout(const weave_moe_config *c)
     L.offsets = take(sizeof(int) * (EE + 1), 256);
     L.bw = take(sizeof(float) * 1024, 256);
     L.tf = take(sizeof(float) * 1024, 256);
+    L.uniq_mask = take(sizeof(unsigned long long) * (size_t)L.nblk_max, 256);
+    L.xs = take(T * c->hidden * 2, 1024);       // expert-parallel share: staged copies of remote tokens
     L.xe = take((size_t)L.p_max * c->hidden * 2, 1024);
     L.hbuf = take((size_t)L.p_max * c->ffn * 2, 1024);
     L.y = take((size_t)L.p_max * c->hidden * 2, 1024);
@@ -101,6 +103,7 @@ struct weave_moe {
     int last_cuda_error;
     void *trace;
     int trace_cap;
+    int ep_rank, ep_size;
     CUtensorMap tm_xe, tm_wgu, tm_h, tm_wd, tm_wgu64;
 };
 
@@ -209,6 +212,8 @@ int weave_moe_create(const weave_moe_config *cfg, weave_moe_t *out)
     h->last_cuda_error = 0;
     h->trace = nullptr;
     h->trace_cap = 0;
+    h->ep_rank = 0;
+    h->ep_size = 1;
 
     e = cudaFuncSetAttribute(weave_moe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) { int rc = cuda_fail(h, e); delete h; return rc; }
@@ -297,6 +302,11 @@ int weave_moe_forward(weave_moe_t h, const void *x, const float *logits, void *o
     p.h_ready = reinterpret_cast<unsigned *>(ws + L.h_ready);
     p.bw = reinterpret_cast<const float *>(ws + L.bw);
     p.tf = reinterpret_cast<const float *>(ws + L.tf);
+    p.ep_rank = h->ep_rank;
+    p.ep_size = h->ep_size;
+    p.ep_tshard = (T + h->ep_size - 1) / h->ep_size;
+    p.xs = reinterpret_cast<__nv_bfloat16 *>(ws + L.xs);
+    p.uniq_mask = reinterpret_cast<unsigned long long *>(ws + L.uniq_mask);
     p.trace = reinterpret_cast<uint4 *>(h->trace);
     p.trace_cap = h->trace_cap;
 
@@ -444,6 +454,29 @@ int weave_moe_status(weave_moe_t h)
     return st;
 }
 
+int weave_moe_set_expert_parallel(weave_moe_t h, int ep_rank, int ep_size)
+{
+    if (!h || ep_size < 1 || ep_rank < 0 || ep_rank >= ep_size) return WEAVE_ERR_INVALID_ARG;
+    if (ep_size > 1 && (h->cfg.num_experts % ep_size != 0 || h->cfg.num_shared != 0)) return WEAVE_ERR_INVALID_ARG;
+    h->ep_rank = ep_rank;
+    h->ep_size = ep_size;
+    return WEAVE_OK;
+}
+
+int weave_moe_get_ep_descriptors(weave_moe_t h, long long *x_local, long long *x_in, long long *x_in_uniq)
+{
+    if (!h) return WEAVE_ERR_INVALID_ARG;
+    cudaError_t e = cudaStreamSynchronize(h->last_stream);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    Ctl ctl;
+    e = cudaMemcpy(&ctl, h->ws + h->L.ctl, sizeof(Ctl), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    if (x_local) *x_local = ctl.ep_x_local;
+    if (x_in) *x_in = ctl.ep_x_in;
+    if (x_in_uniq) *x_in_uniq = ctl.ep_x_in_uniq;
+    return WEAVE_OK;
+}
+
 int weave_moe_set_sm_count(weave_moe_t h, int n_sm)
 {
     if (!h) return WEAVE_ERR_INVALID_ARG;
@@ -578,6 +611,8 @@ int weave_moe_forward_static(int hidden, int ffn, int num_experts, int top_k, in
     h.eff[0] = 1.0f; h.eff[1] = 0.90f; h.eff[2] = 0.80f; h.eff[3] = 0.65f;
     h.timeout_ms = 4000;
     h.withhold_mb = -1;
+    h.ep_rank = 0;
+    h.ep_size = 1;
     const int EE = num_experts + num_shared;
     int r = 0;
     r |= encode_map(sd->encode, &h.tm_xe, h.ws + L.xe, (uint64_t)L.p_max, (uint64_t)hidden, false);
