@@ -88,6 +88,19 @@ int weave_moe_forward(weave_moe_t h, const void *x, const float *router_logits, 
 int weave_moe_forward_host(weave_moe_t h, const void *x_host, const float *router_logits_host,
                            void *out_host, int T, void *cuda_stream);
 
+/* Throughput variant of weave_moe_forward_host for back-to-back calls: the copies run on two
+ * internal copy streams (created on first use, destroyed with the handle) and two staging slots
+ * alternate, so the H2D copy of call i+1 and the D2H copy of call i-1 overlap the kernel of call
+ * i; the kernels stay ordered on cuda_stream.  out_host of a call is complete once
+ * weave_moe_host_wait() returns (or after two further pipelined calls have been waited for);
+ * synchronising cuda_stream alone does NOT cover the last D2H copy.  Host buffers must be pinned
+ * and stay valid until then. */
+int weave_moe_forward_host_pipelined(weave_moe_t h, const void *x_host, const float *router_logits_host,
+                                     void *out_host, int T, void *cuda_stream);
+
+/* Blocks until the output copies of all pipelined calls made so far have arrived in host memory. */
+int weave_moe_host_wait(weave_moe_t h);
+
 /* Releases host state.  Does not touch device memory. */
 int weave_moe_destroy(weave_moe_t h);
 

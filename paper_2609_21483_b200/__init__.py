@@ -61,6 +61,7 @@ EXPORTS = [
     "weave_moe_last_cuda_error", "weave_moe_strerror", "weave_moe_set_trace",
     "weave_moe_forward_static", "weave_moe_static_scratch_bytes", "weave_moe_set_sm_count",
     "weave_moe_set_expert_parallel", "weave_moe_get_ep_descriptors",
+    "weave_moe_forward_host_pipelined", "weave_moe_host_wait",
 ]
 
 
@@ -83,6 +84,10 @@ def load():
     lib.weave_moe_forward.argtypes = [vp, vp, vp, vp, ci, vp]
     lib.weave_moe_forward_host.restype = ci
     lib.weave_moe_forward_host.argtypes = [vp, vp, vp, vp, ci, vp]
+    lib.weave_moe_forward_host_pipelined.restype = ci
+    lib.weave_moe_forward_host_pipelined.argtypes = [vp, vp, vp, vp, ci, vp]
+    lib.weave_moe_host_wait.restype = ci
+    lib.weave_moe_host_wait.argtypes = [vp]
     lib.weave_moe_destroy.restype = ci
     lib.weave_moe_destroy.argtypes = [vp]
     lib.weave_moe_set_schedule.restype = ci
@@ -232,6 +237,25 @@ class WeaveMoE:
                                                 out_host.data_ptr(), T, stream), "weave_moe_forward_host")
         self.last_T = T
         return out_host
+
+    def forward_host_pipelined(self, x_host, logits_host, out_host, stream: Optional[int] = None):
+        """Like forward_host, but copies overlap the neighbouring calls' kernels; call host_wait()
+        before reading out_host."""
+        torch = self._torch
+        T = x_host.shape[0]
+        assert x_host.is_pinned() and logits_host.is_pinned() and out_host.is_pinned()
+        assert x_host.dtype == torch.bfloat16 and logits_host.dtype == torch.float32 and out_host.dtype == torch.bfloat16
+        assert x_host.is_contiguous() and logits_host.is_contiguous() and out_host.is_contiguous()
+        if stream is None:
+            stream = torch.cuda.current_stream(self.gate_up.device).cuda_stream
+        _check(self._lib.weave_moe_forward_host_pipelined(self._h, x_host.data_ptr(), logits_host.data_ptr(),
+                                                          out_host.data_ptr(), T, stream),
+               "weave_moe_forward_host_pipelined")
+        self.last_T = T
+        return out_host
+
+    def host_wait(self):
+        _check(self._lib.weave_moe_host_wait(self._h), "weave_moe_host_wait")
 
     # ---- scheduling
     def set_schedule(self, mode: int, c: int = 0, K: int = 1, steal: int = 0):

@@ -23,7 +23,7 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 struct Layout {
     size_t ctl, fcnt, xe_ready, h_ready, zero_end;       // [0, zero_end) is zeroed at create / recovery
     size_t hist, topk, gates, row_of, token_of, counts, offsets, bw, tf, uniq_mask, xs;
-    size_t xe, hbuf, y, st_x, st_logits, st_out, total;
+    size_t xe, hbuf, y, st_x, st_logits, st_out, st2_x, st2_logits, st2_out, total;
     int nmb_max, nblk_max, p_max;
 };
 
@@ -76,6 +76,9 @@ Layout make_layout(const weave_moe_config *c)
     L.st_x = take(T * c->hidden * 2, 1024);
     L.st_logits = take(T * c->num_experts * 4, 1024);
     L.st_out = take(T * c->hidden * 2, 1024);
+    L.st2_x = take(T * c->hidden * 2, 1024);          // second staging slot of the pipelined host path
+    L.st2_logits = take(T * c->num_experts * 4, 1024);
+    L.st2_out = take(T * c->hidden * 2, 1024);
     L.total = align_up(o, 1024);
     return L;
 }
@@ -104,6 +107,11 @@ struct weave_moe {
     void *trace;
     int trace_cap;
     int ep_rank, ep_size;
+    // pipelined host path: copy streams and per-slot events, created on first use
+    bool pipe_ready;
+    unsigned long long pipe_calls;
+    cudaStream_t pipe_h2d, pipe_d2h;
+    cudaEvent_t pipe_in_ready[2], pipe_k_done[2], pipe_out_done[2];
     CUtensorMap tm_xe, tm_wgu, tm_h, tm_wd, tm_wgu64;
 };
 
@@ -214,6 +222,8 @@ int weave_moe_create(const weave_moe_config *cfg, weave_moe_t *out)
     h->trace_cap = 0;
     h->ep_rank = 0;
     h->ep_size = 1;
+    h->pipe_ready = false;
+    h->pipe_calls = 0;
 
     e = cudaFuncSetAttribute(weave_moe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) { int rc = cuda_fail(h, e); delete h; return rc; }
@@ -346,8 +356,76 @@ int weave_moe_forward_host(weave_moe_t h, const void *x_host, const float *logit
     return WEAVE_OK;
 }
 
+/* Throughput-oriented host path: the copies run on two internal copy streams and two staging
+ * slots alternate, so that the H2D copy of call i+1 and the D2H copy of call i-1 overlap the
+ * kernel of call i (the kernels themselves stay ordered on the caller's stream). */
+int weave_moe_forward_host_pipelined(weave_moe_t h, const void *x_host, const float *logits_host, void *out_host,
+                                     int T, void *stream)
+{
+    if (!h) return WEAVE_ERR_INVALID_ARG;
+    if (T < 0 || T > h->cfg.max_tokens) return WEAVE_ERR_INVALID_ARG;
+    if (T == 0) return WEAVE_OK;
+    if (!x_host || !logits_host || !out_host) return WEAVE_ERR_INVALID_ARG;
+    cudaError_t e;
+    if (!h->pipe_ready) {
+        if ((e = cudaStreamCreateWithFlags(&h->pipe_h2d, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(h, e);
+        if ((e = cudaStreamCreateWithFlags(&h->pipe_d2h, cudaStreamNonBlocking)) != cudaSuccess) return cuda_fail(h, e);
+        for (int i = 0; i < 2; ++i) {
+            if ((e = cudaEventCreateWithFlags(&h->pipe_in_ready[i], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(h, e);
+            if ((e = cudaEventCreateWithFlags(&h->pipe_k_done[i], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(h, e);
+            if ((e = cudaEventCreateWithFlags(&h->pipe_out_done[i], cudaEventDisableTiming)) != cudaSuccess) return cuda_fail(h, e);
+        }
+        h->pipe_ready = true;
+        h->pipe_calls = 0;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const weave_moe_config &c = h->cfg;
+    const Layout &L = h->L;
+    uint8_t *ws = h->ws;
+    const int slot = (int)(h->pipe_calls & 1ull);
+    uint8_t *sx = ws + (slot ? L.st2_x : L.st_x), *sl = ws + (slot ? L.st2_logits : L.st_logits),
+            *so = ws + (slot ? L.st2_out : L.st_out);
+    const size_t xb = (size_t)T * c.hidden * 2, lb = (size_t)T * c.num_experts * 4;
+    // the slot's inputs may be overwritten once the kernel that read them (two calls ago) is done
+    if (h->pipe_calls >= 2 && (e = cudaStreamWaitEvent(h->pipe_h2d, h->pipe_k_done[slot], 0)) != cudaSuccess) return cuda_fail(h, e);
+    if ((e = cudaMemcpyAsync(sx, x_host, xb, cudaMemcpyHostToDevice, h->pipe_h2d)) != cudaSuccess) return cuda_fail(h, e);
+    if ((e = cudaMemcpyAsync(sl, logits_host, lb, cudaMemcpyHostToDevice, h->pipe_h2d)) != cudaSuccess) return cuda_fail(h, e);
+    if ((e = cudaEventRecord(h->pipe_in_ready[slot], h->pipe_h2d)) != cudaSuccess) return cuda_fail(h, e);
+    // the kernel needs its inputs, and its output slot must have been copied out (two calls ago)
+    if ((e = cudaStreamWaitEvent(st, h->pipe_in_ready[slot], 0)) != cudaSuccess) return cuda_fail(h, e);
+    if (h->pipe_calls >= 2 && (e = cudaStreamWaitEvent(st, h->pipe_out_done[slot], 0)) != cudaSuccess) return cuda_fail(h, e);
+    int rc = weave_moe_forward(h, sx, reinterpret_cast<const float *>(sl), so, T, stream);
+    if (rc) return rc;
+    if ((e = cudaEventRecord(h->pipe_k_done[slot], st)) != cudaSuccess) return cuda_fail(h, e);
+    if ((e = cudaStreamWaitEvent(h->pipe_d2h, h->pipe_k_done[slot], 0)) != cudaSuccess) return cuda_fail(h, e);
+    if ((e = cudaMemcpyAsync(out_host, so, xb, cudaMemcpyDeviceToHost, h->pipe_d2h)) != cudaSuccess) return cuda_fail(h, e);
+    if ((e = cudaEventRecord(h->pipe_out_done[slot], h->pipe_d2h)) != cudaSuccess) return cuda_fail(h, e);
+    h->pipe_calls += 1;
+    return WEAVE_OK;
+}
+
+int weave_moe_host_wait(weave_moe_t h)
+{
+    if (!h) return WEAVE_ERR_INVALID_ARG;
+    if (!h->pipe_ready || h->pipe_calls == 0) return WEAVE_OK;
+    cudaError_t e = cudaStreamSynchronize(h->pipe_d2h);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    return WEAVE_OK;
+}
+
 int weave_moe_destroy(weave_moe_t h)
 {
+    if (h && h->pipe_ready) {
+        cudaStreamSynchronize(h->pipe_d2h);
+        cudaStreamSynchronize(h->pipe_h2d);
+        for (int i = 0; i < 2; ++i) {
+            cudaEventDestroy(h->pipe_in_ready[i]);
+            cudaEventDestroy(h->pipe_k_done[i]);
+            cudaEventDestroy(h->pipe_out_done[i]);
+        }
+        cudaStreamDestroy(h->pipe_h2d);
+        cudaStreamDestroy(h->pipe_d2h);
+    }
     delete h;
     return WEAVE_OK;
 }

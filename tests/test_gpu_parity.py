@@ -231,6 +231,31 @@ def test_forward_host_equals_forward():
     moe.close()
 
 
+def test_pipelined_host_path_keeps_batches_apart():
+    """Five different batches back to back through the pipelined host path (two staging slots,
+    copies overlapping the neighbouring kernels): every output equals the device path's."""
+    cfg = _small("pipe", 384, 256, 384, 16, 4)
+    inp = wl.make_inputs(cfg)
+    x, lg, gu, dn = to_dev(inp)
+    moe = pk.WeaveMoE(gu, dn, cfg.E, cfg.k, cfg.S, max_tokens=cfg.T)
+    xs, ls, refs, outs = [], [], [], []
+    for i in range(5):
+        T = cfg.T - 37 * i
+        xi = torch.roll(x, shifts=i * 11, dims=0)[:T].contiguous()
+        li = torch.roll(lg, shifts=i * 5, dims=0)[:T].contiguous()
+        refs.append(moe.forward(xi, li).clone())
+        moe.check()
+        xs.append(xi.cpu().pin_memory()); ls.append(li.cpu().pin_memory())
+        outs.append(torch.zeros(T, cfg.H, dtype=torch.bfloat16).pin_memory())
+    for i in range(5):
+        moe.forward_host_pipelined(xs[i], ls[i], outs[i])
+    moe.host_wait()
+    moe.check()
+    for i in range(5):
+        assert torch.equal(outs[i].view(torch.int16), refs[i].cpu().view(torch.int16)), f"batch {i}"
+    moe.close()
+
+
 # ------------------------------------------------------------------ cost model and scheduler
 
 def _n_tiles_of_K(counts_fine, geo, H, I):
