@@ -126,6 +126,20 @@ def test_shape_edges(H, I, E, k, S):
     moe.close()
 
 
+def test_many_tokens_small_experts():
+    """A long batch (625 routing blocks, 8 fine chunks of 78-79 blocks, ~80 000 rows) on small
+    experts, chunked and unchunked: exercises the block/chunk prefix machinery at size."""
+    cfg = _small("long", 40000, 128, 128, 8, 2, zipf=0.7)
+    inp = wl.make_inputs(cfg)
+    dev = to_dev(inp)
+    moe, out0, _ = run_case(cfg, inp=inp, dev_tensors=dev)
+    bits = out0.view(torch.int16).clone()
+    for s in [(pk.SCHED_FIXED, 40, 8, 2), (pk.SCHED_SERIAL, 0, 1, 0)]:
+        _, out, _ = run_case(cfg, sched=s, inp=inp, dev_tensors=dev, moe=moe)
+        assert torch.equal(out.view(torch.int16), bits)
+    moe.close()
+
+
 def test_all_tokens_to_one_expert_and_ties():
     """Degenerate routing: (a) every token picks experts 3 and 5 (two huge segments, the rest
     empty); (b) all logits equal, so ties decide everything (indices 0..k-1)."""
