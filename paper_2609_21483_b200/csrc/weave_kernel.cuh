@@ -593,6 +593,9 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
             }
             if (lane == 0 && ok && max_tiles > 0) ok = flag_wait_ge(&p.ctl->pull_done, (unsigned)p.nblk, p, 15);
             ok = __shfl_sync(0xffffffffu, ok, 0);
+            // only lane 0 walked the ring so far; from here on every lane addresses the buffers
+            b = __shfl_sync(0xffffffffu, b, 0);
+            ph = __shfl_sync(0xffffffffu, ph, 0);
         }
         for (int taken = 0; ok && taken < max_tiles; ++taken) {
             int mb = 0;
@@ -603,21 +606,26 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
             decode_mblock(S, p.EE, mb, row0, nrows);
             for (int i = lane; i < nrows; i += 32) S.tok[i] = __ldcg(p.token_of + row0 + i);
             __syncwarp();
-            if (lane == 0) {
-                for (int r0 = 0; r0 < nrows; r0 += R) {
-                    const int nr = min(R, nrows - r0);
-                    if (!mbar_wait(&S.dv_empty[b], ph ^ 1u, p, 11)) { ok = false; break; }
-                    S.mv[b].a = row0 + r0; S.mv[b].b = nr; S.mv[b].c = mb; S.mv[b].d = (r0 + nr >= nrows) ? 1 : 0;
-                    mbar_arrive_expect_tx(&S.dv_full[b], (uint32_t)nr * rowb);
-                    const uint32_t dst = smem_u32(stages + b * kMvBuf);
-                    for (int i = 0; i < nr; ++i) {
-                        const int tk = S.tok[r0 + i];
-                        // a remote token (another rank's shard) is read from its staged copy
-                        const __nv_bfloat16 *src = (p.ep_size > 1 && tk / p.ep_tshard != p.ep_rank) ? p.xs : p.x;
-                        bulk_load(dst + (uint32_t)i * rowb, src + (size_t)tk * p.H, rowb, &S.dv_full[b]);
+            for (int r0 = 0; r0 < nrows && ok; r0 += R) {
+                const int nr = min(R, nrows - r0);
+                if (lane == 0) {
+                    if (!mbar_wait(&S.dv_empty[b], ph ^ 1u, p, 11)) ok = false;
+                    else {
+                        S.mv[b].a = row0 + r0; S.mv[b].b = nr; S.mv[b].c = mb; S.mv[b].d = (r0 + nr >= nrows) ? 1 : 0;
+                        mbar_arrive_expect_tx(&S.dv_full[b], (uint32_t)nr * rowb);
                     }
-                    if (++b == kStages) { b = 0; ph ^= 1u; }
                 }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                // the expected byte count is registered; the lanes issue the row copies side by side
+                const uint32_t dst = smem_u32(stages + b * kMvBuf);
+                for (int i = lane; i < nr; i += 32) {
+                    const int tk = S.tok[r0 + i];
+                    // a remote token (another rank's shard) is read from its staged copy
+                    const __nv_bfloat16 *src = (p.ep_size > 1 && tk / p.ep_tshard != p.ep_rank) ? p.xs : p.x;
+                    bulk_load(dst + (uint32_t)i * rowb, src + (size_t)tk * p.H, rowb, &S.dv_full[b]);
+                }
+                if (++b == kStages) { b = 0; ph ^= 1u; }
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
             __syncwarp();
@@ -744,29 +752,37 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uin
                 S.cgate[tt][j] = j < p.k ? __ldcg(p.gates + (size_t)t * p.k + j) : 1.0f;
             }
             __syncwarp();
-            if (lane == 0) {
-                for (int tt = 0; tt < ntok && ok; ++tt) {
-                    for (int col0 = 0; col0 < p.H; col0 += W) {
-                        const int w = min(W, p.H - col0);
-                        if (!mbar_wait(&S.cb_empty[b], ph ^ 1u, p, 22)) { ok = false; break; }
-                        S.mv[b].a = t0 + tt; S.mv[b].b = col0; S.mv[b].c = w; S.mv[b].d = 0;
-                        int nv = 0;      // slots whose expert lives on another rank have row -1 and are skipped
-                        for (int j = 0; j < kk; ++j)
-                            if (S.crow[tt][j] >= 0) S.mv[b].g[nv++] = S.cgate[tt][j];
-                        S.mv[b].n = nv;
+            for (int tt = 0; tt < ntok && ok; ++tt) {
+                // lane j owns slot j of the token: its rank among the slots that have a row here (slots
+                // whose expert lives on another rank have row -1 and are skipped)
+                const int myrow = lane < kk ? S.crow[tt][lane] : -1;
+                const unsigned vmask = __ballot_sync(0xffffffffu, myrow >= 0);
+                const int nv = __popc(vmask), mypos = __popc(vmask & ((1u << lane) - 1u));
+                for (int col0 = 0; col0 < p.H && ok; col0 += W) {
+                    const int w = min(W, p.H - col0);
+                    if (lane == 0) {
+                        if (!mbar_wait(&S.cb_empty[b], ph ^ 1u, p, 22)) ok = false;
+                        else {
+                            S.mv[b].a = t0 + tt; S.mv[b].b = col0; S.mv[b].c = w; S.mv[b].d = 0; S.mv[b].n = nv;
+                        }
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) break;
+                    if (myrow >= 0) S.mv[b].g[mypos] = S.cgate[tt][lane];
+                    __syncwarp();
+                    if (lane == 0) {
                         if (nv > 0) mbar_arrive_expect_tx(&S.cb_full[b], (uint32_t)(nv * w * 2));
                         else mbar_arrive(&S.cb_full[b]);
-                        const uint32_t dst = smem_u32(stages + b * kMvBuf);
-                        int q2 = 0;
-                        for (int j = 0; j < kk; ++j)
-                            if (S.crow[tt][j] >= 0)
-                                bulk_load(dst + (uint32_t)((q2++) * w * 2), p.y + (size_t)S.crow[tt][j] * p.H + col0,
-                                          (uint32_t)(w * 2), &S.cb_full[b]);
-                        if (++b == kStages) { b = 0; ph ^= 1u; }
                     }
+                    __syncwarp();
+                    // the byte count is registered; the lanes issue the row copies side by side
+                    if (myrow >= 0)
+                        bulk_load(smem_u32(stages + b * kMvBuf) + (uint32_t)(mypos * w * 2),
+                                  p.y + (size_t)myrow * p.H + col0, (uint32_t)(w * 2), &S.cb_full[b]);
+                    if (++b == kStages) { b = 0; ph ^= 1u; }
                 }
-                trace_ev(p, S, kEvCombine, (unsigned)q, tc0, trace_now(p), 0u);
             }
+            if (lane == 0) trace_ev(p, S, kEvCombine, (unsigned)q, tc0, trace_now(p), 0u);
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) break;
             __syncwarp();
