@@ -125,7 +125,9 @@ def calibrate(cfg, layer=0, verbose=True):
 
     def interp(pts, n_max):
         xs = np.array(sorted(pts))
-        ys = np.array([pts[v] for v in xs])
+        # more SMs are never modelled as slower than fewer (the extra ones could stay idle): measured
+        # rates of a small layer saturate and then wobble with the noise
+        ys = np.maximum.accumulate(np.array([pts[v] for v in xs]))
         grid = np.arange(n_max + 1, dtype=np.float64)
         out = np.interp(grid, np.concatenate([[0], xs]), np.concatenate([[0], ys]))
         out[0] = out[1]

@@ -180,7 +180,7 @@ __device__ __noinline__ void give_up(Ctl *ctl, int where)
 
 // Optional timeline: one 16-byte record {start ns, end ns, kind<<24 | id, extra} per event, per CTA.
 enum { kEvRoute = 1, kEvSetup = 2, kEvFixup = 3, kEvDispatch = 4, kEvGemmLoad = 5, kEvGemmEpi = 6,
-       kEvCombine = 7, kEvWaitChunk = 8, kEvBarrier = 9, kEvDepWait = 10 };
+       kEvCombine = 7, kEvWaitChunk = 8, kEvBarrier = 9, kEvDepWait = 10, kEvMma = 11 };
 __device__ __forceinline__ void trace_ev(const KParams &p, SmemTail &S, int kind, unsigned id,
                                          unsigned long long t0, unsigned long long t1, unsigned extra)
 {
@@ -460,56 +460,81 @@ __device__ __forceinline__ void decode_mblock(const SmemTail &S, int EE, int mb,
     nrows = min(kBM, S.seg_rows[s] - m * kBM);
 }
 
-// largest s in [lo, hi) with (seg_pt0[s] - base) * mul <= key
-__device__ __forceinline__ int seg_search_pt(const SmemTail &S, int lo, int hi, int base, int mul, int key)
+// number of regular (two-m-block) pair tiles / of unpaired m-blocks in the chunk's segments before s:
+// a segment with pts pair tiles has 2*pts - u m-blocks, u = 1 if its last m-block is unpaired
+__device__ __forceinline__ int seg_reg0(const SmemTail &S, int s, int cmb0, int cpt0)
 {
-    while (hi - lo > 1) {
-        int mid = (lo + hi) >> 1;
-        if ((S.seg_pt0[mid] - base) * mul <= key) lo = mid; else hi = mid;
-    }
-    return lo;
+    return (S.seg_mb0[s] - cmb0) - (S.seg_pt0[s] - cpt0);
+}
+__device__ __forceinline__ int seg_swap0(const SmemTail &S, int s, int cmb0, int cpt0)
+{
+    return 2 * (S.seg_pt0[s] - cpt0) - (S.seg_mb0[s] - cmb0);
 }
 
 // GEMM queue order (the chunk-pipeline DAG order): chunk by chunk; inside a chunk all gemm0 tiles,
-// then all gemm1 tiles; inside those expert-major, then groups of kPairGroup pair tiles, n-tile,
-// pair tile fastest (consecutive tiles share a weight panel, and a group's rows stay in L2 while
-// all its n-tiles pass).  A pair tile = two consecutive m-blocks of one segment: `lead` describes
-// the leader CTA's half, `peer` the other CTA's (nrows = 0, mb = -1 when the segment's m-block
-// count is odd and this is its last pair tile).
+// then all gemm1 tiles.  Inside those, two streams are interleaved at a constant ratio:
+//  - the regular pair tiles (two consecutive m-blocks of one segment), expert-major, then groups of
+//    kPairGroup pair tiles, n-tile, pair tile fastest (consecutive tiles share a weight panel, and a
+//    group's rows stay in L2 while all its n-tiles pass); these are bound by the tensor pipe;
+//  - the unpaired last m-blocks of the segments (operands swapped), expert-major, n-tile fastest;
+//    each streams a weight panel that nobody else reads, so they are bound by HBM.
+// Spreading the second stream evenly over the first keeps both resources busy all the time; in
+// expert order a run of small experts would leave the tensor pipes waiting on HBM, and a large
+// expert would leave HBM idle.  `lead` describes the leader CTA's half, `peer` the other CTA's.
 __device__ __forceinline__ void decode_pair_tile(const SmemTail &S, const KParams &p, int g, TileInfo &lead,
                                                  TileInfo &peer)
 {
     int j = 0;
     while (j + 1 < S.K && g >= S.chunk_tile0[j + 1]) ++j;
     int local = g - S.chunk_tile0[j];
-    const int cpt0 = S.chunk_pt0[j];
+    const int cpt0 = S.chunk_pt0[j], cmb0 = S.chunk_mb0[j];
     const int nptj = S.chunk_pt0[j + 1] - cpt0;
     int type = 0, nt = p.nt0;
     if (local >= nptj * p.nt0) { type = 1; local -= nptj * p.nt0; nt = p.nt1; }
-    const int s = seg_search_pt(S, j * p.EE, (j + 1) * p.EE, cpt0, nt, local);
-    const int pts = S.seg_pt0[s + 1] - S.seg_pt0[s];
-    const int within = local - (S.seg_pt0[s] - cpt0) * nt;
+    const long long n_sw = (long long)S.chunk_nswap[j] * nt, total = (long long)nptj * nt;
+    const int sw_before = (int)((local * n_sw) / total);
+    const bool swapped = (int)(((local + 1) * n_sw) / total) > sw_before;
+    lead.type = peer.type = type;
+    lead.chunk = peer.chunk = j;
+    lead.nkb = peer.nkb = (type == 0 ? p.H : p.I) / kBK;
+    int lo = j * p.EE, hi = (j + 1) * p.EE;
+    if (swapped) {
+        // both CTAs work on the one m-block with the operands swapped, so the MMA costs
+        // ceil(nrows/16)*16 columns instead of a half-empty 256-row tile
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (seg_swap0(S, mid, cmb0, cpt0) * nt <= sw_before) lo = mid; else hi = mid;
+        }
+        const int s = lo;
+        const int m0 = 2 * (S.seg_pt0[s + 1] - S.seg_pt0[s] - 1);
+        lead.type = type + 3;
+        lead.e = s - j * p.EE;
+        lead.n = sw_before - seg_swap0(S, s, cmb0, cpt0) * nt;
+        lead.mb = S.seg_mb0[s] + m0;
+        lead.row0 = S.seg_row0[s] + m0 * kBM;
+        lead.nrows = S.seg_rows[s] - m0 * kBM;
+        peer = lead;
+        return;
+    }
+    const int reg = local - sw_before;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (seg_reg0(S, mid, cmb0, cpt0) * nt <= reg) lo = mid; else hi = mid;
+    }
+    const int s = lo;
+    const int pts = seg_reg0(S, s + 1, cmb0, cpt0) - seg_reg0(S, s, cmb0, cpt0);
+    const int within = reg - seg_reg0(S, s, cmb0, cpt0) * nt;
     const int gi = within / (kPairGroup * nt);
     const int wg = within - gi * kPairGroup * nt;
     const int gsize = min(kPairGroup, pts - gi * kPairGroup);
     const int n = wg / gsize;
     const int m0 = 2 * (gi * kPairGroup + (wg - n * gsize));
     const int rows = S.seg_rows[s];
-    lead.type = peer.type = type;
     lead.e = peer.e = s - j * p.EE;
     lead.n = peer.n = n;
-    lead.chunk = peer.chunk = j;
-    lead.nkb = peer.nkb = (type == 0 ? p.H : p.I) / kBK;
     lead.mb = S.seg_mb0[s] + m0;
     lead.row0 = S.seg_row0[s] + m0 * kBM;
-    lead.nrows = min(kBM, rows - m0 * kBM);
-    if (rows - (m0 + 1) * kBM <= 0) {
-        // the segment's last, unpaired m-block: both CTAs work on it with the operands swapped,
-        // so the MMA costs ceil(nrows/16)*16 columns instead of a half-empty 256-row tile
-        lead.type = type + 3;
-        peer = lead;
-        return;
-    }
+    lead.nrows = kBM;
     peer.nrows = min(kBM, rows - (m0 + 1) * kBM);
     peer.mb = lead.mb + 1;
     peer.row0 = lead.row0 + kBM;
@@ -831,6 +856,10 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uin
 
 // ------------------------------------------------------------------------------------ phase B: GEMM
 
+// Tensor maps of the GEMM operands: bf16 matrices, boxes of 64 columns (one 128-byte swizzle row) by
+// 128 rows (64 rows for the gate and up halves of a swapped tile's weight operand).
+struct TmaMaps { CUtensorMap xe, wgu, h, wd, wgu64; };
+
 struct PipeState {     // per-role ring positions; they persist across the tiles of a phase
     int stage = 0;  uint32_t stage_phase = 0;
     int acc = 0;    uint32_t acc_phase = 0;
@@ -884,9 +913,7 @@ __device__ __forceinline__ void direct_store_32(const uint32_t (&o)[16], __nv_bf
 // budget = how many pair tiles this CTA pair may claim (the steal count for a movement pair).
 // Called by both CTAs of a pair with the same arguments.
 __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_t *stages, uint32_t tmem_base,
-                                           const CUtensorMap *tm_xe, const CUtensorMap *tm_wgu,
-                                           const CUtensorMap *tm_h, const CUtensorMap *tm_wd,
-                                           const CUtensorMap *tm_wgu64, int budget, PipeState &ps)
+                                           const TmaMaps *tm, int budget, PipeState &ps)
 {
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint32_t rank = cluster_ctarank();      // 0 = leader (issues the MMAs), 1 = peer
@@ -949,39 +976,45 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
         }
         __syncwarp();
     } else if (warp == 0) {
-        // ---------------- TMA producer (both CTAs): this CTA's 128 rows of A and its half of B
-        if (lane == 0) {
-            bool dead = false;
-            while (!dead) {
-                if (!mbar_wait_cluster(&S.ti_full[ps.slot], ps.slot_phase, p, 35)) { dead = true; break; }
-                const TileInfo ti = S.ti[ps.slot];
-                mbar_arrive_cluster(mapa_u32(smem_u32(&S.ti_empty[ps.slot]), 0u));
-                ps.next_slot();
-                if (ti.type == 2) break;
+        // ---------------- TMA producer (both CTAs): this CTA's 128 rows of A and its half of B;
+        // lane 0 issues the loads, the warp stays together tile by tile
+        bool dead = false;
+        while (!dead) {
+            bool ok = true;
+            if (lane == 0) ok = mbar_wait_cluster(&S.ti_full[ps.slot], ps.slot_phase, p, 35);
+            if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
+            const TileInfo ti = S.ti[ps.slot];
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(mapa_u32(smem_u32(&S.ti_empty[ps.slot]), 0u));
+            ps.next_slot();
+            if (ti.type == 2) break;
+            bool dead_l = false;
+            if (lane == 0) {
                 fence_proxy_async();     // rows written with ordinary stores elsewhere, read by TMA here
                 const CUtensorMap *tma_a, *tma_b;
                 int arow, brow, arow2 = -1;
-                const int nhalf = (((ti.nrows + 15) >> 4) << 4) >> 1;     // swapped tiles: rows per CTA on the N axis
+                // swapped tiles: rows per CTA on the N axis (the MMA's N, a multiple of 16, split in two)
+                const int nhalf = (((ti.nrows + 15) >> 4) << 4) >> 1;
                 if (ti.type == 0) {      // leader holds the gate rows of the n-tile, peer the up rows
-                    tma_a = tm_xe; tma_b = tm_wgu;
+                    tma_a = &tm->xe; tma_b = &tm->wgu;
                     arow = ti.row0;
                     brow = ti.e * 2 * p.I + ti.n * kTN0 + (int)rank * p.I;
                 } else if (ti.type == 1) {   // 256 output columns: leader the first 128 weight rows, peer the rest
-                    tma_a = tm_h; tma_b = tm_wd;
+                    tma_a = &tm->h; tma_b = &tm->wd;
                     arow = ti.row0;
                     brow = ti.e * p.H + ti.n * 256 + (int)rank * 128;
                 } else if (ti.type == 3) {   // M axis: 64 gate rows then 64 up rows of this CTA's 64 h-columns
-                    tma_a = tm_wgu64; tma_b = tm_xe;
+                    tma_a = &tm->wgu64; tma_b = &tm->xe;
                     arow = ti.e * 2 * p.I + ti.n * kTN0 + (int)rank * 64;
                     arow2 = arow + p.I;
                     brow = ti.row0 + (int)rank * nhalf;
                 } else {                     // M axis: this CTA's 128 of the n-tile's 256 out-columns
-                    tma_a = tm_wd; tma_b = tm_h;
+                    tma_a = &tm->wd; tma_b = &tm->h;
                     arow = ti.e * p.H + ti.n * 256 + (int)rank * 128;
                     brow = ti.row0 + (int)rank * nhalf;
                 }
                 for (int kb = 0; kb < ti.nkb; ++kb) {
-                    if (!mbar_wait(&S.empty[ps.stage], ps.stage_phase ^ 1u, p, 33)) { dead = true; break; }
+                    if (!mbar_wait(&S.empty[ps.stage], ps.stage_phase ^ 1u, p, 33)) { dead_l = true; break; }
                     uint8_t *sa = stages + ps.stage * kStageBytes;
                     const uint32_t lbar = mapa_u32(smem_u32(&S.full[ps.stage]), 0u);
                     if (rank == 0) mbar_arrive_expect_tx(&S.full[ps.stage], 2u * kStageBytes);
@@ -991,42 +1024,53 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                     ps.next_stage();
                 }
             }
-            if (dead) linger_after_abort();
+            dead = __any_sync(0xffffffffu, dead_l);
         }
+        if (dead && lane == 0) linger_after_abort();
         __syncwarp();
     } else if (warp == 1 && rank == 0) {
-        // ---------------- MMA issuer (leader only): one thread drives both SMs' tensor cores
-        if (lane == 0) {
-            bool dead = false;
-            while (!dead) {
-                if (!mbar_wait(&S.ti_full[ps.slot], ps.slot_phase, p, 40)) { dead = true; break; }
-                const TileInfo ti = S.ti[ps.slot];
-                mbar_arrive(&S.ti_empty[ps.slot]);
-                ps.next_slot();
-                if (ti.type == 2) break;
-                // regular tiles: 256 rows x 256 columns; swapped tiles: 256 weight rows x (rows rounded up to 16)
-                const uint32_t idesc = umma_idesc_bf16(2 * kBM, ti.type >= 3 ? (uint32_t)(((ti.nrows + 15) >> 4) << 4) : 256u);
-                if (!mbar_wait_cluster(&S.tmem_empty[ps.acc], ps.acc_phase ^ 1u, p, 41)) { dead = true; break; }
-                tc_fence_after();
-                const uint32_t d = tmem_base + (uint32_t)ps.acc * 256u;
-                for (int kb = 0; kb < ti.nkb; ++kb) {
-                    if (!mbar_wait_cluster(&S.full[ps.stage], ps.stage_phase, p, 42)) { dead = true; break; }
-                    tc_fence_after();
-                    const uint32_t a0 = smem_u32(stages + ps.stage * kStageBytes);
-                    const uint32_t b0 = a0 + kStageA;
-#pragma unroll
-                    for (int kk = 0; kk < kBK / 16; ++kk)
-                        tc_mma_bf16_pair(d, umma_desc_sw128(a0 + kk * 32), umma_desc_sw128(b0 + kk * 32), idesc,
-                                         (uint32_t)((kb | kk) != 0));
-                    tc_commit_pair(&S.empty[ps.stage], 3);      // both CTAs' stage is free once read
-                    ps.next_stage();
-                }
-                if (dead) break;
-                tc_commit_pair(&S.tmem_full[ps.acc], 3);        // accumulators complete in both CTAs
-                ps.next_acc();
+        // ---------------- MMA issuer (leader only): one elected thread drives both SMs' tensor cores.
+        // The whole warp walks the loop so that control flow and operands stay warp-uniform; lane 0
+        // does the waiting, the elected lane the issuing.
+        bool dead = false;
+        const uint64_t desc0 = umma_desc_sw128(smem_u32(stages));      // stage 0, A operand, first 16 of K
+        while (!dead) {
+            bool ok = true;
+            if (lane == 0) ok = mbar_wait(&S.ti_full[ps.slot], ps.slot_phase, p, 40);
+            if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
+            const TileInfo ti = S.ti[ps.slot];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&S.ti_empty[ps.slot]);
+            ps.next_slot();
+            if (ti.type == 2) break;
+            // regular tiles: 256 rows x 256 columns; swapped tiles: 256 weight rows x (rows rounded up to 16)
+            const uint32_t idesc = umma_idesc_bf16(2 * kBM, ti.type >= 3 ? (uint32_t)(((ti.nrows + 15) >> 4) << 4) : 256u);
+            // timeline record of this tile: extra = time spent waiting for a free accumulator (ns)
+            const unsigned long long tm0 = trace_now(p);
+            if (lane == 0) ok = mbar_wait_cluster(&S.tmem_empty[ps.acc], ps.acc_phase ^ 1u, p, 41);
+            if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
+            tc_fence_after();
+            const unsigned long long tm1 = trace_now(p);
+            const uint32_t d = tmem_base + (uint32_t)ps.acc * 256u;
+            for (int kb = 0; kb < ti.nkb; ++kb) {
+                // The operands were written by TMA (either CTA's, into its own shared memory) and are
+                // read by the tensor cores only: the barrier's completion is all the ordering needed.
+                // A wait that gives up has raised the abort flag: the following ones return at once,
+                // and the tile's (meaningless) MMAs only touch memory this pair owns.
+                if (lane == 0) ok = mbar_wait(&S.full[ps.stage], ps.stage_phase, p, 42) && ok;
+                __syncwarp();
+                const uint64_t da = desc0 + (uint64_t)(ps.stage * (kStageBytes >> 4));
+                tc_mma_kstep_pair(d, da, da + (uint64_t)(kStageA >> 4), idesc, (uint32_t)(kb != 0), &S.empty[ps.stage], 3);
+                ps.next_stage();
             }
-            if (dead) linger_after_abort();
+            if (elect_one()) tc_commit_pair(&S.tmem_full[ps.acc], 3);        // accumulators complete in both CTAs
+            if (lane == 0)
+                trace_ev(p, S, kEvMma, (unsigned)(ti.type << 16 | min(ti.nrows, 65535)), tm0, trace_now(p),
+                         (unsigned)min(0xFFFFFFFFull, tm1 - tm0));
+            ps.next_acc();
+            if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
         }
+        if (dead && lane == 0) linger_after_abort();
         __syncwarp();
     } else if (warp >= 4) {
         // ---------------- epilogue (both CTAs): TMEM -> registers -> (SwiGLU) -> bf16 -> staged store
@@ -1210,9 +1254,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
 constexpr int kErrNoPairs = -2;     // reported as "unsupported device"
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUtensorMap tm_xe,
-                 const __grid_constant__ CUtensorMap tm_wgu, const __grid_constant__ CUtensorMap tm_h,
-                 const __grid_constant__ CUtensorMap tm_wd, const __grid_constant__ CUtensorMap tm_wgu64)
+weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaMaps tm)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *stages = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -1242,7 +1284,8 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
         }
         mbar_init(&S.xg_full, 2); mbar_init(&S.xg_empty, 2);
         fence_mbar_init();
-        tma_prefetch_desc(&tm_xe); tma_prefetch_desc(&tm_wgu); tma_prefetch_desc(&tm_h); tma_prefetch_desc(&tm_wd); tma_prefetch_desc(&tm_wgu64);
+        tma_prefetch_desc(&tm.xe); tma_prefetch_desc(&tm.wgu); tma_prefetch_desc(&tm.h); tma_prefetch_desc(&tm.wd);
+        tma_prefetch_desc(&tm.wgu64);
     }
     if (warp == 1) { tmem_alloc_pair(&S.tmem_base, kTmemCols); tmem_relinquish_pair(); }
     tc_fence_before();
@@ -1498,7 +1541,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
         if (p.mode == kModeSerial) {
             dispatch_phase(p, S, stages, 0x7fffffff);
             alive = grid_barrier(p, S, 2u * n_sm, 2);
-            if (alive) gemm_phase(p, S, stages, tmem_base, &tm_xe, &tm_wgu, &tm_h, &tm_wd, &tm_wgu64, 0x7fffffff, ps);
+            if (alive) gemm_phase(p, S, stages, tmem_base, &tm, 0x7fffffff, ps);
             alive = alive && grid_barrier(p, S, 3u * n_sm, 3);
             if (alive) combine_phase(p, S, stages);
         } else {
@@ -1510,7 +1553,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ CUte
             const int dmax = mover ? 0x7fffffff : (p.elastic_steal ? 1 : 0);
             if (dmax > 0) dispatch_phase(p, S, stages, dmax);
             const int budget = mover ? plan_steal : 0x7fffffff;
-            if (budget > 0 || p.elastic_steal) gemm_phase(p, S, stages, tmem_base, &tm_xe, &tm_wgu, &tm_h, &tm_wd, &tm_wgu64, budget, ps);
+            if (budget > 0 || p.elastic_steal) gemm_phase(p, S, stages, tmem_base, &tm, budget, ps);
             combine_phase(p, S, stages);
         }
     }

@@ -112,7 +112,7 @@ struct weave_moe {
     unsigned long long pipe_calls;
     cudaStream_t pipe_h2d, pipe_d2h;
     cudaEvent_t pipe_in_ready[2], pipe_k_done[2], pipe_out_done[2];
-    CUtensorMap tm_xe, tm_wgu, tm_h, tm_wd, tm_wgu64;
+    TmaMaps tm;
 };
 
 namespace {
@@ -136,6 +136,18 @@ int encode_map(EncodeTiledFn fn, CUtensorMap *m, const void *base, uint64_t rows
                     weights ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? 0 : (int)r;
+}
+
+int encode_maps(EncodeTiledFn fn, TmaMaps *m, const void *xe, const void *hbuf, const void *gate_up, const void *down,
+                uint64_t p_max, uint64_t EE, uint64_t hidden, uint64_t ffn)
+{
+    int r = 0;
+    r |= encode_map(fn, &m->xe, xe, p_max, hidden, false);
+    r |= encode_map(fn, &m->wgu, gate_up, EE * 2 * ffn, hidden, true);
+    r |= encode_map(fn, &m->h, hbuf, p_max, ffn, false);
+    r |= encode_map(fn, &m->wd, down, EE * hidden, ffn, true);
+    r |= encode_map(fn, &m->wgu64, gate_up, EE * 2 * ffn, hidden, true, 64);
+    return r;
 }
 
 void default_tables(int n_sm, std::vector<float> &bw, std::vector<float> &tf)
@@ -248,11 +260,8 @@ int weave_moe_create(const weave_moe_config *cfg, weave_moe_t *out)
     EncodeTiledFn enc = reinterpret_cast<EncodeTiledFn>(fnp);
     const int EE = cfg->num_experts + cfg->num_shared;
     int r = 0;
-    r |= encode_map(enc, &h->tm_xe, h->ws + L.xe, (uint64_t)L.p_max, (uint64_t)cfg->hidden, false);
-    r |= encode_map(enc, &h->tm_wgu, cfg->gate_up, (uint64_t)EE * 2 * cfg->ffn, (uint64_t)cfg->hidden, true);
-    r |= encode_map(enc, &h->tm_h, h->ws + L.hbuf, (uint64_t)L.p_max, (uint64_t)cfg->ffn, false);
-    r |= encode_map(enc, &h->tm_wd, cfg->down, (uint64_t)EE * cfg->hidden, (uint64_t)cfg->ffn, true);
-    r |= encode_map(enc, &h->tm_wgu64, cfg->gate_up, (uint64_t)EE * 2 * cfg->ffn, (uint64_t)cfg->hidden, true, 64);
+    r = encode_maps(enc, &h->tm, h->ws + L.xe, h->ws + L.hbuf, cfg->gate_up, cfg->down, (uint64_t)L.p_max, (uint64_t)EE,
+                    (uint64_t)cfg->hidden, (uint64_t)cfg->ffn);
     if (r) { h->last_cuda_error = r; delete h; return WEAVE_ERR_CUDA; }
 
     e = cudaMemset(h->ws, 0, L.zero_end);
@@ -320,7 +329,7 @@ int weave_moe_forward(weave_moe_t h, const void *x, const float *logits, void *o
     p.trace = reinterpret_cast<uint4 *>(h->trace);
     p.trace_cap = h->trace_cap;
 
-    void *args[] = {&p, &h->tm_xe, &h->tm_wgu, &h->tm_h, &h->tm_wd, &h->tm_wgu64};
+    void *args[] = {&p, &h->tm};
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // one CTA per SM; the kernel is compiled with a cluster shape of two neighbouring CTAs (the GEMM
     // phase's CTA pairs); cooperative, so that all CTAs are co-resident for the in-kernel grid
@@ -693,11 +702,8 @@ int weave_moe_forward_static(int hidden, int ffn, int num_experts, int top_k, in
     h.ep_size = 1;
     const int EE = num_experts + num_shared;
     int r = 0;
-    r |= encode_map(sd->encode, &h.tm_xe, h.ws + L.xe, (uint64_t)L.p_max, (uint64_t)hidden, false);
-    r |= encode_map(sd->encode, &h.tm_wgu, gate_up, (uint64_t)EE * 2 * ffn, (uint64_t)hidden, true);
-    r |= encode_map(sd->encode, &h.tm_h, h.ws + L.hbuf, (uint64_t)L.p_max, (uint64_t)ffn, false);
-    r |= encode_map(sd->encode, &h.tm_wd, down, (uint64_t)EE * hidden, (uint64_t)ffn, true);
-    r |= encode_map(sd->encode, &h.tm_wgu64, gate_up, (uint64_t)EE * 2 * ffn, (uint64_t)hidden, true, 64);
+    r = encode_maps(sd->encode, &h.tm, h.ws + L.xe, h.ws + L.hbuf, gate_up, down, (uint64_t)L.p_max, (uint64_t)EE,
+                    (uint64_t)hidden, (uint64_t)ffn);
     if (r) return WEAVE_ERR_CUDA;
 
     // the array keeps whatever the last call left behind: zero the control words, refill the tables

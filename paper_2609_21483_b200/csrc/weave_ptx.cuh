@@ -372,6 +372,43 @@ __device__ __forceinline__ void tc_commit_pair(uint64_t *bar, uint16_t mask)
         : "memory");
 }
 
+// One thread of the (converged) warp: the same one every time for a given set of lanes, so what it
+// issues is tracked by the commits it issues later.
+__device__ __forceinline__ uint32_t elect_one()
+{
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred;
+}
+
+// One k-step of a pair tile, called by the whole (converged) warp: the elected thread issues the four
+// K=16 MMAs over a 64-wide stage (descriptors advance by 32 bytes = 2 address units) and then the
+// commit that frees the stage in both CTAs.  Keeping everything else warp-uniform lets the
+// operands live in uniform registers instead of being moved there before every instruction.
+__device__ __forceinline__ void tc_mma_kstep_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                  uint32_t accumulate_first, uint64_t *empty_bar, uint16_t mask)
+{
+    asm volatile(
+        "{\n\t.reg .pred pe, pa, pt;\n\t"
+        ".reg .b64 a1, a2, a3, b1, b2, b3;\n\t"
+        "elect.sync _|pe, 0xffffffff;\n\t"
+        "setp.ne.b32 pa, %4, 0;\n\t"
+        "setp.eq.u32 pt, %0, %0;\n\t"
+        "add.u64 a1, %1, 2;\n\tadd.u64 a2, %1, 4;\n\tadd.u64 a3, %1, 6;\n\t"
+        "add.u64 b1, %2, 2;\n\tadd.u64 b2, %2, 4;\n\tadd.u64 b3, %2, 6;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, pa;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16 [%0], a1, b1, %3, pt;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16 [%0], a2, b2, %3, pt;\n\t"
+        "@pe tcgen05.mma.cta_group::2.kind::f16 [%0], a3, b3, %3, pt;\n\t"
+        "@pe tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%5], %6;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate_first), "r"(smem_u32(empty_bar)), "h"(mask)
+        : "memory");
+}
+
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint4 v)
 {
     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
