@@ -60,7 +60,7 @@ def timeline(moe, x, lg, H, I):
     d = ev[ev[:, 3] == 4]
     e6 = ev[ev[:, 3] == 6]
     typ = e6[:, 5] >> 16
-    flops = 2.0 * 128 * 256 * np.where(typ == 0, H, I)
+    flops = 2.0 * 128 * 256 * np.where((typ == 0) | (typ == 3), H, I)      # gemm0 (regular, swapped) : gemm1
     out = {"end": us(ev[:, 2].max()), "gemm_first": us(e6[:, 1].min()), "gemm_last": us(e6[:, 2].max()),
            "gemm_ends": us(e6[:, 2]), "gemm_flops": flops}
     if len(d):

@@ -74,3 +74,20 @@ def test_calibration_produces_usable_tables_and_auto_follows_them():
     p = moe.plan()
     assert 2 <= p["c"] <= n // 2 and p["c"] % 2 == 0 and p["K"] in (1, 2, 4, 8) and p["t_total_us"] > 0
     moe.close()
+
+
+@pytest.mark.gpu
+def test_utilisation_report_from_the_kernel_timeline():
+    """AUTO overlaps movement with tensor-core work; with barriers between the phases nothing overlaps."""
+    from paper_2609_21483_b200 import timeline
+    cfg = wl.CONFIGS["c3_qwen3_30b"].with_T(4096)
+    auto, trace = timeline.run(cfg, "auto")
+    serial, _ = timeline.run(cfg, "serial")
+    for rep in (auto, serial):
+        assert 0.0 < rep["sm_busy"] <= 1.0 and 0.0 < rep["tensor_active"] <= 1.0
+        assert rep["overlap_ratio"] <= min(rep["movement_active"], rep["tensor_active"]) + 1e-9
+        assert rep["gemm_TFLOPs"] > 0 and rep["dispatch_GBps"] > 0 and rep["combine_GBps"] > 0
+    assert auto["overlap_ratio"] > 0.05
+    assert serial["overlap_ratio"] < 0.01
+    txt = timeline.ascii_timeline(trace, width=60).splitlines()
+    assert len(txt) == auto["n_cta"] + 1 and any("G" in l for l in txt[1:])
