@@ -272,18 +272,12 @@ __device__ __forceinline__ int block_excl_scan(int v, SmemTail &S, int &total)
 
 // ------------------------------------------------------------------------------------ phase R
 
-// One warp routes one token: the k largest logits (ties to the lowest expert index) in descending
-// order, gates = softmax over those k.  Lane l holds the logits of experts l, l+32, ... (NS of them).
-template <int NS>
-__device__ __forceinline__ void load_logits(const KParams &p, int t, float (&v)[NS])
-{
-    const int lane = threadIdx.x & 31;
-#pragma unroll
-    for (int m = 0; m < NS; ++m) {
-        const int e = lane + 32 * m;
-        v[m] = e < p.E ? __ldg(p.logits + (size_t)t * p.E + e) : __int_as_float(0xff800000);
-    }
-}
+// Four threads route one token, so a CTA's 256 threads take a whole 64-token block at once and no
+// lane idles.  The block's logits are staged in shared memory (row stride = 4 mod 32 words, so the
+// 32 lanes of a warp - eight tokens x four threads - hit 32 different banks).  Thread q of a quad
+// scans experts q, q+4, ... in ascending order and keeps its KC >= k best in a sorted register list;
+// the four lists are then merged k times through two shuffle steps.  Order: larger logit first,
+// equal logits by lower expert index (-0 == +0); gates = softmax over the selected k.
 
 // fp32 -> uint32 that orders like the float (finite values; -0 has been folded into +0)
 __device__ __forceinline__ unsigned float_order_key(float v)
@@ -296,114 +290,120 @@ __device__ __forceinline__ float float_from_order_key(unsigned k)
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
 }
 
-// Two tokens per warp at a time: the two selections are independent instruction streams, so the
-// warp-reduction latencies of one hide behind the other.  `nt` (1 or 2) tokens are valid.
-template <int NS>
-__device__ __forceinline__ void route_tokens2(const KParams &p, const int (&t)[2], const int (&tl)[2], int nt,
-                                              float (&v)[2][NS], unsigned long long *r_mask, int *r_idx, int *r_cnt)
-{
-    const int lane = threadIdx.x & 31;
-    const int e_lo = p.ep_size > 1 ? p.ep_rank * (p.E / p.ep_size) : 0;
-    const int e_hi = p.ep_size > 1 ? e_lo + p.E / p.ep_size : p.E;
-    // keys: 0 = absent / already taken; every finite logit maps to a key >= 1 that orders like
-    // the float, with -0.0 == +0.0 (the comparison rule of the routing definition)
-    unsigned key[2][NS];
-    bool bad = false;
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-#pragma unroll
-        for (int m = 0; m < NS; ++m) {
-            key[u][m] = 0u;
-            if (u < nt && lane + 32 * m < p.E) {
-                float x = v[u][m];
-                if (!(fabsf(x) <= 3.402823466e38f)) {   // NaN or +-inf: flag it, keep indices in range
-                    bad = true;
-                    x = -3.402823466e38f;
-                }
-                x = __fadd_rn(x, 0.0f);                  // folds -0 into +0, leaves everything else alone
-                key[u][m] = float_order_key(x);
-            }
-        }
-    }
-    if (__any_sync(0xffffffffu, bad) && lane == 0) atomicCAS(&p.ctl->status, 0, kErrNonFinite);
+__device__ __forceinline__ int route_row_stride(int E) { return ((E + 27) / 32) * 32 + 4; }
 
-    int my_e[2] = {0, 0};
-    unsigned my_key[2] = {0u, 0u};
-    for (int j = 0; j < p.k; ++j) {
-        unsigned bk[2], wk[2];
-        int be[2], we[2];
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            bk[u] = 0u;
-            be[u] = 0x7fffffff;
-#pragma unroll
-            for (int m = 0; m < NS; ++m)
-                if (key[u][m] > bk[u]) { bk[u] = key[u][m]; be[u] = lane + 32 * m; }   // strict '>' keeps the lower index
-        }
-#pragma unroll
-        for (int u = 0; u < 2; ++u) wk[u] = __reduce_max_sync(0xffffffffu, bk[u]);          // largest logit
-#pragma unroll
-        for (int u = 0; u < 2; ++u)                                                          // lowest index with it
-            we[u] = (int)__reduce_min_sync(0xffffffffu, bk[u] == wk[u] ? (unsigned)be[u] : 0x7fffffffu);
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            if ((we[u] & 31) == lane) {
-#pragma unroll
-                for (int m = 0; m < NS; ++m)
-                    if (m == (we[u] >> 5)) key[u][m] = 0u;                                   // taken
-            }
-            if (lane == j) { my_e[u] = we[u]; my_key[u] = wk[u]; }
-        }
+// cooperative copy of the block's logit rows into shared memory, a warp per row, coalesced; all copies
+// are in flight together (one memory round trip); the caller's __syncthreads() publishes them
+__device__ __forceinline__ void stage_logits(const KParams &p, int b, float *lg_s)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ntok = min(kRouteBlock, p.T - b * kRouteBlock);
+    const int stride = route_row_stride(p.E);
+    for (int r = warp; r < ntok; r += kThreads / 32) {
+        const float *src = p.logits + (size_t)(b * kRouteBlock + r) * p.E;
+        for (int c = lane; c < p.E; c += 32) cp_async_4(smem_u32(lg_s + r * stride + c), src + c);
     }
-#pragma unroll
-    for (int u = 0; u < 2; ++u) {
-        if (u < nt) {
-            const float my_v = float_from_order_key(my_key[u]);
-            const float vmax = __shfl_sync(0xffffffffu, my_v, 0);
-            const float pj = lane < p.k ? expf(my_v - vmax) : 0.f;
-            float sum = 0.f;
-            for (int j = 0; j < p.k; ++j) sum += __shfl_sync(0xffffffffu, pj, j);   // slot order
-            // expert-parallel share: only the experts hosted here get rows; the gates stay normalised
-            // over all k selected experts
-            const bool local = lane < p.k && my_e[u] >= e_lo && my_e[u] < e_hi;
-            if (lane < p.k) {
-                p.topk_idx[(size_t)t[u] * p.k + lane] = my_e[u];
-                p.gates[(size_t)t[u] * p.k + lane] = __fdiv_rn(pj, sum);
-                r_idx[tl[u] * kMaxTopK + lane] = local ? my_e[u] : -1;
-                if (local) atomicOr(&r_mask[my_e[u]], 1ull << tl[u]);
-            }
-            if (p.ep_size > 1) {
-                const int nloc = __popc(__ballot_sync(0xffffffffu, local));
-                if (lane == 0 && nloc) {
-                    if (t[u] / p.ep_tshard == p.ep_rank) atomicAdd(&r_cnt[0], nloc);
-                    else { atomicAdd(&r_cnt[1], nloc); atomicOr(&r_mask[kMaxEE], 1ull << tl[u]); }
-                }
-            }
-        }
-    }
+    cp_async_wait_all();
 }
 
-// the tokens of one 64-token block that belong to this warp (tl = warp, warp + 8, ...), two at a time
-template <int NS>
-__device__ __forceinline__ void route_block_tokens(const KParams &p, int b, unsigned long long *r_mask, int *r_idx,
-                                                   int *r_cnt)
+template <int KC>
+__device__ __forceinline__ void route_block_quads(const KParams &p, int b, const float *lg_s, unsigned long long *r_mask,
+                                                  int *r_idx, int *r_cnt)
 {
-    const int warp = threadIdx.x >> 5;
-    constexpr int kStep = kThreads / 32;
-    for (int tl0 = warp; tl0 < kRouteBlock; tl0 += 2 * kStep) {
-        int t[2], tl[2];
-        tl[0] = tl0; tl[1] = tl0 + kStep;
-        t[0] = b * kRouteBlock + tl[0]; t[1] = b * kRouteBlock + tl[1];
-        if (t[0] >= p.T) break;
-        const int nt = (tl[1] < kRouteBlock && t[1] < p.T) ? 2 : 1;
-        float v[2][NS];
-        load_logits<NS>(p, t[0], v[0]);
-        if (nt == 2) load_logits<NS>(p, t[1], v[1]);
-        else {
+    static_assert(kThreads == 4 * kRouteBlock, "four threads per token of a routing block");
+    const int tl = threadIdx.x >> 2, q = threadIdx.x & 3;
+    const int t = b * kRouteBlock + tl;
+    const bool valid = t < p.T;
+    const int stride = route_row_stride(p.E);
+    const int e_lo = p.ep_size > 1 ? p.ep_rank * (p.E / p.ep_size) : 0;
+    const int e_hi = p.ep_size > 1 ? e_lo + p.E / p.ep_size : p.E;
+
+    // keys: 0 = empty slot; every finite logit maps to a key >= 1 that orders like the float
+    unsigned key[KC];
+    int idx[KC];
 #pragma unroll
-            for (int m = 0; m < NS; ++m) v[1][m] = 0.f;
+    for (int j = 0; j < KC; ++j) { key[j] = 0u; idx[j] = 0x7fffffff; }
+    bool bad = false;
+    if (valid) {
+        for (int e = q; e < p.E; e += 4) {
+            float x = lg_s[tl * stride + e];
+            if (!(fabsf(x) <= 3.402823466e38f)) {   // NaN or +-inf: flag it, keep indices in range
+                bad = true;
+                x = -3.402823466e38f;
+            }
+            x = __fadd_rn(x, 0.0f);                  // folds -0 into +0, leaves everything else alone
+            const unsigned c = float_order_key(x);
+            if (c > key[KC - 1]) {
+                // insert behind every entry that is >= c (they have lower indices): from the bottom,
+                // an entry smaller than c moves down one slot, and c lands above the first such entry
+#pragma unroll
+                for (int j = KC - 1; j >= 1; --j) {
+                    if (c > key[j - 1]) { key[j] = key[j - 1]; idx[j] = idx[j - 1]; }
+                    else if (c > key[j]) { key[j] = c; idx[j] = e; }
+                }
+                if (c > key[0]) { key[0] = c; idx[0] = e; }
+            }
         }
-        route_tokens2<NS>(p, t, tl, nt, v, r_mask, r_idx, r_cnt);
+    }
+    if (__any_sync(0xffffffffu, bad) && (threadIdx.x & 31) == 0) atomicCAS(&p.ctl->status, 0, kErrNonFinite);
+
+    // merge: slot j = the best head of the quad's four lists; its owner pops it
+    unsigned sel_key[KC];
+    int sel_idx[KC];
+#pragma unroll
+    for (int j = 0; j < KC; ++j) {
+        sel_key[j] = 0u; sel_idx[j] = 0;
+        if (j < p.k) {
+            unsigned hk = key[0];
+            int hi = idx[0];
+#pragma unroll
+            for (int o = 1; o <= 2; o <<= 1) {
+                const unsigned ok = __shfl_xor_sync(0xffffffffu, hk, o);
+                const int oi = __shfl_xor_sync(0xffffffffu, hi, o);
+                if (ok > hk || (ok == hk && oi < hi)) { hk = ok; hi = oi; }
+            }
+            sel_key[j] = hk; sel_idx[j] = hi;
+            if (hi == idx[0]) {
+#pragma unroll
+                for (int i = 0; i + 1 < KC; ++i) { key[i] = key[i + 1]; idx[i] = idx[i + 1]; }
+                key[KC - 1] = 0u; idx[KC - 1] = 0x7fffffff;
+            }
+        }
+    }
+
+    if (valid) {
+        // every thread of the quad holds all k selections; thread q writes slots q, q+4, ...
+        const float vmax = float_from_order_key(sel_key[0]);
+        float pj[KC];
+        float sum = 0.f;
+#pragma unroll
+        for (int j = 0; j < KC; ++j) {
+            pj[j] = 0.f;
+            if (j < p.k) { pj[j] = expf(float_from_order_key(sel_key[j]) - vmax); sum += pj[j]; }   // slot order
+        }
+        int nloc = 0;
+#pragma unroll
+        for (int j = 0; j < KC; ++j) {
+            if (j < p.k) {
+                // expert-parallel share: only the experts hosted here get rows; the gates stay
+                // normalised over all k selected experts
+                const bool local = sel_idx[j] >= e_lo && sel_idx[j] < e_hi;
+                nloc += local ? 1 : 0;
+                if ((j & 3) == q) {
+                    p.topk_idx[(size_t)t * p.k + j] = sel_idx[j];
+                    p.gates[(size_t)t * p.k + j] = __fdiv_rn(pj[j], sum);
+                    r_idx[tl * kMaxTopK + j] = local ? sel_idx[j] : -1;
+                    if (local) atomicOr(reinterpret_cast<unsigned *>(&r_mask[sel_idx[j]]) + (tl >> 5), 1u << (tl & 31));
+                }
+            }
+        }
+        if (p.ep_size > 1 && q == 0 && nloc) {
+            if (t / p.ep_tshard == p.ep_rank) atomicAdd(&r_cnt[0], nloc);
+            else {
+                atomicAdd(&r_cnt[1], nloc);
+                atomicOr(reinterpret_cast<unsigned *>(&r_mask[kMaxEE]) + (tl >> 5), 1u << (tl & 31));
+            }
+        }
     }
 }
 
@@ -1301,16 +1301,19 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
     int *r_idx = reinterpret_cast<int *>(stages + 2048 + 64);                              // [64][16]
     int *r_base = reinterpret_cast<int *>(stages + 2048 + 64 + kRouteBlock * kMaxTopK * 4);    // [256]
     int *r_cnt = r_base + kMaxEE;                                                          // [2] local / remote pairs
+    float *lg_s = reinterpret_cast<float *>(stages + 8192);                                // [64][route_row_stride(E)]
 
     // ================= phase R: routing
     for (int b = blockIdx.x; b < p.nblk; b += n_sm) {
         for (int e = tid; e < EE; e += kThreads) r_mask[e] = 0ull;
         if (tid == 0) { r_mask[kMaxEE] = 0ull; r_cnt[0] = 0; r_cnt[1] = 0; }
         __syncthreads();
-        if (p.E <= 32) route_block_tokens<1>(p, b, r_mask, r_idx, r_cnt);
-        else if (p.E <= 64) route_block_tokens<2>(p, b, r_mask, r_idx, r_cnt);
-        else if (p.E <= 128) route_block_tokens<4>(p, b, r_mask, r_idx, r_cnt);
-        else route_block_tokens<8>(p, b, r_mask, r_idx, r_cnt);
+        stage_logits(p, b, lg_s);
+        __syncthreads();
+        if (p.k <= 2) route_block_quads<2>(p, b, lg_s, r_mask, r_idx, r_cnt);
+        else if (p.k <= 4) route_block_quads<4>(p, b, lg_s, r_mask, r_idx, r_cnt);
+        else if (p.k <= 8) route_block_quads<8>(p, b, lg_s, r_mask, r_idx, r_cnt);
+        else route_block_quads<16>(p, b, lg_s, r_mask, r_idx, r_cnt);
         __syncthreads();
         // in-block rank of each (token, slot): tokens before it in the block that chose the same expert
         for (int pi = tid; pi < kRouteBlock * p.k; pi += kThreads) {

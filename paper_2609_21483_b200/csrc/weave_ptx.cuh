@@ -439,6 +439,13 @@ __device__ __forceinline__ void bulk_store(void *gdst, uint32_t smem_src, uint32
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_src), "r"(bytes)
                  : "memory");
 }
+// 4-byte asynchronous copy global -> shared (no register staging, any number in flight)
+__device__ __forceinline__ void cp_async_4(uint32_t smem_dst, const void *gsrc)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_dst), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // wait until at most N of this thread's bulk groups are still incomplete (writes performed)
 template <int N>
