@@ -195,6 +195,19 @@ int weave_moe_debug_withhold_flag(weave_moe_t h, int m_block);
  * 9 grid barrier. */
 int weave_moe_set_trace(weave_moe_t h, void *buf, int events_per_cta);
 
+/* HOST-ONLY (no GPU needed, no handle): the order in which the kernel's GEMM schedulers claim pair
+ * tiles (Section 4: tile queues "in chunk-pipeline DAG order"), for `num_chunks` chunks of
+ * `num_segments` expert segments whose row counts are rows[chunk * num_segments + expert], n-tile
+ * counts nt0 (gemm0) and nt1 (gemm1).  Writes up to max_tiles records of
+ * 6 ints {type (0 gemm0, 1 gemm1, +3 when the operands are swapped), leader m-block, peer m-block
+ * (-1 for a swapped tile), n-tile, chunk, rows of the leader m-block} to `out` (host memory, may be
+ * NULL) and returns the total number of tiles, or a negative error for bad arguments (chunks not
+ * in {1,2,4,8}, more than 1024 segments in total, non-positive tile counts).  This is the same
+ * decoding routine the device runs; tests use it to check that every tile a gemm1 tile waits for
+ * comes earlier in the queue. */
+int weave_moe_debug_gemm_queue(const int32_t *rows, int num_segments, int num_chunks, int nt0, int nt1,
+                               int32_t *out, int max_tiles);
+
 /* ---- for callers that cannot allocate ---------------------------------------------------------
  *
  * (No counterpart in the paper: this is a packaging variant of the same kernel.)

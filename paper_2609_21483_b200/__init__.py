@@ -17,6 +17,7 @@ LIB_PATH = os.path.join(_HERE, "libweave_moe.so")
 _SOURCES = ["weave_moe.cu", "weave_kernel.cuh", "weave_ptx.cuh"]
 
 WEAVE_OK = 0
+WEAVE_ERR_INVALID_ARG = -1
 SCHED_AUTO, SCHED_FIXED, SCHED_SERIAL = 0, 1, 2
 ERR_NONFINITE_LOGITS, ERR_TIMEOUT = -5, -6
 
@@ -61,7 +62,7 @@ EXPORTS = [
     "weave_moe_last_cuda_error", "weave_moe_strerror", "weave_moe_set_trace",
     "weave_moe_forward_static", "weave_moe_static_scratch_bytes", "weave_moe_set_sm_count",
     "weave_moe_set_expert_parallel", "weave_moe_get_ep_descriptors",
-    "weave_moe_forward_host_pipelined", "weave_moe_host_wait",
+    "weave_moe_forward_host_pipelined", "weave_moe_host_wait", "weave_moe_debug_gemm_queue",
 ]
 
 
@@ -122,6 +123,8 @@ def load():
     lib.weave_moe_static_scratch_bytes.argtypes = []
     lib.weave_moe_last_cuda_error.restype = ci
     lib.weave_moe_last_cuda_error.argtypes = [vp]
+    lib.weave_moe_debug_gemm_queue.restype = ci
+    lib.weave_moe_debug_gemm_queue.argtypes = [vp, ci, ci, ci, ci, vp, ci]
     lib.weave_moe_strerror.restype = ctypes.c_char_p
     lib.weave_moe_strerror.argtypes = [ci]
     _lib = lib
@@ -130,6 +133,24 @@ def load():
 
 def strerror(code: int) -> str:
     return load().weave_moe_strerror(code).decode()
+
+
+def gemm_queue(rows, nt0: int, nt1: int):
+    """Host-only: the GEMM tile queue for rows[chunk][expert] -> int32 array [n_tiles, 6] of
+    (type, leader m-block, peer m-block or -1, n-tile, chunk, leader rows); no GPU involved."""
+    import numpy as np
+    rows = np.ascontiguousarray(rows, dtype=np.int32)
+    if rows.ndim == 1:
+        rows = rows[None, :]
+    K, EE = rows.shape
+    n = load().weave_moe_debug_gemm_queue(rows.ctypes.data, EE, K, nt0, nt1, None, 0)
+    if n < 0:
+        raise WeaveError(n, "weave_moe_debug_gemm_queue")
+    out = np.zeros((n, 6), np.int32)
+    if n:
+        _check(0 if load().weave_moe_debug_gemm_queue(rows.ctypes.data, EE, K, nt0, nt1, out.ctypes.data, n) == n
+               else WEAVE_ERR_INVALID_ARG, "weave_moe_debug_gemm_queue")
+    return out
 
 
 def workspace_bytes(hidden, ffn, num_experts, top_k, num_shared, max_tokens) -> int:

@@ -462,38 +462,44 @@ __device__ __forceinline__ void decode_mblock(const SmemTail &S, int EE, int mb,
 
 // number of regular (two-m-block) pair tiles / of unpaired m-blocks in the chunk's segments before s:
 // a segment with pts pair tiles has 2*pts - u m-blocks, u = 1 if its last m-block is unpaired
-__device__ __forceinline__ int seg_reg0(const SmemTail &S, int s, int cmb0, int cpt0)
+__host__ __device__ __forceinline__ int seg_reg0(const SmemTail &S, int s, int cmb0, int cpt0)
 {
     return (S.seg_mb0[s] - cmb0) - (S.seg_pt0[s] - cpt0);
 }
-__device__ __forceinline__ int seg_swap0(const SmemTail &S, int s, int cmb0, int cpt0)
+__host__ __device__ __forceinline__ int seg_swap0(const SmemTail &S, int s, int cmb0, int cpt0)
 {
     return 2 * (S.seg_pt0[s] - cpt0) - (S.seg_mb0[s] - cmb0);
 }
 
 // GEMM queue order (the chunk-pipeline DAG order): chunk by chunk; inside a chunk all gemm0 tiles,
-// then all gemm1 tiles.  Inside those, two streams are interleaved at a constant ratio:
-//  - the regular pair tiles (two consecutive m-blocks of one segment), expert-major, then groups of
-//    kPairGroup pair tiles, n-tile, pair tile fastest (consecutive tiles share a weight panel, and a
-//    group's rows stay in L2 while all its n-tiles pass); these are bound by the tensor pipe;
-//  - the unpaired last m-blocks of the segments (operands swapped), expert-major, n-tile fastest;
-//    each streams a weight panel that nobody else reads, so they are bound by HBM.
-// Spreading the second stream evenly over the first keeps both resources busy all the time; in
-// expert order a run of small experts would leave the tensor pipes waiting on HBM, and a large
-// expert would leave HBM idle.  `lead` describes the leader CTA's half, `peer` the other CTA's.
-__device__ __forceinline__ void decode_pair_tile(const SmemTail &S, const KParams &p, int g, TileInfo &lead,
-                                                 TileInfo &peer)
+// then all gemm1 tiles (every gemm0 tile a gemm1 tile waits for comes earlier in the queue and waits
+// only for dispatch, which keeps the in-order schedulers free of deadlock).  Each GEMM's tiles are
+// taken in UNITS of one pair tile's worth of n-tiles, of two kinds:
+//  - regular pair tiles (two consecutive m-blocks of one segment): expert-major, then in groups of
+//    kPairGroup pair tiles, n-tile, pair tile fastest (consecutive tiles share a weight panel, and
+//    a group's rows stay in L2 while all its n-tiles pass); bound by the tensor pipe;
+//  - the unpaired last m-blocks of the segments (operands swapped): expert-major, the n-tiles of
+//    one m-block back to back; each streams weight panels that nobody else reads.
+// The swapped units are spread evenly over the regular ones, so that neither HBM nor the tensor
+// pipes idle while a run of small experts (or one large expert) passes.
+// (Alternating gemm1 units with gemm0 units was measured and dropped: it hides the epilogues of the
+// short gemm1 main loops, +1 % at I = 512, but doubles the weight working set in L2, -9 % on the
+// 24-layer Qwen3-235B-shaped stack.)
+// `lead` describes the leader CTA's half of the pair tile, `peer` the other CTA's.  Host-callable so
+// that the order can be checked without a GPU.
+__host__ __device__ __forceinline__ void decode_pair_tile(const SmemTail &S, const KParams &p, int g, TileInfo &lead,
+                                                          TileInfo &peer)
 {
     int j = 0;
     while (j + 1 < S.K && g >= S.chunk_tile0[j + 1]) ++j;
     int local = g - S.chunk_tile0[j];
     const int cpt0 = S.chunk_pt0[j], cmb0 = S.chunk_mb0[j];
-    const int nptj = S.chunk_pt0[j + 1] - cpt0;
+    const int nptj = S.chunk_pt0[j + 1] - cpt0, nswj = S.chunk_nswap[j];
     int type = 0, nt = p.nt0;
     if (local >= nptj * p.nt0) { type = 1; local -= nptj * p.nt0; nt = p.nt1; }
-    const long long n_sw = (long long)S.chunk_nswap[j] * nt, total = (long long)nptj * nt;
-    const int sw_before = (int)((local * n_sw) / total);
-    const bool swapped = (int)(((local + 1) * n_sw) / total) > sw_before;
+    const int unit = local / nt, w = local - unit * nt;
+    const int sw_before = (int)(((long long)unit * nswj) / nptj);
+    const bool swapped = (int)(((long long)(unit + 1) * nswj) / nptj) > sw_before;
     lead.type = peer.type = type;
     lead.chunk = peer.chunk = j;
     lead.nkb = peer.nkb = (type == 0 ? p.H : p.I) / kBK;
@@ -503,20 +509,20 @@ __device__ __forceinline__ void decode_pair_tile(const SmemTail &S, const KParam
         // ceil(nrows/16)*16 columns instead of a half-empty 256-row tile
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
-            if (seg_swap0(S, mid, cmb0, cpt0) * nt <= sw_before) lo = mid; else hi = mid;
+            if (seg_swap0(S, mid, cmb0, cpt0) <= sw_before) lo = mid; else hi = mid;
         }
         const int s = lo;
         const int m0 = 2 * (S.seg_pt0[s + 1] - S.seg_pt0[s] - 1);
         lead.type = type + 3;
         lead.e = s - j * p.EE;
-        lead.n = sw_before - seg_swap0(S, s, cmb0, cpt0) * nt;
+        lead.n = w;
         lead.mb = S.seg_mb0[s] + m0;
         lead.row0 = S.seg_row0[s] + m0 * kBM;
         lead.nrows = S.seg_rows[s] - m0 * kBM;
         peer = lead;
         return;
     }
-    const int reg = local - sw_before;
+    const int reg = (unit - sw_before) * nt + w;
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
         if (seg_reg0(S, mid, cmb0, cpt0) * nt <= reg) lo = mid; else hi = mid;
@@ -526,7 +532,7 @@ __device__ __forceinline__ void decode_pair_tile(const SmemTail &S, const KParam
     const int within = reg - seg_reg0(S, s, cmb0, cpt0) * nt;
     const int gi = within / (kPairGroup * nt);
     const int wg = within - gi * kPairGroup * nt;
-    const int gsize = min(kPairGroup, pts - gi * kPairGroup);
+    const int gsize = (pts - gi * kPairGroup) < kPairGroup ? (pts - gi * kPairGroup) : kPairGroup;
     const int n = wg / gsize;
     const int m0 = 2 * (gi * kPairGroup + (wg - n * gsize));
     const int rows = S.seg_rows[s];
@@ -535,7 +541,7 @@ __device__ __forceinline__ void decode_pair_tile(const SmemTail &S, const KParam
     lead.mb = S.seg_mb0[s] + m0;
     lead.row0 = S.seg_row0[s] + m0 * kBM;
     lead.nrows = kBM;
-    peer.nrows = min(kBM, rows - (m0 + 1) * kBM);
+    peer.nrows = (rows - (m0 + 1) * kBM) < kBM ? (rows - (m0 + 1) * kBM) : kBM;
     peer.mb = lead.mb + 1;
     peer.row0 = lead.row0 + kBM;
 }

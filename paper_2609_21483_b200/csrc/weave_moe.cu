@@ -597,6 +597,45 @@ int weave_moe_set_trace(weave_moe_t h, void *buf, int events_per_cta)
 
 int weave_moe_last_cuda_error(weave_moe_t h) { return h ? h->last_cuda_error : 0; }
 
+int weave_moe_debug_gemm_queue(const int32_t *rows, int num_segments, int num_chunks, int nt0, int nt1, int32_t *out,
+                               int max_tiles)
+{
+    if (!rows || num_segments < 1 || nt0 < 1 || nt1 < 1) return WEAVE_ERR_INVALID_ARG;
+    if (num_chunks != 1 && num_chunks != 2 && num_chunks != 4 && num_chunks != 8) return WEAVE_ERR_INVALID_ARG;
+    if (num_segments * num_chunks > kMaxSeg) return WEAVE_ERR_INVALID_ARG;
+    // the tables the kernel's set-up builds in shared memory, built here the same way
+    std::vector<unsigned char> raw(sizeof(SmemTail), 0);
+    SmemTail &S = *reinterpret_cast<SmemTail *>(raw.data());
+    KParams p;
+    memset(&p, 0, sizeof(p));
+    p.EE = num_segments; p.nt0 = nt0; p.nt1 = nt1; p.H = kBK; p.I = kBK;
+    int mb = 0, pt = 0, row = 0;
+    for (int j = 0; j < num_chunks; ++j) {
+        S.chunk_mb0[j] = mb; S.chunk_pt0[j] = pt; S.chunk_tile0[j] = pt * (nt0 + nt1);
+        int nodd = 0;
+        for (int e = 0; e < num_segments; ++e) {
+            const int r = rows[j * num_segments + e];
+            if (r < 0) return WEAVE_ERR_INVALID_ARG;
+            const int mbs = (r + kBM - 1) / kBM;
+            S.seg_mb0[j * num_segments + e] = mb; S.seg_pt0[j * num_segments + e] = pt;
+            S.seg_row0[j * num_segments + e] = row; S.seg_rows[j * num_segments + e] = r;
+            mb += mbs; pt += (mbs + 1) / 2; row += r; nodd += mbs & 1;
+        }
+        S.chunk_nswap[j] = nodd;
+    }
+    S.seg_mb0[num_chunks * num_segments] = mb; S.seg_pt0[num_chunks * num_segments] = pt;
+    S.chunk_mb0[num_chunks] = mb; S.chunk_pt0[num_chunks] = pt; S.chunk_tile0[num_chunks] = pt * (nt0 + nt1);
+    S.K = num_chunks;
+    const int n = pt * (nt0 + nt1);
+    for (int g = 0; g < n && g < max_tiles && out; ++g) {
+        TileInfo tl, tp;
+        decode_pair_tile(S, p, g, tl, tp);
+        int32_t *o = out + (size_t)g * 6;
+        o[0] = tl.type; o[1] = tl.mb; o[2] = tl.type >= 3 ? -1 : tp.mb; o[3] = tl.n; o[4] = tl.chunk; o[5] = tl.nrows;
+    }
+    return n;
+}
+
 }  // extern "C"
 
 // ------------------------------------------------------------------------------------------------
