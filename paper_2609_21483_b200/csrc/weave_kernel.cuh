@@ -200,12 +200,16 @@ __device__ __forceinline__ unsigned long long trace_now(const KParams &p)
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, const KParams &p, int where)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = globaltimer_ns();
+    // the clock is read only every 32 polls (the first reading starts the limit): a reading costs far
+    // more than a poll, and most waits end within a few polls
+    unsigned long long t0 = 0;
     unsigned it = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++it & 31u) == 0u) {
             if (ld_relaxed_u32(&p.ctl->abort)) return false;
-            if (globaltimer_ns() - t0 > p.timeout_ns) {
+            const unsigned long long now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > p.timeout_ns) {
                 give_up(p.ctl, where);
                 return false;
             }
@@ -217,13 +221,15 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, const 
 __device__ __forceinline__ bool flag_wait_ge(const unsigned *flag, unsigned target, const KParams &p, int where)
 {
     if (ld_acquire_u32(flag) >= target) return true;
-    const unsigned long long t0 = globaltimer_ns();
+    unsigned long long t0 = 0;
     unsigned it = 0;
     while (ld_acquire_u32(flag) < target) {
         __nanosleep(40);
         if ((++it & 31u) == 0u) {
             if (ld_relaxed_u32(&p.ctl->abort)) return false;
-            if (globaltimer_ns() - t0 > p.timeout_ns) {
+            const unsigned long long now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > p.timeout_ns) {
                 give_up(p.ctl, where);
                 return false;
             }
@@ -863,8 +869,9 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uin
 // ------------------------------------------------------------------------------------ phase B: GEMM
 
 // Tensor maps of the GEMM operands: bf16 matrices, boxes of 64 columns (one 128-byte swizzle row) by
-// 128 rows (64 rows for the gate and up halves of a swapped tile's weight operand).
-struct TmaMaps { CUtensorMap xe, wgu, h, wd, wgu64; };
+// 128 rows (64 rows for the gate and up halves of a swapped tile's weight operand; 8, 16, 32 or 64
+// rows for a swapped tile's row operand, whichever covers its half of the m-block's rows).
+struct TmaMaps { CUtensorMap xe, wgu, h, wd, wgu64, xe_n[4], h_n[4]; };
 
 struct PipeState {     // per-role ring positions; they persist across the tiles of a phase
     int stage = 0;  uint32_t stage_phase = 0;
@@ -884,12 +891,14 @@ __device__ __forceinline__ float silu_mul(float g, float u)
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity, const KParams &p, int where)
 {
     if (mbar_try_wait_cluster(bar, parity)) return true;
-    const unsigned long long t0 = globaltimer_ns();
+    unsigned long long t0 = 0;
     unsigned it = 0;
     while (!mbar_try_wait_cluster(bar, parity)) {
         if ((++it & 31u) == 0u) {
             if (ld_relaxed_u32(&p.ctl->abort)) return false;
-            if (globaltimer_ns() - t0 > p.timeout_ns) {
+            const unsigned long long now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > p.timeout_ns) {
                 give_up(p.ctl, where);
                 return false;
             }
@@ -1001,6 +1010,10 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                 int arow, brow, arow2 = -1;
                 // swapped tiles: rows per CTA on the N axis (the MMA's N, a multiple of 16, split in two)
                 const int nhalf = (((ti.nrows + 15) >> 4) << 4) >> 1;
+                // ... fetched with the smallest box that covers them (the copy engine takes in a fixed
+                // number of rows per cycle, so rows nobody reads cost as much as the others)
+                const int bi = nhalf <= 8 ? 0 : nhalf <= 16 ? 1 : nhalf <= 32 ? 2 : 3;
+                uint32_t tx = 2u * kStageBytes;                  // bytes landing in both CTAs per k-step
                 if (ti.type == 0) {      // leader holds the gate rows of the n-tile, peer the up rows
                     tma_a = &tm->xe; tma_b = &tm->wgu;
                     arow = ti.row0;
@@ -1010,12 +1023,14 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                     arow = ti.row0;
                     brow = ti.e * p.H + ti.n * 256 + (int)rank * 128;
                 } else if (ti.type == 3) {   // M axis: 64 gate rows then 64 up rows of this CTA's 64 h-columns
-                    tma_a = &tm->wgu64; tma_b = &tm->xe;
+                    tma_a = &tm->wgu64; tma_b = &tm->xe_n[bi];
+                    tx = 2u * (kStageA + (1024u << bi));
                     arow = ti.e * 2 * p.I + ti.n * kTN0 + (int)rank * 64;
                     arow2 = arow + p.I;
                     brow = ti.row0 + (int)rank * nhalf;
                 } else {                     // M axis: this CTA's 128 of the n-tile's 256 out-columns
-                    tma_a = &tm->wd; tma_b = &tm->h;
+                    tma_a = &tm->wd; tma_b = &tm->h_n[bi];
+                    tx = 2u * (kStageA + (1024u << bi));
                     arow = ti.e * p.H + ti.n * 256 + (int)rank * 128;
                     brow = ti.row0 + (int)rank * nhalf;
                 }
@@ -1023,7 +1038,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                     if (!mbar_wait(&S.empty[ps.stage], ps.stage_phase ^ 1u, p, 33)) { dead_l = true; break; }
                     uint8_t *sa = stages + ps.stage * kStageBytes;
                     const uint32_t lbar = mapa_u32(smem_u32(&S.full[ps.stage]), 0u);
-                    if (rank == 0) mbar_arrive_expect_tx(&S.full[ps.stage], 2u * kStageBytes);
+                    if (rank == 0) mbar_arrive_expect_tx(&S.full[ps.stage], tx);
                     tma_load_2d_pair(sa, tma_a, kb * kBK, arow, lbar);
                     if (arow2 >= 0) tma_load_2d_pair(sa + kStageA / 2, tma_a, kb * kBK, arow2, lbar);
                     tma_load_2d_pair(sa + kStageA, tma_b, kb * kBK, brow, lbar);
@@ -1292,6 +1307,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
         fence_mbar_init();
         tma_prefetch_desc(&tm.xe); tma_prefetch_desc(&tm.wgu); tma_prefetch_desc(&tm.h); tma_prefetch_desc(&tm.wd);
         tma_prefetch_desc(&tm.wgu64);
+        for (int i = 0; i < 4; ++i) { tma_prefetch_desc(&tm.xe_n[i]); tma_prefetch_desc(&tm.h_n[i]); }
     }
     if (warp == 1) { tmem_alloc_pair(&S.tmem_base, kTmemCols); tmem_relinquish_pair(); }
     tc_fence_before();

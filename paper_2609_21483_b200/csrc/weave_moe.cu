@@ -147,6 +147,10 @@ int encode_maps(EncodeTiledFn fn, TmaMaps *m, const void *xe, const void *hbuf, 
     r |= encode_map(fn, &m->h, hbuf, p_max, ffn, false);
     r |= encode_map(fn, &m->wd, down, EE * hidden, ffn, true);
     r |= encode_map(fn, &m->wgu64, gate_up, EE * 2 * ffn, hidden, true, 64);
+    for (int i = 0; i < 4; ++i) {
+        r |= encode_map(fn, &m->xe_n[i], xe, p_max, hidden, false, 8u << i);
+        r |= encode_map(fn, &m->h_n[i], hbuf, p_max, ffn, false, 8u << i);
+    }
     return r;
 }
 
