@@ -1217,18 +1217,24 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                         direct_store_32(o, dst + (size_t)lane * p.I + c * 32, lane < rows_valid);
                     }
                 } else {
-                    // batches of 64 out-columns, double-buffered
+                    // batches of 64 out-columns in two register buffers.  A TMEM load takes most of a
+                    // microsecond while the tensor core works on the next tile, and a wait covers every
+                    // load in flight, so the tile's epilogue is a chain of load latencies: the batches
+                    // are fetched two at a time (two latencies instead of four before the accumulator
+                    // can be handed back).
                     __nv_bfloat16 *dst = p.y + (size_t)(ti.row0 + q * 32) * p.H + (size_t)ti.n * 256;
                     const int nb = min(256, p.H - ti.n * 256) / 64;   // the last n-tile may be half wide
                     uint32_t ar[2][64], o[16];
                     tmem_ld_32x64(taddr, ar[0]);
+                    if (nb > 1) tmem_ld_32x64(taddr + 64, ar[1]);
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         if (c < nb) {
-                            tmem_ld_wait64(ar[c & 1]);
-                            if (c + 1 < nb) {
-                                tmem_ld_32x64(taddr + (c + 1) * 64, ar[(c + 1) & 1]);
-                            } else {
+                            if ((c & 1) == 0) {              // an odd batch lands together with the one before it
+                                tmem_ld_wait64(ar[0]);
+                                reg_fence64(ar[1]);
+                            }
+                            if (c + 2 >= nb && !acc_released) {      // every load of the tile has landed
                                 tc_fence_before();
                                 __syncwarp();
                                 if (lane == 0) mbar_arrive_cluster(mapa_u32(smem_u32(&S.tmem_empty[ps.acc]), 0u));
@@ -1242,6 +1248,8 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                                                        __uint_as_float(ar[c & 1][hh * 32 + 2 * i + 1]));
                                 direct_store_32(o, dst + (size_t)lane * p.H + c * 64 + hh * 32, lane < rows_valid);
                             }
+                            // this buffer is free again: fetch the batch after next into it
+                            if (c + 2 < nb) tmem_ld_32x64(taddr + (c + 2) * 64, ar[c & 1]);
                         }
                     }
                 }
