@@ -466,87 +466,59 @@ __device__ __forceinline__ void decode_mblock(const SmemTail &S, int EE, int mb,
     nrows = min(kBM, S.seg_rows[s] - m * kBM);
 }
 
-// number of regular (two-m-block) pair tiles / of unpaired m-blocks in the chunk's segments before s:
-// a segment with pts pair tiles has 2*pts - u m-blocks, u = 1 if its last m-block is unpaired
-__host__ __device__ __forceinline__ int seg_reg0(const SmemTail &S, int s, int cmb0, int cpt0)
-{
-    return (S.seg_mb0[s] - cmb0) - (S.seg_pt0[s] - cpt0);
-}
-__host__ __device__ __forceinline__ int seg_swap0(const SmemTail &S, int s, int cmb0, int cpt0)
-{
-    return 2 * (S.seg_pt0[s] - cpt0) - (S.seg_mb0[s] - cmb0);
-}
-
 // GEMM queue order (the chunk-pipeline DAG order): chunk by chunk; inside a chunk all gemm0 tiles,
 // then all gemm1 tiles (every gemm0 tile a gemm1 tile waits for comes earlier in the queue and waits
-// only for dispatch, which keeps the in-order schedulers free of deadlock).  Each GEMM's tiles are
-// taken in UNITS of one pair tile's worth of n-tiles, of two kinds:
-//  - regular pair tiles (two consecutive m-blocks of one segment): expert-major, then in groups of
-//    kPairGroup pair tiles, n-tile, pair tile fastest (consecutive tiles share a weight panel, and
-//    a group's rows stay in L2 while all its n-tiles pass); bound by the tensor pipe;
-//  - the unpaired last m-blocks of the segments (operands swapped): expert-major, the n-tiles of
-//    one m-block back to back; each streams weight panels that nobody else reads.
-// The swapped units are spread evenly over the regular ones, so that neither HBM nor the tensor
-// pipes idle while a run of small experts (or one large expert) passes.
-// (Alternating gemm1 units with gemm0 units was measured and dropped: it hides the epilogues of the
-// short gemm1 main loops, +1 % at I = 512, but doubles the weight working set in L2, -9 % on the
-// 24-layer Qwen3-235B-shaped stack.)
-// `lead` describes the leader CTA's half of the pair tile, `peer` the other CTA's.  Host-callable so
-// that the order can be checked without a GPU.
+// only for dispatch, which keeps the in-order schedulers free of deadlock); inside those
+// expert-major, then groups of kPairGroup pair tiles, n-tile, pair tile fastest: consecutive tiles
+// share a weight panel, and a group's rows stay in L2 while all its n-tiles pass.  A pair tile = two
+// consecutive m-blocks of one segment; a segment's last, unpaired m-block is a member of its group
+// like any other pair tile (operands swapped), so it reads each weight panel right beside the
+// expert's regular tiles.  `lead` describes the leader CTA's half, `peer` the other CTA's.
+// Two other orders were measured and dropped: spreading the swapped tiles evenly over the queue
+// (no faster, and a large expert's panels were fetched a second time for its last m-block: +27 %
+// DRAM traffic on the Mixtral-shaped layer), and alternating gemm1 with gemm0 units (+1 % at
+// I = 512, -9 % on the Qwen3-235B-shaped stack: two weight working sets in L2).
+// Host-callable so that the order can be checked without a GPU.
 __host__ __device__ __forceinline__ void decode_pair_tile(const SmemTail &S, const KParams &p, int g, TileInfo &lead,
                                                           TileInfo &peer)
 {
     int j = 0;
     while (j + 1 < S.K && g >= S.chunk_tile0[j + 1]) ++j;
     int local = g - S.chunk_tile0[j];
-    const int cpt0 = S.chunk_pt0[j], cmb0 = S.chunk_mb0[j];
-    const int nptj = S.chunk_pt0[j + 1] - cpt0, nswj = S.chunk_nswap[j];
+    const int cpt0 = S.chunk_pt0[j];
+    const int nptj = S.chunk_pt0[j + 1] - cpt0;
     int type = 0, nt = p.nt0;
     if (local >= nptj * p.nt0) { type = 1; local -= nptj * p.nt0; nt = p.nt1; }
-    const int unit = local / nt, w = local - unit * nt;
-    const int sw_before = (int)(((long long)unit * nswj) / nptj);
-    const bool swapped = (int)(((long long)(unit + 1) * nswj) / nptj) > sw_before;
-    lead.type = peer.type = type;
-    lead.chunk = peer.chunk = j;
-    lead.nkb = peer.nkb = (type == 0 ? p.H : p.I) / kBK;
+    // largest s of the chunk with (seg_pt0[s] - cpt0) * nt <= local (empty segments share a start)
     int lo = j * p.EE, hi = (j + 1) * p.EE;
-    if (swapped) {
-        // both CTAs work on the one m-block with the operands swapped, so the MMA costs
-        // ceil(nrows/16)*16 columns instead of a half-empty 256-row tile
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (seg_swap0(S, mid, cmb0, cpt0) <= sw_before) lo = mid; else hi = mid;
-        }
-        const int s = lo;
-        const int m0 = 2 * (S.seg_pt0[s + 1] - S.seg_pt0[s] - 1);
-        lead.type = type + 3;
-        lead.e = s - j * p.EE;
-        lead.n = w;
-        lead.mb = S.seg_mb0[s] + m0;
-        lead.row0 = S.seg_row0[s] + m0 * kBM;
-        lead.nrows = S.seg_rows[s] - m0 * kBM;
-        peer = lead;
-        return;
-    }
-    const int reg = (unit - sw_before) * nt + w;
     while (hi - lo > 1) {
         const int mid = (lo + hi) >> 1;
-        if (seg_reg0(S, mid, cmb0, cpt0) * nt <= reg) lo = mid; else hi = mid;
+        if ((S.seg_pt0[mid] - cpt0) * nt <= local) lo = mid; else hi = mid;
     }
     const int s = lo;
-    const int pts = seg_reg0(S, s + 1, cmb0, cpt0) - seg_reg0(S, s, cmb0, cpt0);
-    const int within = reg - seg_reg0(S, s, cmb0, cpt0) * nt;
+    const int pts = S.seg_pt0[s + 1] - S.seg_pt0[s];
+    const int within = local - (S.seg_pt0[s] - cpt0) * nt;
     const int gi = within / (kPairGroup * nt);
     const int wg = within - gi * kPairGroup * nt;
     const int gsize = (pts - gi * kPairGroup) < kPairGroup ? (pts - gi * kPairGroup) : kPairGroup;
     const int n = wg / gsize;
     const int m0 = 2 * (gi * kPairGroup + (wg - n * gsize));
     const int rows = S.seg_rows[s];
+    lead.type = peer.type = type;
     lead.e = peer.e = s - j * p.EE;
     lead.n = peer.n = n;
+    lead.chunk = peer.chunk = j;
+    lead.nkb = peer.nkb = (type == 0 ? p.H : p.I) / kBK;
     lead.mb = S.seg_mb0[s] + m0;
     lead.row0 = S.seg_row0[s] + m0 * kBM;
-    lead.nrows = kBM;
+    lead.nrows = (rows - m0 * kBM) < kBM ? (rows - m0 * kBM) : kBM;
+    if (rows - (m0 + 1) * kBM <= 0) {
+        // the segment's last, unpaired m-block: both CTAs work on it with the operands swapped,
+        // so the MMA costs ceil(nrows/16)*16 columns instead of a half-empty 256-row tile
+        lead.type = type + 3;
+        peer = lead;
+        return;
+    }
     peer.nrows = (rows - (m0 + 1) * kBM) < kBM ? (rows - (m0 + 1) * kBM) : kBM;
     peer.mb = lead.mb + 1;
     peer.row0 = lead.row0 + kBM;

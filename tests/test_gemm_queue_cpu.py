@@ -64,17 +64,13 @@ def test_empty_layer_and_single_block():
     assert (q[:, 0] >= 3).all() and len(q) == 5                   # one swapped unit: 3 gemm0 then 2 gemm1 tiles
 
 
-def test_swapped_units_are_spread_over_the_regular_ones():
-    """16 one-block experts followed by one large expert: the swapped units do not form one run."""
-    rows = np.array([[100] * 16 + [128 * 2 * 160]], np.int32)
-    q = replay(rows, 4, 2)
-    g0 = q[q[:, 0] % 3 == 0]                                      # gemm0 tiles (types 0 and 3)
-    sw = np.flatnonzero(g0[:, 0] == 3) // 4                       # unit position of each swapped tile
-    units = np.unique(sw)
-    assert len(units) == 16 and np.diff(units).min() >= 5         # 176 units, 16 swapped: every 11th
-    # a swapped unit's n-tiles are consecutive
-    for u in units:
-        assert (g0[u * 4:(u + 1) * 4, 0] == 3).all() and list(g0[u * 4:(u + 1) * 4, 3]) == [0, 1, 2, 3]
+def test_an_unpaired_block_reads_each_weight_panel_beside_its_expert():
+    """One expert with five m-blocks: its last, unpaired m-block is a member of the group, so the tile
+    of n-tile j comes right after the two regular pair tiles of n-tile j (same weight panel)."""
+    q = replay([[128 * 5]], 3, 2)
+    g0 = q[:9]
+    assert list(g0[:, 0]) == [0, 0, 3] * 3 and list(g0[:, 3]) == [0, 0, 0, 1, 1, 1, 2, 2, 2]
+    assert list(g0[:, 1]) == [0, 2, 4] * 3
 
 
 def test_bad_arguments():
