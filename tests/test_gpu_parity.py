@@ -119,6 +119,7 @@ def test_ragged_token_counts(T):
     (256, 128, 16, 16, 0),    # the largest k
     (256, 256, 248, 8, 8),    # E + S = 256, the largest expert count; most experts empty or tiny
     (512, 640, 5, 3, 1),      # odd expert count, one shared expert
+    (16384, 128, 4, 2, 0),    # the largest hidden size: one row fills a whole movement buffer
 ])
 def test_shape_edges(H, I, E, k, S):
     cfg = _small(f"edge_{H}_{I}_{E}_{k}_{S}", 200, H, I, E, k, S)
