@@ -173,15 +173,34 @@ def grid_sweep(moe, xl, cfg, tables, verbose=True):
             moe.set_schedule(pk.SCHED_FIXED, c, K, plan["n_steal"])
             res[(c, K)] = time_it(3)
     best = min(res, key=res.get)
+    # the model's own (c*, K*) as a forced point: the selection gap inside the grid (the AUTO run above
+    # also has the elastic stealing and the first dispatch wave on all SMs, which no forced run has)
+    moe.set_schedule(pk.SCHED_FIXED, plan["c"], plan["K"], plan["n_steal"])
+    t_pick = time_it(3)
     moe.set_schedule(pk.SCHED_SERIAL)
     t_serial = time_it()
+    # what the in-kernel search costs: set-up time with and without it, from the timeline
+    def setup_us(mode, *a):
+        moe.set_schedule(mode, *a)
+        moe.enable_trace(4096)
+        moe.forward(x, lg)
+        moe.forward(x, lg)
+        ev = _events(moe)
+        moe.enable_trace(0)
+        e = ev[ev[:, 3] == 2]
+        return float(((e[:, 2] - e[:, 1]) / 1e3).mean())
+    su_auto, su_fixed = setup_us(pk.SCHED_AUTO), setup_us(pk.SCHED_FIXED, plan["c"], plan["K"], plan["n_steal"])
     if verbose:
         print("grid (us):")
         for c in C_POINTS:
             print(f"  c={c:3d} " + " ".join(f"K={K}:{res.get((c, K), float('nan')):8.1f}" for K in K_POINTS))
         print(f"AUTO plan {plan} -> {t_auto:.1f} us; measured optimum {best} -> {res[best]:.1f} us; "
               f"gap {100 * (t_auto / res[best] - 1):.1f} %; SERIAL {t_serial:.1f} us")
-    return {"auto_us": t_auto, "plan": plan, "best": best, "best_us": res[best], "serial_us": t_serial}
+        print(f"model's pick forced: {t_pick:.1f} us, selection gap inside the grid {100 * (t_pick / min(res[best], t_pick) - 1):.1f} %; "
+              f"set-up {su_auto:.2f} us with the search, {su_fixed:.2f} us without")
+    return {"workload": cfg.name, "auto_us": t_auto, "plan": plan, "best": list(best), "best_us": res[best],
+            "pick_us": t_pick, "selection_gap": t_pick / min(res[best], t_pick) - 1, "auto_vs_best": t_auto / res[best] - 1,
+            "serial_us": t_serial, "setup_us_auto": su_auto, "setup_us_fixed": su_fixed, "grid_points": len(res)}
 
 
 def main():
@@ -196,7 +215,7 @@ def main():
     moe, xl, tables = calibrate(cfg, args.layer)
     print("alpha", tables["alpha"], "eff_chunk", tables["eff_chunk"].tolist())
     if args.grid:
-        grid_sweep(moe, xl, cfg, tables)
+        print(json.dumps(grid_sweep(moe, xl, cfg, tables)))
     if args.out:
         with open(args.out, "w") as f:
             json.dump({k: (v.tolist() if isinstance(v, np.ndarray) else v) for k, v in tables.items()}, f)
