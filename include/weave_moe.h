@@ -151,8 +151,10 @@ int weave_moe_get_plan(weave_moe_t h, int *c, int *K, int *n_steal, float *t_tot
 /* Geometry the scheduler works with: number of SMs used (= persistent CTAs; an even number,
  * because the GEMM phase runs on pairs of neighbouring SMs), rows per m-block (the unit of the
  * dispatch queue and of the ready flags), h-columns per gemm0 tile, out-columns per gemm1 tile,
- * tokens per routing block, tokens per combine tile, rows per GEMM tile (two m-blocks of one
- * expert segment; a segment with an odd number of m-blocks ends in a half-empty tile).
+ * tokens per routing block, tokens per combine tile (the largest size: a batch that would give
+ * fewer tiles than SMs is cut into tiles of half that size, repeatedly, down to one token), rows
+ * per GEMM tile (two m-blocks of one expert segment; a segment with an odd number of m-blocks ends
+ * in a half-empty tile).
  * Any pointer may be NULL. */
 int weave_moe_get_geometry(weave_moe_t h, int *n_sm, int *block_m, int *tile_n0, int *tile_n1,
                            int *route_block, int *combine_tile, int *gemm_tile_m);

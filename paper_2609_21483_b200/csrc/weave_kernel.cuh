@@ -32,7 +32,7 @@ constexpr int kStageB = 128 * kBK * 2;                  // 16 KB: this CTA's hal
 constexpr int kStageBytes = kStageA + kStageB;          // 32 KB
 constexpr int kEpiStageBytes = 4 * 32 * 64;             // epilogue staging: per warp 32 rows x 64 bytes
 constexpr int kRouteBlock = 64;  // tokens per routing block (one 64-bit mask per expert)
-constexpr int kCombTile = 16;    // tokens per combine tile
+constexpr int kCombTile = 16;    // tokens per combine tile (fewer when the batch would give fewer tiles than SMs)
 constexpr int kMaxEE = 256;      // routed + shared experts
 constexpr int kMaxTopK = 16;
 constexpr int kFine = 8;         // fine chunks = largest chunk count K
@@ -152,6 +152,7 @@ struct SmemTail {
     int scan_w[8];
     int scan_total;
     int c, K, steal, nmb, n_gemm, n_comb;
+    int comb_tok;                // tokens per combine tile of this launch: 16, 8, 4, 2 or 1
     unsigned trace_n;
     int chunk_mb0[kFine + 1];
     int chunk_pt0[kFine + 1];
@@ -738,7 +739,7 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uin
             if (lane == 0) q = (int)atomicAdd(&p.ctl->q_comb, 1u);
             q = __shfl_sync(0xffffffffu, q, 0);
             if (q >= S.n_comb) break;
-            const int t0 = q * kCombTile;
+            const int t0 = q * S.comb_tok;
             const int chunk = (((t0 / kRouteBlock) * kFine) / p.nblk) / g;
             if (chunk > ready_upto) {
                 if (lane == 0) {
@@ -754,7 +755,7 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uin
                 ready_upto = chunk;
             }
             const unsigned long long tc0 = trace_now(p);
-            const int ntok = min(kCombTile, p.T - t0);
+            const int ntok = min(S.comb_tok, p.T - t0);
             for (int i = lane; i < ntok * kk; i += 32) {
                 const int tt = i / kk, j = i - tt * kk, t = t0 + tt;
                 S.crow[tt][j] = j < p.k ? __ldcg(p.row_of + (size_t)t * p.k + j) : S.offsets[p.E + (j - p.k)] + t;
@@ -937,7 +938,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                         const unsigned qc = ld_relaxed_u32(&p.ctl->q_comb);
                         if (qc >= (unsigned)S.n_comb) more = true;
                         else {
-                            const int ch = ((((int)qc * kCombTile / kRouteBlock) * kFine) / p.nblk) / (kFine / S.K);
+                            const int ch = ((((int)qc * S.comb_tok / kRouteBlock) * kFine) / p.nblk) / (kFine / S.K);
                             more = ld_acquire_u32(&p.ctl->y_done[ch]) < y_done_target(S, p, ch);
                         }
                     }
@@ -1487,7 +1488,13 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
             S.c = plan_c; S.K = K; S.steal = plan_steal;
             S.nmb = mb_base;
             S.n_gemm = pt_base * (p.nt0 + p.nt1);
-            S.n_comb = (p.T + kCombTile - 1) / kCombTile;
+            // a small batch is cut into smaller combine tiles (powers of two, so that a tile never
+            // straddles two chunks) until every SM has one: its final combine is a latency chain
+            // per tile, not a bandwidth problem
+            int ct = kCombTile;
+            while (ct > 1 && (p.T + ct - 1) / ct < n_sm) ct >>= 1;
+            S.comb_tok = ct;
+            S.n_comb = (p.T + ct - 1) / ct;
             if (blockIdx.x == 0) {
                 p.ctl->plan_c = plan_c; p.ctl->plan_K = K; p.ctl->plan_steal = plan_steal; p.ctl->plan_t = plan_t;
                 p.ctl->plan_nmb = mb_base; p.ctl->plan_ngemm = pt_base * (p.nt0 + p.nt1);
