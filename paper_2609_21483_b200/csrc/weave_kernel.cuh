@@ -887,15 +887,35 @@ __device__ __forceinline__ void linger_after_abort()
     while (globaltimer_ns() - t0 < 50000ull) __nanosleep(1000);
 }
 
-// Thread = row: 32 columns of bf16 (16 packed words) straight from registers as two 32-byte stores,
-// each a full sector.  No shared memory: during the GEMM phase its bandwidth belongs to the TMA
-// writes and the tensor core's operand reads, and a staged epilogue would queue behind them.
-__device__ __forceinline__ void direct_store_32(const uint32_t (&o)[16], __nv_bfloat16 *dst_row, bool valid)
+// 32 rows x 32 columns of bf16 held one row per thread (16 packed words each) go out through the
+// warp's own 2 KB of shared memory, so that every store instruction writes 16 rows x 64 contiguous
+// bytes (two lanes per row) instead of 32 rows x 32 bytes.  An SM retires st.global at 32 B per
+// cycle but at most one 128-byte line every two cycles: one row per thread is 15.8 B/clk per SM,
+// two lanes per row 31 B/clk (measured with a store-only probe, alone or on all SMs).
+// Shared-memory layout: row r at r*64, its 16-byte chunk c at position c ^ ((r >> 1) & 3): the
+// row-per-thread writes and the two-lanes-per-row reads are both free of bank conflicts.
+// dst = first of the warp's 32 rows (this batch's first column), pitch in elements.
+__device__ __forceinline__ void staged_store_32(const uint32_t (&o)[16], uint32_t stage, __nv_bfloat16 *dst, int pitch,
+                                                int rows_valid, int lane)
 {
-    if (valid) {
-        st_v8(dst_row, &o[0]);
-        st_v8(dst_row + 16, &o[8]);
+    const uint32_t wbase = stage + (uint32_t)lane * 64u, wsw = (uint32_t)((lane >> 1) & 3);
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+        st_shared_v4(wbase + (((uint32_t)c ^ wsw) << 4), make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]));
+    __syncwarp();
+    const int half = lane & 1;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        const int r = 16 * j + (lane >> 1);
+        const uint32_t rbase = stage + (uint32_t)r * 64u, rsw = (uint32_t)((r >> 1) & 3);
+        const uint4 q0 = ld_shared_v4(rbase + (((uint32_t)(2 * half) ^ rsw) << 4));
+        const uint4 q1 = ld_shared_v4(rbase + (((uint32_t)(2 * half + 1) ^ rsw) << 4));
+        if (r < rows_valid) {
+            const uint32_t v[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+            st_v8(dst + (size_t)r * pitch + half * 16, v);
+        }
     }
+    __syncwarp();      // the region is rewritten by the next batch
 }
 
 // budget = how many pair tiles this CTA pair may claim (the steal count for a movement pair).
@@ -1086,6 +1106,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
             tc_fence_after();
             const unsigned long long te0 = trace_now(p);
             const int rows_valid = ti.nrows - q * 32;          // rows of this warp's quadrant that exist
+            const uint32_t epi_stage = smem_u32(stages + kStages * kStageBytes) + (uint32_t)q * 2048u;   // this warp's staging
             bool acc_released = false;
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)ps.acc * 256u;
             if (ti.type == 3) {
@@ -1187,7 +1208,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                         for (int i = 0; i < 16; ++i)
                             o[i] = pack_bf16x2(silu_mul(__uint_as_float(gr[c & 1][2 * i]), __uint_as_float(ur[c & 1][2 * i])),
                                                silu_mul(__uint_as_float(gr[c & 1][2 * i + 1]), __uint_as_float(ur[c & 1][2 * i + 1])));
-                        direct_store_32(o, dst + (size_t)lane * p.I + c * 32, lane < rows_valid);
+                        staged_store_32(o, epi_stage, dst + c * 32, p.I, rows_valid, lane);
                     }
                 } else {
                     // batches of 64 out-columns in two register buffers.  A TMEM load takes most of a
@@ -1219,7 +1240,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                                 for (int i = 0; i < 16; ++i)
                                     o[i] = pack_bf16x2(__uint_as_float(ar[c & 1][hh * 32 + 2 * i]),
                                                        __uint_as_float(ar[c & 1][hh * 32 + 2 * i + 1]));
-                                direct_store_32(o, dst + (size_t)lane * p.H + c * 64 + hh * 32, lane < rows_valid);
+                                staged_store_32(o, epi_stage, dst + c * 64 + hh * 32, p.H, rows_valid, lane);
                             }
                             // this buffer is free again: fetch the batch after next into it
                             if (c + 2 < nb) tmem_ld_32x64(taddr + (c + 2) * 64, ar[c & 1]);
