@@ -78,7 +78,10 @@ int weave_moe_create(const weave_moe_config *cfg, weave_moe_t *out_handle);
  * (fully overwritten).  All three 16-byte aligned, not aliasing each other or the workspace.
  * 0 <= T <= max_tokens (T = 0 is a no-op).  cuda_stream: a cudaStream_t (NULL = default stream).
  * Launches exactly one kernel; returns once it is enqueued.  Device-side failures
- * (WEAVE_ERR_NONFINITE_LOGITS, WEAVE_ERR_TIMEOUT) are reported by weave_moe_status(). */
+ * (WEAVE_ERR_NONFINITE_LOGITS, WEAVE_ERR_TIMEOUT) are reported by weave_moe_status().
+ * The call makes no other CUDA call (no allocation, copy, memset or synchronisation: the kernel
+ * re-zeroes its own control words), so a sequence of layers may be captured into a CUDA graph on
+ * `cuda_stream`; the replay reads the arguments and the schedule settings given at capture time. */
 int weave_moe_forward(weave_moe_t h, const void *x, const float *router_logits, void *out, int T,
                       void *cuda_stream);
 

@@ -231,6 +231,33 @@ def test_handle_reuse_smaller_batches_and_run_to_run_bits():
     moe.close()
 
 
+def test_layers_captured_in_a_cuda_graph_replay_bit_for_bit():
+    """forward() enqueues one (cooperative) kernel and nothing else, so a stack of layers can be
+    captured into a CUDA graph; the replay gives the bits of the direct calls."""
+    cfg = _small("graph", 300, 256, 384, 8, 2)
+    inp = wl.make_inputs(cfg)
+    x, lg, gu, dn = to_dev(inp)
+    moe = pk.WeaveMoE(gu, dn, cfg.E, cfg.k, cfg.S, max_tokens=cfg.T)
+    ref1 = moe.forward(x, lg).clone()
+    ref2 = moe.forward(ref1, lg).clone()           # a second "layer" fed by the first
+    moe.check()
+    o1, o2 = torch.empty_like(x), torch.empty_like(x)
+    s = torch.cuda.Stream()
+    s.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=s):
+        moe.forward(x, lg, out=o1)
+        moe.forward(o1, lg, out=o2)
+    for _ in range(3):
+        o1.zero_(); o2.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(o1.view(torch.int16), ref1.view(torch.int16))
+        assert torch.equal(o2.view(torch.int16), ref2.view(torch.int16))
+    moe.check()
+    moe.close()
+
+
 def test_forward_host_equals_forward():
     cfg = wl.CONFIGS["c1_tiny"]
     inp = wl.make_inputs(cfg)
