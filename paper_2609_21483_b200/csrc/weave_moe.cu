@@ -228,7 +228,7 @@ int weave_moe_create(const weave_moe_config *cfg, weave_moe_t *out)
     h->c_max = h->n_sm / 2;
     h->c_step = 2;
     h->alpha = 0.8f;
-    h->eff[0] = 1.0f; h->eff[1] = 0.90f; h->eff[2] = 0.80f; h->eff[3] = 0.65f;
+    h->eff[0] = 1.0f; h->eff[1] = 0.83f; h->eff[2] = 0.62f; h->eff[3] = 0.43f;     // measured (calibration tool)
     h->timeout_ms = 4000;
     h->withhold_mb = -1;
     h->last_T = 0;
@@ -738,7 +738,7 @@ int weave_moe_forward_static(int hidden, int ffn, int num_experts, int top_k, in
     h.fixed_c = (h.n_sm * 15 / 100 + 1) & ~1; h.fixed_K = 1; h.fixed_steal = 0;
     h.c_min = 2; h.c_max = h.n_sm / 2; h.c_step = 2;
     h.alpha = 0.8f;
-    h.eff[0] = 1.0f; h.eff[1] = 0.90f; h.eff[2] = 0.80f; h.eff[3] = 0.65f;
+    h.eff[0] = 1.0f; h.eff[1] = 0.83f; h.eff[2] = 0.62f; h.eff[3] = 0.43f;
     h.timeout_ms = 4000;
     h.withhold_mb = -1;
     h.ep_rank = 0;
