@@ -1,7 +1,8 @@
 // The persistent MoE-layer megakernel: one CTA per SM, one launch per layer.
 //
-//   phase R  (all CTAs)   warp-level top-k routing, per-block expert bitmasks -> in-block ranks and
-//                         a [block][expert] histogram; grid barrier (bounded)
+//   phase R  (all CTAs)   top-k routing of 64-token blocks (four threads per token, lists merged by
+//                         shuffles), per-block expert bitmasks -> in-block ranks and a
+//                         [block][expert] histogram; grid barrier (bounded)
 //   set-up   (every CTA, redundantly) counts, offsets, candidate tile counts, cost model -> plan
 //                         (c, K, n_steal), segment tables of the chosen K; permutation fix-up
 //   phase A  (movement CTAs: blockIdx < c)  dispatch tiles: gather x rows into expert-major Xe
