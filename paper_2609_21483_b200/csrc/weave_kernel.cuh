@@ -769,8 +769,11 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uin
                 const int myrow = lane < kk ? S.crow[tt][lane] : -1;
                 const unsigned vmask = __ballot_sync(0xffffffffu, myrow >= 0);
                 const int nv = __popc(vmask), mypos = __popc(vmask & ((1u << lane) - 1u));
-                for (int col0 = 0; col0 < p.H && ok; col0 += W) {
-                    const int w = min(W, p.H - col0);
+                // a token with few rows here (expert-parallel share) takes wider pieces: as many columns
+                // as fit the buffer with the rows it really has
+                const int Wt = nv >= kk ? W : min(p.H, ((kMvBuf / (2 * max(nv, 1))) / 64) * 64);
+                for (int col0 = 0; col0 < p.H && ok; col0 += Wt) {
+                    const int w = min(Wt, p.H - col0);
                     if (lane == 0) {
                         if (!mbar_wait(&S.cb_empty[b], ph ^ 1u, p, 22)) ok = false;
                         else {
