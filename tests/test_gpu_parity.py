@@ -127,6 +127,32 @@ def test_shape_edges(H, I, E, k, S):
     moe.close()
 
 
+@pytest.mark.parametrize("seed", range(64))
+def test_random_shapes_and_schedules(seed):
+    """Seeded random layer shapes, routing skews and schedules against the oracle (whole output)."""
+    rng = np.random.default_rng(1000 + seed)
+    E = int(rng.choice([1, 2, 3, 5, 8, 16, 33, 64, 100]))
+    k = int(rng.integers(1, min(E, 8) + 1))
+    S = int(rng.choice([0, 0, 1, 2]))
+    T = int(rng.choice([1, 7, 64, 65, 127, 200, 333, 512, 700]))
+    H = int(rng.choice([128, 256, 384, 640, 1024]))
+    I = int(rng.choice([128, 256, 384, 768]))
+    zipf = [None, 0.5, 1.5, 3.0][int(rng.integers(0, 4))]
+    cfg = _small(f"rand{seed}", T, H, I, E, k, S, zipf=zipf, cfg_id=200 + seed)
+    mode = int(rng.integers(0, 3))
+    if mode == 0:
+        sched = None
+    elif mode == 1:
+        sched = (pk.SCHED_SERIAL, 0, 1, 0)
+    else:
+        K = int(rng.choice([1, 2, 4, 8]))
+        while K * (E + S) > 1024:
+            K //= 2
+        sched = (pk.SCHED_FIXED, int(rng.integers(2, 80)), K, int(rng.integers(0, 50)))
+    moe, _, _ = run_case(cfg, sched=sched)
+    moe.close()
+
+
 def test_many_tokens_small_experts():
     """A long batch (625 routing blocks, 8 fine chunks of 78-79 blocks, ~80 000 rows) on small
     experts, chunked and unchunked: exercises the block/chunk prefix machinery at size."""
