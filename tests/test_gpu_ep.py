@@ -126,3 +126,34 @@ def test_c5_shaped_rank_share_sampled():
     ref = oracle.moe_tokens_ep(inp.x, inp.logits, inp.gate_up, inp.down, cfg.k, toks, 0, 4)
     check_values(bf16_to_np(out[torch.from_numpy(toks).long().cuda()]), ref, "c5 rank 0")
     moe.close()
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_groups_shapes_and_ranks(seed):
+    """Seeded random EP groups: one rank's routing, descriptors and partial output against the oracle."""
+    rng = np.random.default_rng(7000 + seed)
+    R = int(rng.choice([2, 4, 8]))
+    E = R * int(rng.choice([1, 2, 4, 8]))
+    k = int(rng.integers(1, min(E, 8) + 1))
+    T = int(rng.choice([1, 5, 64, 130, 300, 700]))
+    H = int(rng.choice([128, 256, 640]))
+    I = int(rng.choice([128, 384]))
+    zipf = [None, 1.0, 3.0][int(rng.integers(0, 3))]
+    cfg = wl.MoEConfig(f"ep_rand{seed}", 300 + seed, T=T, H=H, I=I, E=E, k=k, zipf_s=zipf)
+    inp = wl.make_inputs(cfg)
+    x, lg, gu, dn = to_dev(inp)
+    moe = pk.WeaveMoE(gu, dn, cfg.E, cfg.k, cfg.S, max_tokens=cfg.T)
+    r = int(rng.integers(0, R))
+    moe.set_expert_parallel(r, R)
+    if rng.random() < 0.5:
+        K = int(rng.choice([1, 2, 4]))
+        moe.set_schedule(pk.SCHED_FIXED, int(rng.integers(2, 60)), K, int(rng.integers(0, 20)))
+    out = moe.forward(x, lg)
+    moe.check()
+    _check_rank(moe, inp, r, R)
+    ref = oracle.moe_tokens_ep(inp.x, inp.logits, inp.gate_up, inp.down, cfg.k, np.arange(cfg.T, dtype=np.int32), r, R)
+    if np.abs(ref).max() > 0:
+        check_values(bf16_to_np(out), ref, f"seed {seed} rank {r}/{R}")
+    else:
+        assert bool((out == 0).all())
+    moe.close()
