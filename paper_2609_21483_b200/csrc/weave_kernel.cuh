@@ -31,7 +31,7 @@ constexpr int kStages = 6;
 constexpr int kStageA = kBM * kBK * 2;                  // 16 KB: this CTA's 128 rows of A
 constexpr int kStageB = 128 * kBK * 2;                  // 16 KB: this CTA's half (128 rows) of the 256-row B tile
 constexpr int kStageBytes = kStageA + kStageB;          // 32 KB
-constexpr int kEpiStageBytes = 4 * 32 * 64;             // epilogue staging: per warp 32 rows x 64 bytes
+constexpr int kEpiStageBytes = 4 * 2 * 32 * 64;         // epilogue staging: per warp two buffers of 32 rows x 64 bytes
 constexpr int kRouteBlock = 64;  // tokens per routing block (one 64-bit mask per expert)
 constexpr int kCombTile = 16;    // tokens per combine tile (fewer when the batch would give fewer tiles than SMs)
 constexpr int kMaxEE = 256;      // routed + shared experts
@@ -145,7 +145,6 @@ struct SmemTail {
     uint64_t cb_full[kStages], cb_empty[kStages];   // combine: loader -> reducing warps
     uint64_t xg_full, xg_empty;                     // swapped gemm0 epilogue: up warps -> gate warps
     TileInfo ti[kTinfo];
-    MvDesc mv[kStages];
     uint32_t tmem_base;
     int bcast[3];
     int red_i[8][4];
@@ -160,14 +159,25 @@ struct SmemTail {
     int chunk_nswap[kFine];      // per chunk: segments with an odd number of m-blocks
     int chunk_tile0[kFine + 1];
     int offsets[kMaxEE + 1];
-    int tok[kBM];
-    int crow[kCombTile][kMaxTopK + 8];
-    float cgate[kCombTile][kMaxTopK + 8];
     int seg_mb0[kMaxSeg + 1];
     int seg_pt0[kMaxSeg + 1];    // prefix of pair tiles: ceil(m-blocks / 2) per segment
     int seg_row0[kMaxSeg];
     int seg_rows[kMaxSeg];
 };
+
+// Scratch of the movement phases (dispatch, combine).  A CTA is in one phase at a time, so it shares
+// its space with the second half of the GEMM epilogue's staging area.
+struct MoveScratch {
+    MvDesc mv[kStages];
+    int tok[kBM];
+    int crow[kCombTile][kMaxTopK + 8];
+    float cgate[kCombTile][kMaxTopK + 8];
+};
+static_assert(sizeof(MoveScratch) <= kEpiStageBytes / 2, "movement scratch must fit half of the staging area");
+__device__ __forceinline__ MoveScratch &move_scratch(uint8_t *stages)
+{
+    return *reinterpret_cast<MoveScratch *>(stages + kStages * kStageBytes + kEpiStageBytes / 2);
+}
 
 constexpr int kSmemBytes = kStages * kStageBytes + kEpiStageBytes + (int)sizeof(SmemTail) + 1024;
 static_assert(kSmemBytes <= 232448, "exceeds the 227 KB a CTA may opt into");
@@ -542,6 +552,7 @@ __device__ __forceinline__ unsigned y_done_target(const SmemTail &S, const KPara
 // its last store has completed.
 __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, uint8_t *stages, int max_tiles)
 {
+    MoveScratch &M = move_scratch(stages);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     fence_proxy_async();      // the buffers held routing scratch written with ordinary stores
     __syncthreads();
@@ -569,7 +580,7 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
                     const int bit = lane + 32 * hh;
-                    if ((um >> bit) & 1ull) S.tok[__popcll(um & ((1ull << bit) - 1ull))] = blk * kRouteBlock + bit;
+                    if ((um >> bit) & 1ull) M.tok[__popcll(um & ((1ull << bit) - 1ull))] = blk * kRouteBlock + bit;
                 }
                 __syncwarp();
                 if (lane == 0) {
@@ -580,12 +591,12 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
                         for (int r0 = 0; r0 < n; r0 += Rp) {
                             const int nr = min(Rp, n - r0);
                             if (!mbar_wait(&S.dv_empty[b], ph ^ 1u, p, 14)) { ok = false; break; }
-                            S.mv[b].a = 0; S.mv[b].b = nr; S.mv[b].c = blk; S.mv[b].d = (r0 + nr >= n) ? 4 : 3;
-                            for (int i = 0; i < nr; ++i) S.mv[b].tok[i] = S.tok[r0 + i];
+                            M.mv[b].a = 0; M.mv[b].b = nr; M.mv[b].c = blk; M.mv[b].d = (r0 + nr >= n) ? 4 : 3;
+                            for (int i = 0; i < nr; ++i) M.mv[b].tok[i] = M.tok[r0 + i];
                             mbar_arrive_expect_tx(&S.dv_full[b], (uint32_t)nr * rowb);
                             const uint32_t dst = smem_u32(stages + b * kMvBuf);
                             for (int i = 0; i < nr; ++i)
-                                bulk_load(dst + (uint32_t)i * rowb, p.x + (size_t)S.tok[r0 + i] * p.H, rowb, &S.dv_full[b]);
+                                bulk_load(dst + (uint32_t)i * rowb, p.x + (size_t)M.tok[r0 + i] * p.H, rowb, &S.dv_full[b]);
                             if (++b == kStages) { b = 0; ph ^= 1u; }
                         }
                     }
@@ -597,7 +608,7 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
             // complete and publish what it still holds back (d = 5), then wait for everybody's blocks
             if (lane == 0 && ok) {
                 if (mbar_wait(&S.dv_empty[b], ph ^ 1u, p, 16)) {
-                    S.mv[b].d = 5;
+                    M.mv[b].d = 5;
                     mbar_arrive(&S.dv_full[b]);
                     if (++b == kStages) { b = 0; ph ^= 1u; }
                 } else ok = false;
@@ -615,14 +626,14 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
             if (mb >= S.nmb) break;
             int row0, nrows;
             decode_mblock(S, p.EE, mb, row0, nrows);
-            for (int i = lane; i < nrows; i += 32) S.tok[i] = __ldcg(p.token_of + row0 + i);
+            for (int i = lane; i < nrows; i += 32) M.tok[i] = __ldcg(p.token_of + row0 + i);
             __syncwarp();
             for (int r0 = 0; r0 < nrows && ok; r0 += R) {
                 const int nr = min(R, nrows - r0);
                 if (lane == 0) {
                     if (!mbar_wait(&S.dv_empty[b], ph ^ 1u, p, 11)) ok = false;
                     else {
-                        S.mv[b].a = row0 + r0; S.mv[b].b = nr; S.mv[b].c = mb; S.mv[b].d = (r0 + nr >= nrows) ? 1 : 0;
+                        M.mv[b].a = row0 + r0; M.mv[b].b = nr; M.mv[b].c = mb; M.mv[b].d = (r0 + nr >= nrows) ? 1 : 0;
                         mbar_arrive_expect_tx(&S.dv_full[b], (uint32_t)nr * rowb);
                     }
                 }
@@ -631,7 +642,7 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
                 // the expected byte count is registered; the lanes issue the row copies side by side
                 const uint32_t dst = smem_u32(stages + b * kMvBuf);
                 for (int i = lane; i < nr; i += 32) {
-                    const int tk = S.tok[r0 + i];
+                    const int tk = M.tok[r0 + i];
                     // a remote token (another rank's shard) is read from its staged copy
                     const __nv_bfloat16 *src = (p.ep_size > 1 && tk / p.ep_tshard != p.ep_rank) ? p.xs : p.x;
                     bulk_load(dst + (uint32_t)i * rowb, src + (size_t)tk * p.H, rowb, &S.dv_full[b]);
@@ -642,7 +653,7 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
             __syncwarp();
         }
         if (lane == 0 && ok && mbar_wait(&S.dv_empty[b], ph ^ 1u, p, 12)) {
-            S.mv[b].d = 2;
+            M.mv[b].d = 2;
             mbar_arrive(&S.dv_full[b]);
         }
         __syncwarp();
@@ -676,7 +687,7 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
             unsigned long long tile_t0 = trace_now(p);
             for (;;) {
                 if (!mbar_wait(&S.dv_full[b], ph, p, 13)) break;
-                const int da = S.mv[b].a, db = S.mv[b].b, dc = S.mv[b].c, dd = S.mv[b].d;
+                const int da = M.mv[b].a, db = M.mv[b].b, dc = M.mv[b].c, dd = M.mv[b].d;
                 if (dd == 2) break;
                 if (dd == 5) {      // flush: everything stored so far becomes visible and is published
                     bulk_wait<0>();
@@ -688,7 +699,7 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
                 }
                 if (dd >= 3) {      // staged remote tokens: one store per row, to the token's own slot of xs
                     for (int i = 0; i < db; ++i)
-                        bulk_store(p.xs + (size_t)S.mv[b].tok[i] * p.H, smem_u32(stages + b * kMvBuf) + (uint32_t)i * rowb, rowb);
+                        bulk_store(p.xs + (size_t)M.mv[b].tok[i] * p.H, smem_u32(stages + b * kMvBuf) + (uint32_t)i * rowb, rowb);
                 } else {
                     bulk_store(p.xe + (size_t)da * p.H, smem_u32(stages + b * kMvBuf), (uint32_t)db * rowb);
                 }
@@ -723,6 +734,7 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
 // each full buffer from shared memory and write the output row piece with coalesced stores.
 __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uint8_t *stages)
 {
+    MoveScratch &M = move_scratch(stages);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     fence_proxy_async();
     __syncthreads();
@@ -759,14 +771,14 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uin
             const int ntok = min(S.comb_tok, p.T - t0);
             for (int i = lane; i < ntok * kk; i += 32) {
                 const int tt = i / kk, j = i - tt * kk, t = t0 + tt;
-                S.crow[tt][j] = j < p.k ? __ldcg(p.row_of + (size_t)t * p.k + j) : S.offsets[p.E + (j - p.k)] + t;
-                S.cgate[tt][j] = j < p.k ? __ldcg(p.gates + (size_t)t * p.k + j) : 1.0f;
+                M.crow[tt][j] = j < p.k ? __ldcg(p.row_of + (size_t)t * p.k + j) : S.offsets[p.E + (j - p.k)] + t;
+                M.cgate[tt][j] = j < p.k ? __ldcg(p.gates + (size_t)t * p.k + j) : 1.0f;
             }
             __syncwarp();
             for (int tt = 0; tt < ntok && ok; ++tt) {
                 // lane j owns slot j of the token: its rank among the slots that have a row here (slots
                 // whose expert lives on another rank have row -1 and are skipped)
-                const int myrow = lane < kk ? S.crow[tt][lane] : -1;
+                const int myrow = lane < kk ? M.crow[tt][lane] : -1;
                 const unsigned vmask = __ballot_sync(0xffffffffu, myrow >= 0);
                 const int nv = __popc(vmask), mypos = __popc(vmask & ((1u << lane) - 1u));
                 // a token with few rows here (expert-parallel share) takes wider pieces: as many columns
@@ -777,12 +789,12 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uin
                     if (lane == 0) {
                         if (!mbar_wait(&S.cb_empty[b], ph ^ 1u, p, 22)) ok = false;
                         else {
-                            S.mv[b].a = t0 + tt; S.mv[b].b = col0; S.mv[b].c = w; S.mv[b].d = 0; S.mv[b].n = nv;
+                            M.mv[b].a = t0 + tt; M.mv[b].b = col0; M.mv[b].c = w; M.mv[b].d = 0; M.mv[b].n = nv;
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, ok, 0);
                     if (!ok) break;
-                    if (myrow >= 0) S.mv[b].g[mypos] = S.cgate[tt][lane];
+                    if (myrow >= 0) M.mv[b].g[mypos] = M.cgate[tt][lane];
                     __syncwarp();
                     if (lane == 0) {
                         if (nv > 0) mbar_arrive_expect_tx(&S.cb_full[b], (uint32_t)(nv * w * 2));
@@ -802,7 +814,7 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uin
             __syncwarp();
         }
         if (lane == 0 && ok && mbar_wait(&S.cb_empty[b], ph ^ 1u, p, 23)) {
-            S.mv[b].d = 2;
+            M.mv[b].d = 2;
             mbar_arrive(&S.cb_full[b]);
         }
         __syncwarp();
@@ -815,7 +827,7 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uin
             bool ok = mbar_wait(&S.cb_full[b], ph, p, 24);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            const MvDesc &d = S.mv[b];
+            const MvDesc &d = M.mv[b];
             if (d.d == 2) break;
             const int w = d.c, nv = w >> 3, nrow = d.n;
             const uint32_t src = smem_u32(stages + b * kMvBuf);
@@ -1110,7 +1122,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
             tc_fence_after();
             const unsigned long long te0 = trace_now(p);
             const int rows_valid = ti.nrows - q * 32;          // rows of this warp's quadrant that exist
-            const uint32_t epi_stage = smem_u32(stages + kStages * kStageBytes) + (uint32_t)q * 2048u;   // this warp's staging
+            const uint32_t epi_stage = smem_u32(stages + kStages * kStageBytes) + (uint32_t)q * 4096u;   // this warp's staging (2 x 2 KB)
             bool acc_released = false;
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)ps.acc * 256u;
             if (ti.type == 3) {
@@ -1120,7 +1132,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                 // each up warp (q = 2, 3) writes into its OWN 2 KB staging region, [32][16] fp32, and gate
                 // warp q - 2 reads it; a warp's region is never written by anybody else, so a warp that
                 // is still busy with the previous tile cannot be overrun
-                const uint32_t xs = smem_u32(stages + kStages * kStageBytes) + (uint32_t)(2 + (q & 1)) * 2048u;
+                const uint32_t xs = smem_u32(stages + kStages * kStageBytes) + (uint32_t)(2 + (q & 1)) * 4096u;
                 const int col = ti.n * kTN0 + (int)rank * 64 + (q & 1) * 32 + lane;      // this thread's h-column
                 const int nch = (ti.nrows + 15) >> 4;
                 for (int c = 0; c < nch && !dead; ++c) {
