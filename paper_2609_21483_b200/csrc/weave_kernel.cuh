@@ -10,7 +10,8 @@
 //                         two neighbouring CTAs (a cluster of 2) share a 256-row tile: a scheduler
 //                         warp claims tiles and waits for their inputs, TMA producers feed a
 //                         6-stage smem ring, one thread issues tcgen05.mma.cta_group::2 into TMEM,
-//                         four epilogue warps per CTA drain it through a staged, coalesced store
+//                         four epilogue warps per CTA drain it through a staged, coalesced store,
+//                         and a releasing warp makes the tiles' arrivals on the ready counters
 //   phase C  (every CTA once it has nothing else)  combine tiles, chunk by chunk as the chunk's
 //                         gemm1 tiles complete
 //
@@ -41,6 +42,8 @@ constexpr int kMaxSeg = 1024;     // (chunk, expert) segments: K * (E+S) <= 1024
 constexpr int kTinfo = 4;        // tile-descriptor ring between the producer and its consumers
 constexpr int kTmemCols = 512;
 constexpr int kEpiWarps = 4;     // warps 4..7
+constexpr int kRel = 3;          // mailbox ring between the epilogue warps and the releasing warp (warp 3)
+constexpr unsigned kRelEnd = 0xFFFFFFFFu;
 constexpr int kPairGroup = 8;    // 256-row pair tiles (= 16 m-blocks) kept L2-resident while all n-tiles pass
 
 constexpr int kErrNonFinite = -5;
@@ -144,6 +147,9 @@ struct SmemTail {
     uint64_t dv_full[kStages], dv_empty[kStages];   // dispatch: loader -> storer ring over the stage buffers
     uint64_t cb_full[kStages], cb_empty[kStages];   // combine: loader -> reducing warps
     uint64_t xg_full, xg_empty;                     // swapped gemm0 epilogue: up warps -> gate warps
+    uint64_t rel_full[kRel], rel_empty[kRel];       // epilogue warps -> releasing warp: a tile's stores are issued
+    unsigned *rel_flag[kRel];                       // the ready counter that tile arrives on, and by how much
+    unsigned rel_cnt[kRel];
     TileInfo ti[kTinfo];
     uint32_t tmem_base;
     int bcast[3];
@@ -869,6 +875,8 @@ struct PipeState {     // per-role ring positions; they persist across the tiles
     __device__ __forceinline__ void next_stage() { if (++stage == kStages) { stage = 0; stage_phase ^= 1u; } }
     __device__ __forceinline__ void next_acc() { if (++acc == 2) { acc = 0; acc_phase ^= 1u; } }
     __device__ __forceinline__ void next_slot() { if (++slot == kTinfo) { slot = 0; slot_phase ^= 1u; } }
+    int rel = 0;    uint32_t rel_phase = 0;
+    __device__ __forceinline__ void next_rel() { if (++rel == kRel) { rel = 0; rel_phase ^= 1u; } }
 };
 
 __device__ __forceinline__ float silu_mul(float g, float u)
@@ -1107,6 +1115,24 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
         const int q = warp & 3;                      // TMEM lane quadrant this warp may read
         bool dead = false;
         uint32_t xg_phase = 0;
+        // A release at GPU scope waits until the thread's stores are performed, ~2 us for a tile's
+        // worth.  The epilogue warps do not wait: once a tile's stores are issued they tell warp 3,
+        // through a shared-memory barrier (which orders their stores before whatever warp 3 does
+        // next), which counter the tile arrives on, and go on to the next tile; warp 3 does the
+        // release.  Warp q = 0 fills the mailbox, all four warps arrive on it.
+        auto post = [&](unsigned *flag, unsigned cnt) -> bool {
+            bool ok = true;
+            if (lane == 0) {
+                if (q == 0) {
+                    ok = mbar_wait(&S.rel_empty[ps.rel], ps.rel_phase ^ 1u, p, 56);
+                    S.rel_flag[ps.rel] = flag;
+                    S.rel_cnt[ps.rel] = cnt;
+                }
+                mbar_arrive(&S.rel_full[ps.rel]);
+            }
+            ps.next_rel();
+            return !__any_sync(0xffffffffu, !ok);
+        };
         while (!dead) {
             if (!mbar_wait_cluster(&S.ti_full[ps.slot], ps.slot_phase, p, 50)) { dead = true; }
             dead = __any_sync(0xffffffffu, dead);
@@ -1115,7 +1141,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(mapa_u32(smem_u32(&S.ti_empty[ps.slot]), 0u));
             ps.next_slot();
-            if (ti.type == 2) break;
+            if (ti.type == 2) { post(nullptr, kRelEnd); break; }
             if (!mbar_wait(&S.tmem_full[ps.acc], ps.acc_phase, p, 51)) { dead = true; }
             dead = __any_sync(0xffffffffu, dead);
             if (dead) break;
@@ -1272,14 +1298,31 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
             __syncwarp();
             if (lane == 0) {
                 if (!acc_released) mbar_arrive_cluster(mapa_u32(smem_u32(&S.tmem_empty[ps.acc]), 0u));
-                // a swapped gemm0 tile is stored by the two gate warps of each CTA (4 arrivals per
-                // m-block and n-tile, like a regular tile); a swapped gemm1 tile by all 8 warps
-                if (ti.type == 0 || (ti.type == 3 && q < 2)) red_release_add_u32(&p.h_ready[ti.mb], 1u);
-                else if (ti.type == 1 || ti.type == 4) red_release_add_u32(&p.ctl->y_done[ti.chunk], 1u);
                 if (q == 0) trace_ev(p, S, kEvGemmEpi, (unsigned)(ti.mb & 0xFFFFFF), te0, trace_now(p),
                                      (unsigned)(ti.type << 16 | (int)min(65535ull, te1 - te0)));
             }
+            // a swapped gemm0 tile is stored by the two gate warps of each CTA (4 arrivals per m-block
+            // and n-tile over the pair, like a regular tile); a swapped gemm1 tile by all 8 warps
+            const bool g0 = ti.type == 0 || ti.type == 3;
+            if (!post(g0 ? &p.h_ready[ti.mb] : &p.ctl->y_done[ti.chunk], ti.type == 3 ? 2u : (unsigned)kEpiWarps)) dead = true;
             ps.next_acc();
+        }
+    } else if (warp == 3) {
+        // ---------------- releasing warp (both CTAs): makes the tiles' arrivals on the ready counters
+        int rs = 0;
+        uint32_t rph = 0;
+        while (true) {
+            if (!mbar_wait(&S.rel_full[rs], rph, p, 57)) break;
+            unsigned *flag = S.rel_flag[rs];
+            const unsigned cnt = S.rel_cnt[rs];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&S.rel_empty[rs]);
+            if (cnt == kRelEnd) break;
+            if (lane == 0) {
+                fence_proxy_async();
+                red_release_add_u32(flag, cnt);
+            }
+            if (++rs == kRel) { rs = 0; rph ^= 1u; }
         }
     }
     tc_fence_before();
@@ -1322,6 +1365,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
             mbar_init(&S.cb_full[i], 1); mbar_init(&S.cb_empty[i], kCombWarps);
         }
         mbar_init(&S.xg_full, 2); mbar_init(&S.xg_empty, 2);
+        for (int i = 0; i < kRel; ++i) { mbar_init(&S.rel_full[i], kEpiWarps); mbar_init(&S.rel_empty[i], 1); }
         fence_mbar_init();
         tma_prefetch_desc(&tm.xe); tma_prefetch_desc(&tm.wgu); tma_prefetch_desc(&tm.h); tma_prefetch_desc(&tm.wd);
         tma_prefetch_desc(&tm.wgu64);
