@@ -998,6 +998,10 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                         if (ok && two) ok = flag_wait_ge(&p.h_ready[tp.mb], need, p, 32);
                     }
                     if (!ok) break;
+                    // the tile's input rows may have been written with ordinary stores on other SMs and
+                    // are read by TMA next: the cross-proxy fence sits here, after the acquire and before
+                    // the hand-over to the producers, off their critical path
+                    fence_proxy_async();
                     trace_ev(p, S, kEvGemmLoad, (unsigned)g, tp0, trace_now(p), 0u);
                 }
                 mbar_arrive(&S.ti_full[ps.slot]);
@@ -1017,12 +1021,11 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
             if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
             const TileInfo ti = S.ti[ps.slot];
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(mapa_u32(smem_u32(&S.ti_empty[ps.slot]), 0u));
+            if (lane == 0) mbar_arrive_remote(mapa_u32(smem_u32(&S.ti_empty[ps.slot]), 0u));
             ps.next_slot();
             if (ti.type == 2) break;
             bool dead_l = false;
             if (lane == 0) {
-                fence_proxy_async();     // rows written with ordinary stores elsewhere, read by TMA here
                 const CUtensorMap *tma_a, *tma_b;
                 int arow, brow, arow2 = -1;
                 // swapped tiles: rows per CTA on the N axis (the MMA's N, a multiple of 16, split in two)
@@ -1139,7 +1142,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
             if (dead) break;
             const TileInfo ti = S.ti[ps.slot];
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(mapa_u32(smem_u32(&S.ti_empty[ps.slot]), 0u));
+            if (lane == 0) mbar_arrive_remote(mapa_u32(smem_u32(&S.ti_empty[ps.slot]), 0u));
             ps.next_slot();
             if (ti.type == 2) { post(nullptr, kRelEnd); break; }
             if (!mbar_wait(&S.tmem_full[ps.acc], ps.acc_phase, p, 51)) { dead = true; }
@@ -1243,7 +1246,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                         } else {
                             tc_fence_before();
                             __syncwarp();
-                            if (lane == 0) mbar_arrive_cluster(mapa_u32(smem_u32(&S.tmem_empty[ps.acc]), 0u));
+                            if (lane == 0) mbar_arrive_remote(mapa_u32(smem_u32(&S.tmem_empty[ps.acc]), 0u));
                             acc_released = true;
                         }
 #pragma unroll
@@ -1273,7 +1276,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                             if (c + 2 >= nb && !acc_released) {      // every load of the tile has landed
                                 tc_fence_before();
                                 __syncwarp();
-                                if (lane == 0) mbar_arrive_cluster(mapa_u32(smem_u32(&S.tmem_empty[ps.acc]), 0u));
+                                if (lane == 0) mbar_arrive_remote(mapa_u32(smem_u32(&S.tmem_empty[ps.acc]), 0u));
                                 acc_released = true;
                             }
 #pragma unroll
@@ -1294,10 +1297,9 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
             // by TMA (gemm1) or by ordinary loads (combine) on other SMs once the counter says so
             const unsigned long long te1 = trace_now(p);
             tc_fence_before();
-            fence_proxy_async();
             __syncwarp();
             if (lane == 0) {
-                if (!acc_released) mbar_arrive_cluster(mapa_u32(smem_u32(&S.tmem_empty[ps.acc]), 0u));
+                if (!acc_released) mbar_arrive_remote(mapa_u32(smem_u32(&S.tmem_empty[ps.acc]), 0u));
                 if (q == 0) trace_ev(p, S, kEvGemmEpi, (unsigned)(ti.mb & 0xFFFFFF), te0, trace_now(p),
                                      (unsigned)(ti.type << 16 | (int)min(65535ull, te1 - te0)));
             }

@@ -315,6 +315,14 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
+// Arrival on a barrier of the pair's other CTA with the default (CTA-scope) release: enough where the
+// arriving thread hands back something it has finished reading (an accumulator, a descriptor slot).
+// The cluster-scope release of mbar_arrive_cluster also waits until the thread's earlier global
+// stores are visible cluster-wide, about a thousand cycles behind an epilogue's stores.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 // acquire at cluster scope: the data guarded by the barrier may have been written by the peer CTA
 __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t *bar, uint32_t parity)
 {
