@@ -33,7 +33,7 @@ DEFAULT_CONFIG = "c2_mixtral"
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the megakernel, from the ncu
 # captures summarised under profiles/ (one capture per workload; None = not captured)
-NCU_DRAM_BYTES_PER_LAUNCH = {"c2_mixtral": 4.053e9, "c3_qwen3_30b": 2.586e9}
+NCU_DRAM_BYTES_PER_LAUNCH = {"c2_mixtral": 4.151e9, "c3_qwen3_30b": 2.586e9}
 
 
 def load_peaks():
