@@ -321,14 +321,16 @@ def run_ours(args):
 
     ablation = {}
     if rank == 0 and not args.no_ablation and world == 1:
-        # the three schedules take turns (round robin), so that clock / power drift over the run
-        # hits them alike
+        # the three schedules take turns (round robin, the order rotating from round to round), so
+        # that clock / power drift over the run and whatever the previous schedule left in L2 hit
+        # them alike
         n_abl, rounds = max(2, min(args.steps, 5)), 3
         tot = {"auto": 0.0, "fixed": 0.0, "serial": 0.0}
-        for _ in range(rounds):
-            for name in tot:
+        names = list(tot)
+        for r in range(rounds):
+            for name in names[r % 3:] + names[:r % 3]:
                 moe.set_schedule(*sched[name])
-                tot[name] += timed(step_dev, n_abl, 1)
+                tot[name] += timed(step_dev, n_abl, 2)
         for name, s in tot.items():
             ablation[name + "_us_per_layer"] = s / (n_abl * rounds) / L * 1e6
         ablation["fixed_c"] = fixed_c
