@@ -40,7 +40,7 @@ enum {
     WEAVE_ERR_TIMEOUT = -6             /* device status: a bounded in-kernel wait expired              */
 };
 
-/* Scheduling modes (the paper's ablation, Section 5.5):
+/* Scheduling modes (the paper's ablation, Section 5.6):
  *   AUTO   - full method: the cost model of Section 3.3 (Eq. 15-16) picks the number of movement
  *            SMs c and the chunk count K from the routing result, Eq. 11-14 give the steal count.
  *   FIXED  - the given c, K and steal count are used as they are ("w/o T" when K = 1, steal = 0).
@@ -107,7 +107,7 @@ int weave_moe_host_wait(weave_moe_t h);
 /* Releases host state.  Does not touch device memory. */
 int weave_moe_destroy(weave_moe_t h);
 
-/* ---- scheduling surface (Section 3; ablation of Section 5.5) -------------------------------- */
+/* ---- scheduling surface (Section 3; ablation of Section 5.6) -------------------------------- */
 
 /* mode: WEAVE_SCHED_*.  For FIXED: c = number of movement SMs (rounded up to whole SM pairs and
  * clamped to [2, n_sm-2]), K = chunk count in {1,2,4,8} (lowered until K*(E+S) <= 1024), steal =
@@ -201,7 +201,7 @@ int weave_moe_debug_withhold_flag(weave_moe_t h, int m_block);
 int weave_moe_set_trace(weave_moe_t h, void *buf, int events_per_cta);
 
 /* HOST-ONLY (no GPU needed, no handle): the order in which the kernel's GEMM schedulers claim pair
- * tiles (Section 4: tile queues "in chunk-pipeline DAG order"), for `num_chunks` chunks of
+ * tiles (Section 4: the queues follow the dependency order of the chunk pipeline), for `num_chunks` chunks of
  * `num_segments` expert segments whose row counts are rows[chunk * num_segments + expert], n-tile
  * counts nt0 (gemm0) and nt1 (gemm1).  Writes up to max_tiles records of
  * 6 ints {type (0 gemm0, 1 gemm1, +3 when the operands are swapped), leader m-block, peer m-block

@@ -1,8 +1,8 @@
 """Calibration of the cost model's hardware tables on the GPU at hand, and the (c, K) grid sweep.
 
-The paper's cost model takes "calibrated communication bandwidth and compute throughput curves as
-functions of SM count" (Section 3, Figure 7), an overlap ratio alpha (Section 3.1) and a chunking
-efficiency eff_chunk(K) (Section 3.2.1, Figure 9a).  This module measures them for one layer shape
+The paper's cost model is fed measured hardware tables: movement bandwidth and GEMM throughput, each
+as a function of the number of SMs given to it (Section 3, Figures 4 and 7), an overlap ratio alpha
+(Section 3.1) and a chunking efficiency eff_chunk(K) (Section 3.2.1, Figure 9a).  This module measures them for one layer shape
 from the kernel's own timeline:
 
   BW(c)        movement bytes of dispatch / time the c movement SMs needed for it, while the other
@@ -14,7 +14,7 @@ from the kernel's own timeline:
   alpha        1 - tail * BW(c) / W_combine, tail = time from the last GEMM tile to the kernel end
 
 and can sweep the whole (c, K) grid to compare the model's pick with the measured optimum
-(Section 5.4's accuracy experiment).
+(Section 5.5's accuracy experiment).
 
     python -m paper_2609_21483_b200.calibrate --config c3_qwen3_30b [--grid]
 """

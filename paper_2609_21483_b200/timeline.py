@@ -1,9 +1,9 @@
 """Utilisation report from the kernel's own timeline.
 
-The paper profiles the layer "from the end of routing to the end of combine" and reports SM
-activity, link utilisation, tensor-core activity and an overlap ratio: the fraction of that window
-during which data movement and tensor-core work are both under way (Section 5.3, Figure 11; the
-per-SM timeline of Figure 6).  On one GPU the movement is the dispatch and combine traffic through
+The paper's profiling window opens when routing is done and closes when the last combine is; over it
+the paper reports SM activity, link utilisation, tensor-core activity and an overlap ratio: the share
+of the window in which data movement and tensor-core work are both under way (Section 5.4, Figure 11;
+Figure 8 draws the SMs' roles over time).  On one GPU the movement is the dispatch and combine traffic through
 HBM.  The kernel records one event per tile and per CTA (weave_moe_set_trace); this module turns
 the records into the same quantities:
 

@@ -88,3 +88,6 @@ def test_table1_bench_configs_cover_every_row_and_sequence_length():
         for T in (2048, 4096, 8192):
             c = wl.CONFIGS[f"t1_{short}_T{T}"]
             assert (c.E, c.k, c.H, c.I) == t1[row] and c.T == T
+    # the scheduler ablation's two shapes also exist at 16k tokens (Section 5.6)
+    for short in ("qwen3_30b", "qwen35_35b"):
+        assert wl.CONFIGS[f"t1_{short}_T16384"].T == 16384
