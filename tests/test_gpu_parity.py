@@ -257,6 +257,28 @@ def test_handle_reuse_smaller_batches_and_run_to_run_bits():
     moe.close()
 
 
+def test_short_tiles_back_to_back_launches_keep_their_bits():
+    """gemm1 tiles of four k-steps and gemm0 tiles of eight: epilogues, ready-counter arrivals (made by
+    the releasing warp from a three-slot mailbox) and descriptor hand-overs follow each other as fast as
+    they can.  40 launches without a host synchronisation in between, three schedules: every output
+    must carry the bits of the first one, which is checked against the oracle."""
+    cfg = _small("short_tiles", 4096, 512, 256, 64, 4, zipf=1.0, cfg_id=93)
+    inp = wl.make_inputs(cfg)
+    dev = to_dev(inp)
+    moe, out0, _ = run_case(cfg, n_sample=32, inp=inp, dev_tensors=dev)
+    bits = out0.view(torch.int16).clone()
+    for s in [(pk.SCHED_AUTO, 0, 1, 0), (pk.SCHED_FIXED, 16, 2, 8), (pk.SCHED_SERIAL, 0, 1, 0)]:
+        moe.set_schedule(*s)
+        outs = []
+        for rep in range(40):
+            outs.append(moe.forward(dev[0], dev[1]).view(torch.int16).clone())
+        torch.cuda.synchronize()
+        moe.check()
+        for rep, o in enumerate(outs):
+            assert torch.equal(o, bits), f"schedule {s}, launch {rep}: output bits changed"
+    moe.close()
+
+
 def test_layers_captured_in_a_cuda_graph_replay_bit_for_bit():
     """forward() enqueues one (cooperative) kernel and nothing else, so a stack of layers can be
     captured into a CUDA graph; the replay gives the bits of the direct calls."""
