@@ -257,6 +257,30 @@ __device__ __forceinline__ bool flag_wait_ge(const unsigned *flag, unsigned targ
 }
 
 // All CTAs are co-resident (cooperative launch); arrivals accumulate over the barriers of a launch.
+// Three exclusive scans in one pass: v = a | b << 24 | c << 48 with a, b < 2^24 and c < 2^16 in total.
+__device__ __forceinline__ unsigned long long block_excl_scan_packed(unsigned long long v, SmemTail &S, unsigned long long &total)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned long long inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long n = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += n;
+    }
+    __syncthreads();
+    if (lane == 31) { S.red_i[warp][0] = (int)(unsigned)inc; S.red_i[warp][1] = (int)(unsigned)(inc >> 32); }
+    __syncthreads();
+    unsigned long long wbase = 0, tot = 0;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) {
+        const unsigned long long sw = (unsigned long long)(unsigned)S.red_i[w][0] | ((unsigned long long)(unsigned)S.red_i[w][1] << 32);
+        if (w < warp) wbase += sw;
+        tot += sw;
+    }
+    total = tot;
+    return wbase + inc - v;
+}
+
 __device__ __forceinline__ bool grid_barrier(const KParams &p, SmemTail &S, unsigned target, int where)
 {
     __syncthreads();
@@ -436,12 +460,11 @@ __device__ __forceinline__ void route_block_quads(const KParams &p, int b, const
 // Eq. 15 for one candidate, in the same fp32 operation order as the CPU restatement:
 // T_comp = W_comp / (TFLOPS(N-c) * eff_chunk(K))  (Eq. 9),  T_comm = (W_disp + W_comb) / BW(c)  (Eq. 5),
 // T_tail = (1 - alpha) * W_comb / (BW(c) * K)  (Eq. 10),  T_total = max(T_comp + T_tail, T_comm).
-__device__ __forceinline__ float model_t_total(const KParams &p, int n_sm, int c, int ki, float w_comp, float w_disp,
+// bw = BW(c), tf = TFLOPS(N - c): the candidate's two table entries
+__device__ __forceinline__ float model_t_total(const KParams &p, float bw, float tf, int ki, float w_comp, float w_disp,
                                                float w_comb)
 {
     const float Kf = (float)(1 << ki);
-    const float bw = p.bw[c];
-    const float tf = p.tf[n_sm - c];
     const float t_comp = __fdiv_rn(w_comp, __fmul_rn(tf, p.eff[ki]));
     const float t_comm = __fdiv_rn(__fadd_rn(w_disp, w_comb), bw);
     const float t_tail = __fmul_rn(__fsub_rn(1.0f, p.alpha), __fdiv_rn(w_comb, __fmul_rn(bw, Kf)));
@@ -449,12 +472,12 @@ __device__ __forceinline__ float model_t_total(const KParams &p, int n_sm, int c
 }
 
 // Eq. 11-14 with W_tile = W_comp / n_tiles (the mean GEMM tile of this layer).
-__device__ __forceinline__ int model_n_steal(const KParams &p, int n_sm, int c, float w_comp, float w_disp,
+__device__ __forceinline__ int model_n_steal(int n_sm, float bw, float tf, float w_comp, float w_disp,
                                              float w_comb, int n_tiles)
 {
     if (n_tiles <= 0) return 0;
-    const float t_comm = __fdiv_rn(__fadd_rn(w_disp, w_comb), p.bw[c]);
-    const float w_partial = __fmul_rn(t_comm, p.tf[n_sm - c]);
+    const float t_comm = __fdiv_rn(__fadd_rn(w_disp, w_comb), bw);
+    const float w_partial = __fmul_rn(t_comm, tf);
     const float w_steal = fmaxf(0.0f, __fsub_rn(w_comp, w_partial));
     const float w_tile = __fdiv_rn(w_comp, (float)n_tiles);
     if (!(w_tile > 0.0f)) return 0;
@@ -1426,6 +1449,12 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
         }
         __syncthreads();
     }
+    // The cost tables do not depend on the routing: this thread's candidate (c, K) asks for its two
+    // entries before the barrier, so that their latency is spent waiting there.
+    const int cm_ki = tid & 3, cm_c = p.c_min + (tid >> 2) * p.c_step;
+    const bool cm_ok = p.mode == kModeAuto && cm_c >= 2 && cm_c <= p.c_max && cm_c <= n_sm - 2 && (EE << cm_ki) <= kMaxSeg;
+    float cm_bw = 0.f, cm_tf = 0.f;
+    if (cm_ok) { cm_bw = p.bw[cm_c]; cm_tf = p.tf[n_sm - cm_c]; }
     const unsigned long long tk1 = trace_now(p);
     bool alive = grid_barrier(p, S, (unsigned)n_sm, 1);
     const unsigned long long tk2 = trace_now(p);
@@ -1448,34 +1477,6 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
         p.offsets[tid] = off;
         if (tid == 0) p.offsets[EE] = total_rows;
     }
-    // pair tiles (256 rows) of the layer for each candidate K (a segment = one expert's rows inside
-    // one chunk; its last pair tile may be half empty)
-    int mbk[4];
-#pragma unroll
-    for (int ki = 0; ki < 4; ++ki) {
-        const int K = 1 << ki, g = kFine / K;
-        int acc = 0;
-        for (int j = 0; j < K; ++j) {
-            int rows = 0;
-#pragma unroll
-            for (int f = 0; f < kFine; ++f) if (f / g == j) rows += cf[f];
-            acc += (rows + 2 * kBM - 1) / (2 * kBM);
-        }
-        mbk[ki] = acc;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mbk[ki] += __shfl_xor_sync(0xffffffffu, mbk[ki], o);
-    }
-    if (lane == 0) { S.red_i[warp][0] = mbk[0]; S.red_i[warp][1] = mbk[1]; S.red_i[warp][2] = mbk[2]; S.red_i[warp][3] = mbk[3]; }
-    __syncthreads();
-    int n_tiles_k[4];
-#pragma unroll
-    for (int ki = 0; ki < 4; ++ki) {
-        int s = 0;
-        for (int w = 0; w < kThreads / 32; ++w) s += S.red_i[w][ki];
-        n_tiles_k[ki] = s * (p.nt0 + p.nt1);
-    }
-    __syncthreads();     // red_i is reused by the arg-min below
-
     const int P = p.T * (p.k + p.S);
     const unsigned ep_xl = alive ? __ldcg(&p.ctl->x_local) : 0u, ep_xi = alive ? __ldcg(&p.ctl->x_in) : 0u,
                    ep_xu = alive ? __ldcg(&p.ctl->x_in_uniq) : 0u;
@@ -1497,11 +1498,8 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
             w_disp = __fmul_rn((float)(p.T + P), B);
             w_comb = __fmul_rn((float)(P + p.T), B);
         }
-        const int ci = tid >> 2, ki = tid & 3;
-        const int cc = p.c_min + ci * p.c_step;
         float t = __int_as_float(0x7f800000);
-        if (cc >= 2 && cc <= p.c_max && cc <= n_sm - 2 && (EE << ki) <= kMaxSeg)
-            t = model_t_total(p, n_sm, cc, ki, w_comp, w_disp, w_comb);
+        if (cm_ok) t = model_t_total(p, cm_bw, cm_tf, cm_ki, w_comp, w_disp, w_comb);
         int bi = tid;       // candidate order = (c ascending, K ascending): ties go to the smaller index
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
@@ -1520,7 +1518,29 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
         plan_c = p.c_min + (bi >> 2) * p.c_step;
         plan_ki = bi & 3;
         plan_t = t;
-        plan_steal = model_n_steal(p, n_sm, plan_c, w_comp, w_disp, w_comb, n_tiles_k[plan_ki]);   // per CTA pair
+        // the winner hands its two table entries to everybody; the pair tiles (256 rows) of the layer at
+        // the chosen K are counted meanwhile (a segment = one expert's rows inside one chunk; its last
+        // pair tile may be half empty)
+        if (tid == bi) { S.red_i[0][1] = __float_as_int(cm_bw); S.red_i[0][2] = __float_as_int(cm_tf); }
+        {
+            const int Kc = 1 << plan_ki, g = kFine / Kc;
+            int acc = 0;
+            for (int j = 0; j < Kc; ++j) {
+                int rows = 0;
+#pragma unroll
+                for (int f = 0; f < kFine; ++f) if (f / g == j) rows += cf[f];
+                acc += (rows + 2 * kBM - 1) / (2 * kBM);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+            if (lane == 0) S.red_i[warp][3] = acc;
+        }
+        __syncthreads();
+        int n_tiles = 0;
+        for (int w = 0; w < kThreads / 32; ++w) n_tiles += S.red_i[w][3];
+        n_tiles *= p.nt0 + p.nt1;
+        plan_steal = model_n_steal(n_sm, __int_as_float(S.red_i[0][1]), __int_as_float(S.red_i[0][2]), w_comp, w_disp, w_comb,
+                                   n_tiles);   // per CTA pair
         __syncthreads();
     } else if (p.mode == kModeFixed) {
         plan_c = max(2, min((p.fixed_c + 1) & ~1, n_sm - 2));     // whole CTA pairs
@@ -1542,10 +1562,12 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
 #pragma unroll
             for (int f = 0; f < kFine; ++f) if (f / g == j) rows += cf[f];
             const int mbs = (rows + kBM - 1) / kBM;
-            int tot, ptot, nodd;
-            const int ex = block_excl_scan(mbs, S, tot);
-            const int pex = block_excl_scan((mbs + 1) >> 1, S, ptot);
-            (void)block_excl_scan(mbs & 1, S, nodd);
+            // m-blocks, pair tiles and unpaired m-blocks of the experts before this one: one packed scan
+            unsigned long long tot3;
+            const unsigned long long ex3 = block_excl_scan_packed((unsigned long long)mbs | ((unsigned long long)((mbs + 1) >> 1) << 24) |
+                                                                      ((unsigned long long)(mbs & 1) << 48), S, tot3);
+            const int ex = (int)(ex3 & 0xFFFFFFull), pex = (int)((ex3 >> 24) & 0xFFFFFFull);
+            const int tot = (int)(tot3 & 0xFFFFFFull), ptot = (int)((tot3 >> 24) & 0xFFFFFFull), nodd = (int)(tot3 >> 48);
             if (tid < EE) {
                 S.seg_mb0[j * EE + tid] = mb_base + ex;
                 S.seg_pt0[j * EE + tid] = pt_base + pex;
