@@ -20,7 +20,7 @@
  *   - S optional shared experts process every token with weight 1.
  *
  * Arithmetic: fp32 on the bf16 inputs, nothing rounded in between; acc_double=1
- * switches every accumulation to fp64 (a cross-check, not the judge).
+ * switches every accumulation to fp64 (a cross-check only; the fp32 path is what the GPU is compared with).
  * Parity pins: tests/test_oracle_*.py (brute force, closed forms, library
  * routines, invariants).
  */
