@@ -96,7 +96,8 @@ def test_c5_qwen3_235b_shaped_two_layers_sampled():
     moe.close()
 
 
-@pytest.mark.parametrize("name", ["t1_dsv3_T2048", "t1_phi35_T2048", "t1_qwen35_35b_T2048", "t1_dsv2_T2048"])
+@pytest.mark.parametrize("name", ["t1_dsv3_T2048", "t1_phi35_T2048", "t1_qwen35_35b_T2048", "t1_dsv2_T2048",
+                                  "t1_qwen35_35b_T16384"])
 def test_remaining_table1_shapes_sampled(name):
     """The Table 1 rows that are not among the five configs of record (256 experts, H = 7168 / 5120,
     I = 512 ... 6400), mildly skewed routing, four sampled tokens each."""
