@@ -5,17 +5,24 @@
 
 A step is one pass of the whole hot path (routing, dispatch, grouped SwiGLU GEMMs, combine: one
 kernel launch per layer) over one batch of seeded synthetic input.  The default workload is the
-Mixtral-8x7B-shaped prefill layer (T=4096, H=4096, I=14336, E=8, top-2).  One JSON line is
-printed by rank 0.  With --gpus N > 1 (launched by torch.distributed.run) every rank runs an
-independent replica of the layer on its own GPU (the path has no cross-GPU exchange step on one
-node: "replicas only"); the value is the number of tokens all ranks processed divided by the
-slowest rank's device time.
+largest single-GPU configuration: a stack of 24 Qwen3-235B-A22B-shaped layers (T=16384, H=4096,
+I=1536, E=128, top-8, a fresh routing skew per layer), one step = 24 launches.  One JSON line is
+printed by rank 0; with the default workload it also carries a `per_config` list with the other
+configurations of record (Mixtral-shaped, Qwen3-30B-shaped, DSv2-Lite-shaped decode batches, the
+tiny layer), each with its burst-window and sustained-run roofline fractions and the scheduler
+ablation.
+
+With --gpus N > 1 the script starts N ranks of itself under torch.distributed.run (or runs as one of
+them when it was started that way): every rank runs an independent replica of the layer on its own
+GPU (the path has no cross-GPU exchange step on one node: "replicas only"); the value is the number
+of tokens all ranks processed divided by the slowest rank's device time.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import subprocess
 import sys
 import threading
@@ -29,15 +36,18 @@ import numpy as np
 
 METRIC = "moe_layer_tokens_per_s"
 UNIT = "tokens/s"
-DEFAULT_CONFIG = "c2_mixtral"
+DEFAULT_CONFIG = "c5_qwen3_235b"
+PER_CONFIG = ["c2_mixtral", "c3_qwen3_30b", "c4_dsv2lite_T64", "c4_dsv2lite_T256", "c4_dsv2lite_T1024", "c1_tiny"]
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the megakernel, from the ncu
-# captures summarised under profiles/ (one capture per workload; None = not captured)
+# captures summarised under profiles/ (one capture per workload; None = not captured).  The
+# Qwen3-235B-shaped layer is too large to capture whole: its figure is the capture of a quarter of
+# the layer (T = 4096, same shape and skew) scaled by the units processed, as profiles/ explains.
 NCU_DRAM_BYTES_PER_LAUNCH = {"c2_mixtral": 4.151e9, "c3_qwen3_30b": 2.586e9}
 
 
 def load_peaks():
-    """Measured roofline denominators of this machine's B200s, else the documented fallback."""
+    """Measured roofline denominators (MEASURED_PEAKS.json beside this file), else the documented fallback."""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
         with open(path) as f:
@@ -63,6 +73,22 @@ def layer_work(cfg, active_experts=None):
            + T * 2.0 * H)
     return {"flops": flops, "bytes": weights + act, "weights_bytes": weights, "act_bytes": act,
             "movement_bytes": (T + P) * 2.0 * H + (P + T) * 2.0 * H}
+
+
+def roofline_of(work, layer_s, peaks, window):
+    """Roofline entry of one layer time.  window = "burst" (a timed region well under half a second that
+    starts from idle clocks: compared with the burst bf16 peak) or "sustained" (a back-to-back run of
+    seconds under the power cap: compared with the sustained bf16 peak).  The bound is decided with the
+    peak of the same window; the HBM copy bandwidth has one measured figure."""
+    tf_peak = peaks["bf16_tflops_sustained"] if window == "sustained" else peaks["bf16_tflops"]
+    t_flops = work["flops"] / (tf_peak * 1e12)
+    t_bytes = work["bytes"] / (peaks["hbm_gbs"] * 1e9)
+    if t_flops >= t_bytes:
+        bound, achieved, peak, unit = "tensor", work["flops"] / layer_s / 1e12, tf_peak, "TFLOP/s"
+    else:
+        bound, achieved, peak, unit = "hbm", work["bytes"] / layer_s / 1e9, peaks["hbm_gbs"], "GB/s"
+    return {"bound": bound, "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
+            "window": window, "layer_roofline_us": max(t_flops, t_bytes) * 1e6}
 
 
 class ClockSampler:
@@ -140,6 +166,32 @@ def whole_job_throughput(tokens_per_rank_step: int, steps: int, world: int, max_
     return tokens_per_rank_step * steps * world / max_seconds
 
 
+def launch_ranks(n: int, argv) -> int:
+    """Starts n ranks of this script on this node under torch.distributed.run and returns its exit code."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
+def launcher_selftest(args):
+    """The multi-rank plumbing without a GPU: gloo ranks, the slowest rank's time decides, rank 0
+    prints the line.  Used by the CPU tests to exercise `--gpus N` as a user starts it."""
+    import torch.distributed as dist
+    rank, world, _ = dist_env()
+    if world > 1:
+        dist.init_process_group("gloo")
+    sec = aggregate_max(1.0 + rank, world, use_cuda=False)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"launcher_selftest": True, "n_gpus": world, "max_seconds": sec,
+                          "value": whole_job_throughput(4096, args.steps, world, sec)}), flush=True)
+
+
 def host_weights_for(cfg, wl, oracle, logits, toks):
     """Host weight arrays for the oracle in which only the experts the sampled tokens use are filled
     in (zero pages that are never touched cost no memory), so that 20 GB layers stay benchable."""
@@ -175,29 +227,39 @@ def run_reference(args):
     import workloads as wl
     cfg = wl.CONFIGS[args.config]
     oracle.build(); wl.build()
-    x_h, lg_h = wl.make_x(cfg), wl.make_logits(cfg)
+    L = cfg.layers
+    x_h = wl.make_x(cfg)
+    lgs = [wl.make_logits(cfg, l) for l in range(L)]
     probe = wl.stratified_token_sample(cfg.T, 8, seed=99)
-    inp = wl.LayerInputs(cfg, x_h, lg_h, *host_weights_for(cfg, wl, oracle, lg_h, probe))
-    n = args.ref_tokens if args.ref_tokens > 0 else cpu_sample_size(
-        oracle, wl, inp, cfg, max(2.0, min(args.cpu_seconds, 120.0 / max(args.steps + 1, 1))))
+    inp = wl.LayerInputs(cfg, x_h, lgs[0], *host_weights_for(cfg, wl, oracle, lgs[0], probe))
+    # per step and layer: full-T routing plus the sampled tokens' FFN/combine; the whole run is bounded
+    budget = max(2.0, min(args.cpu_seconds, 120.0 / max(args.steps + 1, 1)))
+    n = args.ref_tokens if args.ref_tokens > 0 else max(8, cpu_sample_size(oracle, wl, inp, cfg, budget) // L)
     toks = wl.stratified_token_sample(cfg.T, n, seed=cfg.cfg_id)
-    inp.gate_up, inp.down = host_weights_for(cfg, wl, oracle, lg_h, toks)
+    need_logits = np.concatenate([lg[toks] for lg in lgs])
+    idx, _ = oracle.route(np.ascontiguousarray(need_logits), cfg.k)
+    EE = cfg.E + cfg.S
+    gu = np.zeros((EE, 2 * cfg.I, cfg.H), np.uint16)
+    dn = np.zeros((EE, cfg.H, cfg.I), np.uint16)
+    for e in sorted(set(idx.ravel().tolist()) | set(range(cfg.E, EE))):
+        gu[e], dn[e] = wl.expert_weights(cfg, e)
     for _ in range(max(args.warmup, 0) and 1):
-        oracle.moe_tokens(inp.x, inp.logits, inp.gate_up, inp.down, cfg.k, toks[:1], cfg.S)
+        oracle.moe_tokens(x_h, lgs[0], gu, dn, cfg.k, toks[:1], cfg.S)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle.routing(inp.logits, cfg.k, cfg.S)
-        oracle.moe_tokens(inp.x, inp.logits, inp.gate_up, inp.down, cfg.k, toks, cfg.S)
+        for l in range(L):
+            oracle.routing(lgs[l], cfg.k, cfg.S)
+            oracle.moe_tokens(x_h, lgs[l], gu, dn, cfg.k, toks, cfg.S)
     dt = time.perf_counter() - t0
-    val = len(toks) * args.steps / dt
+    val = len(toks) * L * args.steps / dt
     cores = oracle.num_threads()
-    sample = (f"{len(toks)} stratified tokens of T={cfg.T} per step (full-T routing + per-token FFN/combine), "
-              f"{args.steps} steps, {dt:.1f} s")
+    sample = (f"{len(toks)} stratified tokens of T={cfg.T} per layer x {L} layer(s) per step (full-T routing + "
+              f"per-token FFN/combine), {args.steps} steps, {dt:.1f} s")
     line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "I": cfg.I, "E": cfg.E, "top_k": cfg.k,
-                       "shared": cfg.S},
+                       "shared": cfg.S, "layers": L},
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -206,67 +268,73 @@ def run_reference(args):
 
 # --------------------------------------------------------------------------------------- our arm
 
-def run_ours(args):
-    import torch
-    import workloads as wl
-    import paper_2609_21483_b200 as pk
+class Layer:
+    """Device tensors and the handle of one workload."""
 
-    rank, world, local = dist_env()
-    if args.gpus > 1 and world != args.gpus:
-        raise SystemExit(f"--gpus {args.gpus} needs torch.distributed.run with {args.gpus} ranks (WORLD_SIZE={world})")
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device; there is no CPU path (use --impl reference for the oracle)")
-    torch.cuda.set_device(local)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    pk.load()
+    def __init__(self, cfg, args, weights=None):
+        import torch
+        import workloads as wl
+        import paper_2609_21483_b200 as pk
+        self.cfg, self.pk, self.torch = cfg, pk, torch
+        as_bf16 = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)
+        EE = cfg.E + cfg.S
+        if weights is None:
+            gu = torch.empty((EE, 2 * cfg.I, cfg.H), dtype=torch.bfloat16, device="cuda")
+            dn = torch.empty((EE, cfg.H, cfg.I), dtype=torch.bfloat16, device="cuda")
+            for e in range(EE):      # expert by expert: the host never holds the whole (up to 20 GB) tensor
+                g_e, d_e = wl.expert_weights(cfg, e)
+                gu[e].copy_(as_bf16(g_e))
+                dn[e].copy_(as_bf16(d_e))
+            weights = (gu, dn)
+        self.weights = weights
+        self.x_h = as_bf16(wl.make_x(cfg)).pin_memory()
+        self.x = self.x_h.cuda()
+        self.L = cfg.layers
+        self.logits_h = [torch.from_numpy(wl.make_logits(cfg, l)).pin_memory() for l in range(self.L)]
+        self.logits = [t.cuda() for t in self.logits_h]
+        self.out = torch.empty_like(self.x)
+        self.out_h = [torch.empty_like(self.x_h).pin_memory() for _ in range(2)]
+        self.moe = pk.WeaveMoE(weights[0], weights[1], cfg.E, cfg.k, cfg.S, max_tokens=cfg.T)
+        if args.sms:
+            self.moe.set_sm_count(args.sms)
+        if args.ep > 1:
+            self.moe.set_expert_parallel(args.ep_rank, args.ep)
+        geo = self.moe.geometry()
+        self.fixed_c = max(2, int(round(0.15 * geo["n_sm"])))
+        self.stream = torch.cuda.current_stream()
 
-    cfg = wl.CONFIGS[args.config]
-    wl.build()
-    as_bf16 = lambda a: torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)
-    EE = cfg.E + cfg.S
-    gu = torch.empty((EE, 2 * cfg.I, cfg.H), dtype=torch.bfloat16, device="cuda")
-    dn = torch.empty((EE, cfg.H, cfg.I), dtype=torch.bfloat16, device="cuda")
-    for e in range(EE):      # expert by expert: the host never holds the whole (up to 20 GB) tensor
-        g_e, d_e = wl.expert_weights(cfg, e)
-        gu[e].copy_(as_bf16(g_e))
-        dn[e].copy_(as_bf16(d_e))
-    x_h = as_bf16(wl.make_x(cfg)).pin_memory()
-    x = x_h.cuda()
-    L = cfg.layers
-    logits_h = [torch.from_numpy(wl.make_logits(cfg, l)).pin_memory() for l in range(L)]
-    logits = [t.cuda() for t in logits_h]
-    out = torch.empty_like(x)
-    out_h = torch.empty_like(x_h).pin_memory()
-    moe = pk.WeaveMoE(gu, dn, cfg.E, cfg.k, cfg.S, max_tokens=cfg.T)
-    if args.sms:
-        moe.set_sm_count(args.sms)
-    if args.ep > 1:
-        moe.set_expert_parallel(args.ep_rank, args.ep)
-    stream = torch.cuda.current_stream()
-    sched = {"auto": (pk.SCHED_AUTO, 0, 1, 0), "serial": (pk.SCHED_SERIAL, 0, 1, 0)}
-    geo = moe.geometry()
-    fixed_c = max(2, int(round(0.15 * geo["n_sm"])))
-    sched["fixed"] = (pk.SCHED_FIXED, fixed_c, 1, 0)
+    # the schedules of the ablation (Section 5.6): (mode, c, K, steal), plan kinds, elastic switch
+    def schedules(self):
+        pk = self.pk
+        return {
+            "auto": ((pk.SCHED_AUTO, 0, 1, 0), 7, -1),                    # the model over every plan kind
+            "auto_split": ((pk.SCHED_AUTO, 0, 1, 0), 1, -1),              # the paper's plan kind only
+            "fixed": ((pk.SCHED_FIXED, self.fixed_c, 1, 0), 7, 0),        # static 15 % split, nothing else
+            "fixed_elastic": ((pk.SCHED_FIXED, self.fixed_c, 1, 0), 7, 1),  # ... plus elastic stealing and the first dispatch wave
+            "serial": ((pk.SCHED_SERIAL, 0, 1, 0), 7, -1),                # phases separated by grid barriers
+        }
 
-    def step_dev():
-        for l in range(L):
-            moe.forward(x, logits[l], out)
+    def set(self, name):
+        sched, kinds, elastic = self.schedules()[name]
+        self.moe.set_schedule(*sched)
+        self.moe.set_model_options(kinds, elastic)
 
-    out_h2 = torch.empty_like(x_h).pin_memory()
+    def step_dev(self):
+        for l in range(self.L):
+            self.moe.forward(self.x, self.logits[l], self.out)
 
-    def step_host():
+    def step_host(self):
         # the call a user makes for a stream of batches from host memory: inputs and outputs cross
         # PCIe every layer call; the copies overlap the neighbouring calls' kernels
-        for l in range(L):
-            moe.forward_host_pipelined(x_h, logits_h[l], out_h if l % 2 == 0 else out_h2)
+        for l in range(self.L):
+            self.moe.forward_host_pipelined(self.x_h, self.logits_h[l], self.out_h[l % 2])
 
-    def timed(fn, steps, warmup, host_path=False):
+    def timed(self, fn, steps, warmup, world=1, host_path=False):
+        torch = self.torch
         for _ in range(warmup):
             fn()
         if host_path:
-            moe.host_wait()
+            self.moe.host_wait()
         if world > 1:
             torch.distributed.barrier()
         torch.cuda.synchronize()
@@ -276,34 +344,122 @@ def run_ours(args):
             t0 = time.perf_counter()
             for _ in range(steps):
                 fn()
-            moe.host_wait()
+            self.moe.host_wait()
             torch.cuda.synchronize()
             dt = time.perf_counter() - t0
             if world > 1:
                 torch.distributed.barrier()
             return dt
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ev0.record(stream)
+        ev0.record(self.stream)
         for _ in range(steps):
             fn()
-        ev1.record(stream)
+        ev1.record(self.stream)
         torch.cuda.synchronize()
         if world > 1:
             torch.distributed.barrier()
         return ev0.elapsed_time(ev1) * 1e-3
 
-    moe.set_schedule(*sched[args.sched])
+    def sustained(self, step_s, seconds=2.0, local=0):
+        """Layer time of a back-to-back run of at least `seconds` (after 0.3 s of the same load), with
+        the clocks sampled during it: the figure to hold against the sustained peak."""
+        n_warm = max(1, int(0.3 / step_s))
+        n = max(2, int(np.ceil(seconds / step_s)))
+        for _ in range(n_warm):
+            self.step_dev()
+        sampler = ClockSampler(local)
+        sampler.start()
+        sec = self.timed(self.step_dev, n, 0)
+        clocks = sampler.stop()
+        return sec / n / self.L, sec, clocks
+
+    def ablation(self, step_s, rounds=3):
+        """The schedules take turns (round robin, the order rotating from round to round), so that clock
+        and power drift over the run and whatever the previous schedule left in L2 hit them alike.  The
+        part runs under its power cap and the clock follows the last ~50 ms of load: each measurement is
+        preceded by that much of its own schedule."""
+        names = list(self.schedules())
+        n_abl = max(2, min(5, int(0.25 / step_s) + 1))
+        warm = max(1, min(20, int(0.05 / step_s) + 1))
+        tot = {n: 0.0 for n in names}
+        for r in range(rounds):
+            k = r % len(names)
+            for name in names[k:] + names[:k]:
+                self.set(name)
+                tot[name] += self.timed(self.step_dev, n_abl, warm)
+        res = {n + "_us_per_layer": s / (n_abl * rounds) / self.L * 1e6 for n, s in tot.items()}
+        res["fixed_c"] = self.fixed_c
+        self.set("auto")
+        self.moe.check()
+        return res
+
+    def close(self):
+        self.moe.close()
+
+
+def measure_side_config(name, args, peaks, weights_cache):
+    """One entry of `per_config`: burst-window and sustained layer times with their roofline
+    fractions, the plan, the scheduler ablation."""
+    import torch
+    import workloads as wl
+    cfg = wl.CONFIGS[name]
+    key = (cfg.cfg_id, cfg.H, cfg.I, cfg.E, cfg.S)
+    lay = Layer(cfg, args, weights_cache.get(key))
+    weights_cache.clear()
+    weights_cache[key] = lay.weights
+    lay.set("auto")
+    sec = lay.timed(lay.step_dev, 10, 3)
+    lay.moe.check()
+    step_s = sec / 10
+    plan = lay.moe.plan()
+    work = layer_work(cfg)
+    burst = roofline_of(work, step_s / lay.L, peaks, "burst")
+    sus_layer_s, sus_sec, clocks = lay.sustained(step_s, seconds=args.sustain_seconds, local=args.local)
+    sus = roofline_of(work, sus_layer_s, peaks, "sustained")
+    entry = {"workload": cfg.name, "T": cfg.T, "layer_us": step_s / lay.L * 1e6, "frac": burst["frac"],
+             "bound": burst["bound"], "layer_roofline_us": burst["layer_roofline_us"],
+             "layer_us_sustained": sus_layer_s * 1e6, "frac_sustained": sus["frac"], "bound_sustained": sus["bound"],
+             "sustained_run_s": sus_sec, "sm_mhz_sustained": clocks.get("sm_mhz"), "reasons": clocks.get("reasons"),
+             "plan": plan, "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(cfg.name),
+             "ablation": lay.ablation(step_s) if not args.no_ablation else {}}
+    lay.close()
+    del lay
+    torch.cuda.empty_cache()
+    return entry
+
+
+def run_ours(args):
+    import torch
+    import workloads as wl
+    import paper_2609_21483_b200 as pk
+
+    rank, world, local = dist_env()
+    if args.gpus > 1 and world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus}: started as one of {world} ranks")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path (use --impl reference for the oracle)")
+    torch.cuda.set_device(local)
+    args.local = local
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    pk.load()
+    wl.build()
+
+    cfg = wl.CONFIGS[args.config]
+    lay = Layer(cfg, args)
+    L = lay.L
+    lay.set(args.sched)
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
         time.sleep(0.05)
-    sec = timed(step_dev, args.steps, args.warmup)
-    moe.check()
-    plans = []
-    if rank == 0:
-        plans.append(moe.plan())
+    sec = lay.timed(lay.step_dev, args.steps, args.warmup, world)
+    lay.moe.check()
+    plan = lay.moe.plan() if rank == 0 else None
     sec_max = aggregate_max(sec, world, True)
     clocks = sampler.stop() if rank == 0 else None
+    step_s = sec_max / args.steps
     if rank == 0 and (clocks.get("samples") or 0) < 5:
         # the timed region was too short for nvidia-smi's sampling period: repeat the same steps
         # (untimed) for about half a second with the sampler running, and say so
@@ -311,67 +467,52 @@ def run_ours(args):
         probe.start()
         t_end = time.perf_counter() + 0.6
         while time.perf_counter() < t_end:
-            step_dev()
+            lay.step_dev()
             torch.cuda.synchronize()
         clocks = probe.stop()
         clocks["note"] = "timed region shorter than the sampling period; sampled over an untimed 0.6 s repeat of the same steps"
-    sec_e2e = aggregate_max(timed(step_host, max(1, min(args.steps, 10)), 3, host_path=True), world, True)
     e2e_steps = max(1, min(args.steps, 10))
-    moe.check()
-
-    ablation = {}
-    if rank == 0 and not args.no_ablation and world == 1:
-        # the three schedules take turns (round robin, the order rotating from round to round), so
-        # that clock / power drift over the run and whatever the previous schedule left in L2 hit
-        # them alike
-        n_abl, rounds = max(2, min(args.steps, 5)), 3
-        tot = {"auto": 0.0, "fixed": 0.0, "serial": 0.0}
-        names = list(tot)
-        # the part runs under its power cap and the clock follows the last ~50 ms of load: each
-        # measurement is preceded by that much of its own schedule, not by its predecessor's
-        warm = max(2, min(20, int(0.05 / max(sec / args.steps, 1e-6)) + 1))
-        for r in range(rounds):
-            for name in names[r % 3:] + names[:r % 3]:
-                moe.set_schedule(*sched[name])
-                tot[name] += timed(step_dev, n_abl, warm)
-        for name, s in tot.items():
-            ablation[name + "_us_per_layer"] = s / (n_abl * rounds) / L * 1e6
-        ablation["fixed_c"] = fixed_c
-        moe.set_schedule(*sched[args.sched])
-        moe.check()
-
-    if rank != 0:
-        if world > 1:
-            torch.distributed.destroy_process_group()
-        return
+    sec_e2e = aggregate_max(lay.timed(lay.step_host, e2e_steps, 3, world, host_path=True), world, True)
+    lay.moe.check()
 
     peaks = load_peaks()
     work = layer_work(cfg)
     ep_desc = None
     if args.ep > 1:
         # the rank computes only its own pairs: scale the algorithmic work by its share of the pairs
-        ep_desc = moe.ep_descriptors()
+        ep_desc = lay.moe.ep_descriptors()
         share = (ep_desc["x_local"] + ep_desc["x_in"]) / float(cfg.P)
         work = {k: v * share for k, v in work.items()}
-    layer_s = sec_max / args.steps / L
-    # the burst bf16 peak for a kernel timed more or less alone, the sustained one when the timed
-    # region is a long back-to-back run under the power cap (the 24-layer stack, or >= 0.5 s)
-    long_run = L > 1 or sec_max >= 0.5
-    tf_peak = peaks["bf16_tflops_sustained"] if long_run else peaks["bf16_tflops"]
-    t_flops = work["flops"] / (tf_peak * 1e12)
-    t_bytes = work["bytes"] / (peaks["hbm_gbs"] * 1e9)
-    bound = "tensor" if t_flops >= t_bytes else "hbm"
-    if bound == "tensor":
-        achieved, peak, runit = work["flops"] / layer_s / 1e12, tf_peak, "TFLOP/s"
-    else:
-        achieved, peak, runit = work["bytes"] / layer_s / 1e9, peaks["hbm_gbs"], "GB/s"
-    traffic = NCU_DRAM_BYTES_PER_LAUNCH.get(cfg.name)
+    layer_s = step_s / L
+    # which peak the timed region is held against: the burst figure for a region well under half a second
+    # (it starts from idle clocks), the sustained one for a back-to-back run under the power cap
+    window = "sustained" if sec_max >= 0.5 else "burst"
+    roof = roofline_of(work, layer_s, peaks, window)
+    roof["traffic"] = NCU_DRAM_BYTES_PER_LAUNCH.get(cfg.name)
+    roof["peak_source"] = f"{peaks['source']} ({window} window: timed region {sec_max:.2f} s)"
+    roof["flops_per_launch"], roof["bytes_per_launch"] = work["flops"], work["bytes"]
+    # the other window, from its own run: never one window's time over the other window's peak
+    sustained = burst = None
+    if rank == 0 and world == 1 and not args.no_ablation:
+        if window == "burst":
+            s_layer, s_sec, s_clk = lay.sustained(step_s, seconds=args.sustain_seconds, local=local)
+            sustained = dict(roofline_of(work, s_layer, peaks, "sustained"), layer_us=s_layer * 1e6, run_s=s_sec,
+                             sm_mhz=s_clk.get("sm_mhz"))
+        else:
+            torch.cuda.synchronize()
+            time.sleep(1.0)                                   # let the clocks recover
+            n_b = max(1, int(0.3 / step_s))
+            b_sec = lay.timed(lay.step_dev, n_b, 0)
+            burst = dict(roofline_of(work, b_sec / n_b / L, peaks, "burst"), layer_us=b_sec / n_b / L * 1e6, run_s=b_sec)
+    roof["other_window"] = sustained or burst
+
+    ablation = lay.ablation(step_s) if (rank == 0 and not args.no_ablation and world == 1) else {}
 
     cpu_base = None
-    if not args.no_cpu_baseline and args.ep <= 1:
+    if rank == 0 and not args.no_cpu_baseline and args.ep <= 1:
         import oracle
         oracle.build()
-        lg0 = logits_h[0].numpy()
+        lg0 = lay.logits_h[0].numpy()
         probe = wl.stratified_token_sample(cfg.T, 8, seed=99)
         inp = wl.LayerInputs(cfg, wl.make_x(cfg), lg0, *host_weights_for(cfg, wl, oracle, lg0, probe))
         n = args.ref_tokens if args.ref_tokens > 0 else cpu_sample_size(oracle, wl, inp, cfg, args.cpu_seconds)
@@ -382,40 +523,50 @@ def run_ours(args):
         oracle.moe_tokens(inp.x, inp.logits, inp.gate_up, inp.down, cfg.k, toks, cfg.S)
         dt = time.perf_counter() - t0
         cpu_base = {"value": len(toks) / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-                    "sample": f"{len(toks)} stratified tokens of T={cfg.T} (full-T routing + per-token FFN/combine) "
-                              f"in {dt:.1f} s"}
+                    "sample": f"{len(toks)} stratified tokens of T={cfg.T}, layer 0 of {L} (full-T routing + per-token "
+                              f"FFN/combine) in {dt:.1f} s"}
+        del inp
+
+    lay.close()
+    weights_cache = {}
+    del lay
+    torch.cuda.empty_cache()
+    per_config = []
+    if rank == 0 and world == 1 and args.per_config and args.ep <= 1:
+        for name in PER_CONFIG:
+            if name != cfg.name:
+                per_config.append(measure_side_config(name, args, peaks, weights_cache))
+
+    if rank != 0:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return
 
     xb = cfg.T * cfg.H * 2
     line = {
         "metric": METRIC, "value": whole_job_throughput(cfg.T * L, args.steps, world, sec_max), "unit": UNIT,
-        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec_max / args.steps * 1e3,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": cfg.name, "T": cfg.T, "H": cfg.H, "I": cfg.I, "E": cfg.E, "top_k": cfg.k,
                    "shared": cfg.S, "layers": L, "sched": args.sched, "parallelism": f"replicas x{world}",
-                   "l2_policy": "inputs larger than L2 (weights %.2f GB streamed every step)" % (work["weights_bytes"] / 1e9)},
+                   "l2_policy": "inputs larger than L2 (weights %.2f GB streamed every layer)" % (work["weights_bytes"] / 1e9)},
         "layer_us": layer_s * 1e6,
-        "layer_roofline_us": max(t_flops, t_bytes) * 1e6,
-        "roofline": {"bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
-                     "traffic": traffic,
-                     "peak_source": peaks["source"] + (" (sustained: long back-to-back run)" if long_run and bound == "tensor"
-                                                       else " (burst)" if bound == "tensor" else " (copy bandwidth)"),
-                     "frac_of_burst": (achieved / peaks["bf16_tflops"]) if bound == "tensor" else None,
-                     "flops_per_launch": work["flops"], "bytes_per_launch": work["bytes"],
-                     "frac_of_sustained": (achieved / peaks["bf16_tflops_sustained"]) if bound == "tensor" else None},
+        "layer_roofline_us": roof["layer_roofline_us"],
+        "roofline": roof,
         "e2e": {"value": whole_job_throughput(cfg.T * L, e2e_steps, world, sec_e2e), "unit": UNIT,
                 "h2d_bytes_per_step": (xb + cfg.T * cfg.E * 4) * L, "d2h_bytes_per_step": xb * L},
         "gpu_launches": args.steps * L,
         "clocks": clocks,
-        "plan": plans[0] if plans else None,
+        "plan": plan,
         "expert_parallel": ({"ep_size": args.ep, "ep_rank": args.ep_rank, **ep_desc,
                              "note": "work and roofline scaled by this rank's share of the token-expert pairs (last layer's routing)"}
                             if ep_desc else None),
         "ablation": ablation,
+        "per_config": per_config,
         "cpu_baseline": cpu_base,
         "paper_context": "paper reports 2.89x geomean MoE-layer speedup over 5 systems on 4xH100 (EP=4); no 1-GPU or B200 number",
     }
     print(json.dumps(line), flush=True)
-    moe.close()
     if world > 1:
         torch.distributed.destroy_process_group()
 
@@ -427,17 +578,29 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", default=DEFAULT_CONFIG)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--sched", default="auto", choices=["auto", "fixed", "serial"])
+    ap.add_argument("--sched", default="auto", choices=["auto", "auto_split", "fixed", "fixed_elastic", "serial"])
     ap.add_argument("--ref-tokens", type=int, default=0,
                     help="tokens in the CPU oracle's timed sample (0 = sized for --cpu-seconds of work)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--sustain-seconds", type=float, default=2.0,
+                    help="length of the back-to-back run behind every sustained-window figure")
     ap.add_argument("--ep", type=int, default=1, help="model one rank of an expert-parallel group of this size")
     ap.add_argument("--ep-rank", type=int, default=0)
     ap.add_argument("--sms", type=int, default=0, help="SMs the kernel may occupy (0 = all; even)")
     ap.add_argument("--no-ablation", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--per-config", dest="per_config", action="store_true", default=None,
+                    help="also measure the other configurations of record (default with the default workload)")
+    ap.add_argument("--no-per-config", dest="per_config", action="store_false")
+    ap.add_argument("--launcher-selftest", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.per_config is None:
+        args.per_config = args.config == DEFAULT_CONFIG
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and (args.impl == "ours" or args.launcher_selftest):
+        sys.exit(launch_ranks(args.gpus, sys.argv[1:]))
+    if args.launcher_selftest:
+        launcher_selftest(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

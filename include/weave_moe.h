@@ -6,8 +6,10 @@
  * ready-flag scheduler (chunk pipeline, bubble stealing).
  *
  * Conventions for every entry point
- *   - Plain C, no exceptions, no global state.  Return value: 0 = WEAVE_OK, negative = error
- *     (weave_moe_strerror() names it).
+ *   - Plain C, no exceptions.  Return value: 0 = WEAVE_OK, negative = error
+ *     (weave_moe_strerror() names it).  The handle-based calls keep no global state: everything
+ *     lives in the handle and in the caller's workspace.  (The one exception is documented with
+ *     weave_moe_forward_static(), which keeps a per-device record and a built-in scratch array.)
  *   - "device pointer" = address in the memory of the CUDA device that is current when
  *     weave_moe_create() is called; "host pointer" = ordinary (ideally pinned) host memory.
  *   - The caller owns every buffer (weights, workspace, inputs, outputs) and keeps the weights
@@ -43,6 +45,8 @@ enum {
 /* Scheduling modes (the paper's ablation, Section 5.6):
  *   AUTO   - full method: the cost model of Section 3.3 (Eq. 15-16) picks the number of movement
  *            SMs c and the chunk count K from the routing result, Eq. 11-14 give the steal count.
+ *            (Besides the paper's split the model also costs two plan kinds that only make sense
+ *            where movement is a local copy: see weave_moe_set_model_options().)
  *   FIXED  - the given c, K and steal count are used as they are ("w/o T" when K = 1, steal = 0).
  *   SERIAL - dispatch, GEMMs and combine run one after the other on all SMs ("w/o S+T").       */
 enum { WEAVE_SCHED_AUTO = 0, WEAVE_SCHED_FIXED = 1, WEAVE_SCHED_SERIAL = 2 };
@@ -143,13 +147,41 @@ int weave_moe_set_sm_count(weave_moe_t h, int n_sm);
  * tflops[i] = FLOP/us of i GEMM SMs, i in [0, n_sm] (host arrays of n_sm+1 floats, entry 0
  * ignored); eff_chunk[4] = Eq. 9's correction factor for K = 1,2,4,8; alpha = Section 3.1's
  * overlap ratio in [0,1); candidate grid c = c_min, c_min+c_step, ... <= c_max (at most 64
- * values; c_min and c_step even, c_min >= 2).  Synchronous copy to the device. */
+ * values; c_min and c_step even, c_min >= 2).  A candidate (c, K) is skipped when K*(E+S) > 1024
+ * (the kernel's table of (chunk, expert) segments).  Synchronous copy to the device. */
 int weave_moe_set_cost_tables(weave_moe_t h, const float *bw, const float *tflops,
                               const float *eff_chunk, float alpha, int c_min, int c_max, int c_step);
 
 /* Plan of the most recent forward (Section 3.3: SM split, chunk count, steal count) and the
  * model's predicted layer time in us.  Synchronises the handle's last stream. */
 int weave_moe_get_plan(weave_moe_t h, int *c, int *K, int *n_steal, float *t_total_us);
+
+/* Plan kinds.  SPLIT is the paper's execution plan (Section 3.3, Eq. 15): c movement SMs next to
+ * N - c GEMM SMs from the first tile on.  The paper's movement crosses NVLink; here it is a copy
+ * inside one GPU's memory that all SMs can do at full speed, so AUTO's arg-min (Eq. 16) also ranges
+ * over two kinds the paper has no use for, costed from the same tables BW(.), TFLOPS(.), eff_chunk,
+ * alpha:
+ *   DISPATCH_ALL  every SM dispatches, then c SMs combine chunk by chunk while N - c run the GEMMs:
+ *                 T = W_disp/BW(N) + max(T_comp(c,K) + T_tail(c,K), W_comb/BW(c))
+ *   PHASED        no roles: every SM dispatches, then takes GEMM tiles until the queue is empty,
+ *                 then combines (tile-level ready flags, no grid barrier between the phases):
+ *                 T = W_disp/BW(N) + W_comp/TFLOPS(N) + (1-alpha) * W_comb/BW(N);  reported as
+ *                 c = n_sm, K = 1, n_steal = 0.
+ * Ties go to SPLIT, then to the smaller c, then to the smaller K.  The steal quota of Eq. 11-14
+ * belongs to SPLIT; the other kinds report n_steal = 0.  FIXED always runs SPLIT; SERIAL reports
+ * PHASED (it is the same order of work with a grid barrier between the phases). */
+enum { WEAVE_PLAN_SPLIT = 0, WEAVE_PLAN_DISPATCH_ALL = 1, WEAVE_PLAN_PHASED = 2 };
+
+/* Kind of the plan of the most recent forward.  Synchronises the handle's last stream. */
+int weave_moe_get_plan_kind(weave_moe_t h, int *kind);
+
+/* kinds_mask: which plan kinds AUTO's arg-min may choose (bit 1 << WEAVE_PLAN_*; default all
+ * three; 1 = the paper's split only; must be non-zero).  elastic: whether movement SM pairs keep
+ * taking GEMM tiles beyond their steal quota while no combine chunk is ready, and GEMM CTAs
+ * dispatch one m-block before their first GEMM tile: 1 = on, 0 = off, -1 = the default (on under
+ * AUTO, off under FIXED, so that FIXED is the plain static split of the paper's ablation).
+ * Takes effect at the next forward. */
+int weave_moe_set_model_options(weave_moe_t h, int kinds_mask, int elastic);
 
 /* Geometry the scheduler works with: number of SMs used (= persistent CTAs; an even number,
  * because the GEMM phase runs on pairs of neighbouring SMs), rows per m-block (the unit of the
@@ -181,6 +213,11 @@ int weave_moe_get_intermediates(weave_moe_t h, const void **xe, const void **hbu
  * also re-zeroes the control words so that the handle is usable again. */
 int weave_moe_status(weave_moe_t h);
 
+/* After weave_moe_status() returned WEAVE_ERR_TIMEOUT: a small integer naming the wait that gave
+ * up first (1-3 grid barriers, 10-16 dispatch, 20-24 combine, 30-57 GEMM phase); 0 otherwise.
+ * Diagnostic only. */
+int weave_moe_last_timeout_where(weave_moe_t h);
+
 /* Upper bound, in milliseconds, for any single in-kernel wait (grid barrier, ready flag,
  * mbarrier); after it the kernel records WEAVE_ERR_TIMEOUT and every CTA returns.  Default 4000. */
 int weave_moe_set_timeout_ms(weave_moe_t h, int ms);
@@ -197,7 +234,8 @@ int weave_moe_debug_withhold_flag(weave_moe_t h, int m_block);
  * holds the number written.  Kinds: 1 routing, 2 set-up, 3 permutation fix-up, 4 dispatch tile,
  * 5 GEMM tile scheduled (claim until its inputs were ready), 6 GEMM tile epilogue (id = m-block,
  * extra = type << 16 | ns spent before the release), 7 combine tile, 8 wait for a chunk's gemm1,
- * 9 grid barrier. */
+ * 9 grid barrier, 11 GEMM tile main loop on the MMA issuer (id = type << 16 | rows, extra = ns spent
+ * waiting for a free accumulator). */
 int weave_moe_set_trace(weave_moe_t h, void *buf, int events_per_cta);
 
 /* HOST-ONLY (no GPU needed, no handle): the order in which the kernel's GEMM schedulers claim pair
@@ -229,12 +267,12 @@ int weave_moe_debug_gemm_queue(const int32_t *rows, int num_segments, int num_ch
  *     calls fail with WEAVE_ERR_WORKSPACE and must use a handle.  Every GPU on which the library
  *     is loaded holds those 64 MiB until the process exits.
  *   - The first call on each device performs a one-time set-up with that device current (it looks
- *     up the device address of the built-in array, raises the kernel's shared-memory limit and
- *     resolves the TMA descriptor encoder).  Make that first call outside any stream capture.
- *   - All calls on a device share the one array, and it keeps the previous call's contents; the
- *     call re-zeroes the control words and rewrites the cost tables on the stream before it
- *     launches.  Calls that overlap on the GPU (different streams, no ordering between them) race
- *     on the array: order them.
+ *     up the device addresses of the built-in arrays, fills the built-in cost tables with a
+ *     synchronous copy, raises the kernel's shared-memory limit and resolves the TMA descriptor
+ *     encoder).  Make that first call outside any stream capture.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents; every
+ *     call enqueues one memset of the control words and then the kernel.  Calls that overlap on the
+ *     GPU (different streams, no ordering between them) race on the array: order them.
  *   - Scheduling is AUTO with the default cost tables.  Arguments, layouts and alignment as for
  *     weave_moe_create() / weave_moe_forward(); asynchronous on the stream; a device-side failure
  *     of this call (non-finite logits, an expired wait) is not reported - use a handle when the

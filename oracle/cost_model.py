@@ -13,6 +13,16 @@ so with P pairs, T tokens and B = 2H bytes per row
     W_combine  = (P + T) * B            (Eq. 3: P rows read, T rows written)
     W_comm     = W_dispatch + W_combine (Eq. 11's undefined symbol, as in Eq. 5)
 
+Two further plan kinds, outside the paper (its movement crosses NVLink, so it never considers
+them; on one GPU, where movement is an HBM copy that all SMs can do at full speed, they matter):
+    kind 1, "dispatch on all SMs, then split": every SM dispatches, then c SMs combine chunk by
+            chunk while N-c SMs run the GEMMs:
+            T = W_disp/BW(N) + max(T_comp(c,K) + T_tail(c,K), W_comb/BW(c))
+    kind 2, "phased": all SMs per phase, no spatial split (the paper's "w/o S+T" ablation as a
+            candidate):  T = W_disp/BW(N) + W_comp/TFLOPS(N) + (1-alpha) * W_comb/BW(N)
+They take part in the arg-min only when CostTables.kinds has their bit set; ties go to the
+paper's kind, then to the smaller c, then to the smaller K.
+
 Units: work in FLOPs / bytes, rates in FLOP/us and byte/us, times in us.
 Parity: pinned by closed forms in tests/test_oracle_cost_model.py.  The values
 the paper prints for its own runs (c*=40, K*=4 at 1.365 ms; 8.2 % gap; 0.54 us)
@@ -28,6 +38,7 @@ import numpy as np
 
 f32 = np.float32
 K_CANDIDATES = (1, 2, 4, 8)
+KIND_SPLIT, KIND_DISPATCH_ALL, KIND_PHASED = 0, 1, 2
 
 
 @dataclass
@@ -43,6 +54,10 @@ class CostTables:
     c_step: int = 2
     steal_workers: int = 0   # Eq. 14's N: workers that share W_steal (0 = n_sm; a build whose GEMM
                              # worker is an SM pair passes n_sm // 2 and counts tiles per pair)
+    max_segments: int = 0    # a build that keeps a table of (chunk, expert) segments bounds the chunk
+                             # count: candidates with K * n_experts > max_segments are skipped (0 = no bound)
+    kinds: int = 1           # bit mask of the plan kinds in the arg-min: 1 = the paper's split (Eq. 15),
+                             # 2 = dispatch on all SMs then split, 4 = phased
 
 
 @dataclass
@@ -51,6 +66,7 @@ class Plan:
     K: int
     n_steal: int
     t_total: float
+    kind: int = KIND_SPLIT
 
 
 def workloads(T: int, P: int, H: int, I: int):
@@ -83,6 +99,26 @@ def t_total(tab: CostTables, c: int, ki: int, w_comp, w_disp, w_comb) -> np.floa
     return np.maximum(t_comp + t_tail, t_comm)
 
 
+def t_total_dispatch_all(tab: CostTables, c: int, ki: int, w_comp, w_disp, w_comb) -> np.float32:
+    """Kind 1: the dispatch runs on all N SMs first (W_disp / BW(N)); from then on the split of
+    Eq. 15 with only the combine left as communication."""
+    K = f32(K_CANDIDATES[ki])
+    bw = f32(tab.bw[c])
+    tf = f32(tab.tflops[tab.n_sm - c])
+    t_disp = w_disp / f32(tab.bw[tab.n_sm])
+    t_comp = w_comp / (tf * f32(tab.eff_chunk[ki]))
+    t_tail = (f32(1.0) - f32(tab.alpha)) * (w_comb / (bw * K))
+    t_comb = w_comb / bw
+    return t_disp + np.maximum(t_comp + t_tail, t_comb)
+
+
+def t_total_phased(tab: CostTables, w_comp, w_disp, w_comb) -> np.float32:
+    """Kind 2: dispatch, GEMMs and combine one after the other, each on all N SMs."""
+    bw = f32(tab.bw[tab.n_sm])
+    tf = f32(tab.tflops[tab.n_sm])
+    return (w_disp / bw + w_comp / tf) + (f32(1.0) - f32(tab.alpha)) * (w_comb / bw)
+
+
 def candidates(tab: CostTables):
     c = tab.c_min
     while c <= tab.c_max and c <= tab.n_sm - 1:
@@ -108,18 +144,33 @@ def n_steal(tab: CostTables, c: int, w_comp, w_disp, w_comb, n_tiles: int) -> in
     return max(0, min(ns, n_tiles))
 
 
-def plan(tab: CostTables, T: int, P: int, H: int, I: int, n_tiles_of_K: Sequence[int], w=None) -> Plan:
+def plan(tab: CostTables, T: int, P: int, H: int, I: int, n_tiles_of_K: Sequence[int], w=None,
+         n_experts: int = 0) -> Plan:
     """Eq. 16: argmin over the (c,K) grid, ties to the smaller c and then the smaller K;
     then the steal count at (c*,K*).  n_tiles_of_K[ki] = number of GEMM tiles of the
     layer when it is cut into K_CANDIDATES[ki] chunks.  w = (W_comp, W_disp, W_comb) overrides the
-    single-GPU workload terms (used with workloads_ep)."""
+    single-GPU workload terms (used with workloads_ep).  n_experts (routed + shared) matters only
+    with tab.max_segments.  Plan kinds beyond the paper's take part per tab.kinds; they come
+    after the paper's kind in the candidate order, so ties go to the paper's.  The steal quota
+    of Eq. 11-14 belongs to the paper's kind; the other kinds have none (0): in kind 1 the
+    movement SMs are idle from the end of the dispatch on, in kind 2 there are no roles."""
     w_comp, w_disp, w_comb = w if w is not None else workloads(T, P, H, I)
     best = None
-    for c in candidates(tab):
-        for ki in range(len(K_CANDIDATES)):
-            t = t_total(tab, c, ki, w_comp, w_disp, w_comb)
-            if best is None or t < best[0]:
-                best = (t, c, ki)
-    t, c, ki = best
-    return Plan(c, K_CANDIDATES[ki], n_steal(tab, c, w_comp, w_disp, w_comb, n_tiles_of_K[ki]),
-                float(t))
+    evaluators = ((KIND_SPLIT, t_total), (KIND_DISPATCH_ALL, t_total_dispatch_all))
+    for kind, fn in evaluators:
+        if not (tab.kinds >> kind) & 1:
+            continue
+        for c in candidates(tab):
+            for ki in range(len(K_CANDIDATES)):
+                if tab.max_segments and K_CANDIDATES[ki] * n_experts > tab.max_segments:
+                    continue
+                t = fn(tab, c, ki, w_comp, w_disp, w_comb)
+                if best is None or t < best[0]:
+                    best = (t, c, ki, kind)
+    if (tab.kinds >> KIND_PHASED) & 1:
+        t = t_total_phased(tab, w_comp, w_disp, w_comb)
+        if best is None or t < best[0]:
+            best = (t, tab.n_sm, 0, KIND_PHASED)
+    t, c, ki, kind = best
+    steal = n_steal(tab, c, w_comp, w_disp, w_comb, n_tiles_of_K[ki]) if kind == KIND_SPLIT else 0
+    return Plan(c, K_CANDIDATES[ki], steal, float(t), kind)

@@ -19,6 +19,7 @@ _SOURCES = ["weave_moe.cu", "weave_kernel.cuh", "weave_ptx.cuh"]
 WEAVE_OK = 0
 WEAVE_ERR_INVALID_ARG = -1
 SCHED_AUTO, SCHED_FIXED, SCHED_SERIAL = 0, 1, 2
+PLAN_SPLIT, PLAN_DISPATCH_ALL, PLAN_PHASED = 0, 1, 2
 ERR_NONFINITE_LOGITS, ERR_TIMEOUT = -5, -6
 
 _lib = None
@@ -63,6 +64,7 @@ EXPORTS = [
     "weave_moe_forward_static", "weave_moe_static_scratch_bytes", "weave_moe_set_sm_count",
     "weave_moe_set_expert_parallel", "weave_moe_get_ep_descriptors",
     "weave_moe_forward_host_pipelined", "weave_moe_host_wait", "weave_moe_debug_gemm_queue",
+    "weave_moe_get_plan_kind", "weave_moe_set_model_options", "weave_moe_last_timeout_where",
 ]
 
 
@@ -97,6 +99,12 @@ def load():
     lib.weave_moe_set_cost_tables.argtypes = [vp, vp, vp, vp, ctypes.c_float, ci, ci, ci]
     lib.weave_moe_get_plan.restype = ci
     lib.weave_moe_get_plan.argtypes = [vp, cip, cip, cip, cfp]
+    lib.weave_moe_get_plan_kind.restype = ci
+    lib.weave_moe_get_plan_kind.argtypes = [vp, cip]
+    lib.weave_moe_set_model_options.restype = ci
+    lib.weave_moe_set_model_options.argtypes = [vp, ci, ci]
+    lib.weave_moe_last_timeout_where.restype = ci
+    lib.weave_moe_last_timeout_where.argtypes = [vp]
     lib.weave_moe_get_geometry.restype = ci
     lib.weave_moe_get_geometry.argtypes = [vp, cip, cip, cip, cip, cip, cip, cip]
     lib.weave_moe_get_routing.restype = ci
@@ -296,7 +304,17 @@ class WeaveMoE:
         c, K, s, t = ctypes.c_int(), ctypes.c_int(), ctypes.c_int(), ctypes.c_float()
         _check(self._lib.weave_moe_get_plan(self._h, ctypes.byref(c), ctypes.byref(K), ctypes.byref(s),
                                             ctypes.byref(t)), "weave_moe_get_plan")
-        return {"c": c.value, "K": K.value, "n_steal": s.value, "t_total_us": t.value}
+        kind = ctypes.c_int()
+        _check(self._lib.weave_moe_get_plan_kind(self._h, ctypes.byref(kind)), "weave_moe_get_plan_kind")
+        return {"c": c.value, "K": K.value, "n_steal": s.value, "t_total_us": t.value, "kind": kind.value}
+
+    def set_model_options(self, kinds_mask: int = 7, elastic: int = -1):
+        """Plan kinds AUTO may choose (bit 0 the paper's split, bit 1 dispatch-all, bit 2 phased) and
+        the elastic-stealing switch (-1 = on under AUTO only)."""
+        _check(self._lib.weave_moe_set_model_options(self._h, kinds_mask, elastic), "weave_moe_set_model_options")
+
+    def last_timeout_where(self) -> int:
+        return int(self._lib.weave_moe_last_timeout_where(self._h))
 
     def geometry(self):
         v = [ctypes.c_int() for _ in range(7)]

@@ -140,16 +140,19 @@ def calibrate(cfg, layer=0, verbose=True):
     return moe, (x, lg), tables
 
 
-def grid_sweep(moe, xl, cfg, tables, verbose=True):
-    """Measured layer time for every (c, K) of the model's candidate grid, the model's pick and
-    the selection gap (the paper reports 8.2 % on its hardware)."""
+def grid_sweep(moe, xl, cfg, tables, verbose=True, c_points=C_POINTS, reps=3):
+    """Measured layer time for every (c, K) of a grid of the paper's split plans, the model's pick
+    and the selection gap (the paper reports 8.2 % on its hardware).
+
+    A grid point is AUTO with the candidate set cut down to that one (c, K): the device then runs the
+    paper's split at (c, K) with the steal count Eq. 11-14 give at that c, without the elastic
+    stealing and the first dispatch wave.  The model's pick is AUTO over the whole grid under the same
+    restrictions."""
     import torch
     import paper_2609_21483_b200 as pk
     x, lg = xl
     moe.enable_trace(0)
-    moe.set_cost_tables(tables["bw"], tables["tflops"], tables["eff_chunk"], tables["alpha"],
-                        tables["c_min"], tables["c_max"], tables["c_step"])
-    res = {}
+    res, steal_of = {}, {}
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
     def time_it(n=5):
@@ -162,21 +165,35 @@ def grid_sweep(moe, xl, cfg, tables, verbose=True):
         moe.check()
         return ev0.elapsed_time(ev1) / n * 1e3
 
+    def tables_for(c_min, c_max, c_step, only_K=None):
+        eff = np.array(tables["eff_chunk"], np.float32)
+        if only_K is not None:      # every other chunk count priced out of the arg-min
+            eff = np.array([1.0 if K == only_K else 1e-6 for K in K_POINTS], np.float32)
+        moe.set_cost_tables(tables["bw"], tables["tflops"], eff, tables["alpha"], c_min, c_max, c_step)
+
     moe.set_schedule(pk.SCHED_AUTO)
+    tables_for(tables["c_min"], tables["c_max"], tables["c_step"])
+    moe.set_model_options(7, -1)
     t_auto = time_it()
+    plan_auto = moe.plan()
+    moe.set_model_options(1 << pk.PLAN_SPLIT, 0)
+    t_pick = time_it(reps)
     plan = moe.plan()
-    for c in C_POINTS:
+    n_sm = tables["n_sm"]
+    for c in c_points:
+        if c > n_sm - 2 or c % 2:
+            continue
         for K in K_POINTS:
             if K * (cfg.E + cfg.S) > 1024:
                 continue
-            # the forced runs use the steal count the model would compute at this c
-            moe.set_schedule(pk.SCHED_FIXED, c, K, plan["n_steal"])
-            res[(c, K)] = time_it(3)
+            tables_for(c, c, 2, only_K=K)
+            res[(c, K)] = time_it(reps)
+            got = moe.plan()
+            assert (got["c"], got["K"]) == (c, K), (got, c, K)
+            steal_of[f"{c},{K}"] = got["n_steal"]
+    tables_for(tables["c_min"], tables["c_max"], tables["c_step"])
     best = min(res, key=res.get)
-    # the model's own (c*, K*) as a forced point: the selection gap inside the grid (the AUTO run above
-    # also has the elastic stealing and the first dispatch wave on all SMs, which no forced run has)
-    moe.set_schedule(pk.SCHED_FIXED, plan["c"], plan["K"], plan["n_steal"])
-    t_pick = time_it(3)
+    moe.set_model_options(7, -1)
     moe.set_schedule(pk.SCHED_SERIAL)
     t_serial = time_it()
     # what the in-kernel search costs: set-up time with and without it, from the timeline
@@ -190,17 +207,20 @@ def grid_sweep(moe, xl, cfg, tables, verbose=True):
         e = ev[ev[:, 3] == 2]
         return float(((e[:, 2] - e[:, 1]) / 1e3).mean())
     su_auto, su_fixed = setup_us(pk.SCHED_AUTO), setup_us(pk.SCHED_FIXED, plan["c"], plan["K"], plan["n_steal"])
+    moe.set_schedule(pk.SCHED_AUTO)
     if verbose:
         print("grid (us):")
-        for c in C_POINTS:
-            print(f"  c={c:3d} " + " ".join(f"K={K}:{res.get((c, K), float('nan')):8.1f}" for K in K_POINTS))
-        print(f"AUTO plan {plan} -> {t_auto:.1f} us; measured optimum {best} -> {res[best]:.1f} us; "
-              f"gap {100 * (t_auto / res[best] - 1):.1f} %; SERIAL {t_serial:.1f} us")
-        print(f"model's pick forced: {t_pick:.1f} us, selection gap inside the grid {100 * (t_pick / min(res[best], t_pick) - 1):.1f} %; "
+        for c in c_points:
+            print(f"  c={c:3d} " + " ".join(f"K={K}:{res.get((c, K), float('nan')):8.1f} (steal {steal_of.get(f'{c},{K}', '-')})"
+                                            for K in K_POINTS))
+        print(f"AUTO (all plan kinds) {plan_auto} -> {t_auto:.1f} us; measured optimum of the split grid {best} -> "
+              f"{res[best]:.1f} us; AUTO vs that {100 * (t_auto / res[best] - 1):+.1f} %; SERIAL {t_serial:.1f} us")
+        print(f"model's split pick {plan}: {t_pick:.1f} us, selection gap inside the grid {100 * (t_pick / min(res[best], t_pick) - 1):.1f} %; "
               f"set-up {su_auto:.2f} us with the search, {su_fixed:.2f} us without")
-    return {"workload": cfg.name, "auto_us": t_auto, "plan": plan, "best": list(best), "best_us": res[best],
-            "pick_us": t_pick, "selection_gap": t_pick / min(res[best], t_pick) - 1, "auto_vs_best": t_auto / res[best] - 1,
-            "serial_us": t_serial, "setup_us_auto": su_auto, "setup_us_fixed": su_fixed, "grid_points": len(res)}
+    return {"workload": cfg.name, "auto_us": t_auto, "plan_auto": plan_auto, "plan": plan, "best": list(best),
+            "best_us": min(res[best], t_pick), "pick_us": t_pick, "selection_gap": t_pick / min(res[best], t_pick) - 1,
+            "auto_vs_best": t_auto / res[best] - 1, "serial_us": t_serial, "setup_us_auto": su_auto,
+            "setup_us_fixed": su_fixed, "grid_points": len(res), "steal_of": steal_of}
 
 
 def main():

@@ -74,8 +74,17 @@ struct Ctl {
     float plan_t;
     int plan_nmb, plan_ngemm;
     unsigned ep_x_local, ep_x_in, ep_x_in_uniq;
+    int plan_kind;
 };
 constexpr int kCtlZeroWords = 24;
+
+// Plan kinds of the cost model.  kPlanSplit is the paper's (Eq. 15): c movement SMs beside N - c GEMM
+// SMs from the start.  The other two exist because on one GPU the movement is an HBM copy that all
+// SMs can do at full speed: kPlanDispatchAll lets every SM dispatch before the roles split (only the
+// combine is left to the movement SMs), kPlanPhased has no roles at all (every SM dispatches, then
+// runs GEMM tiles until the queue is empty, then combines; the ready flags still order the tiles,
+// no grid barrier separates the phases).
+enum { kPlanSplit = 0, kPlanDispatchAll = 1, kPlanPhased = 2 };
 
 struct KParams {
     int T, H, I, E, S, k, EE;
@@ -89,6 +98,7 @@ struct KParams {
     __nv_bfloat16 *xs;    // [T][H] staging of remote tokens (each unique one is copied once)
     unsigned long long *uniq_mask;   // [nblk] remote tokens of the block that have a local expert
     int elastic_steal;    // movement pairs keep stealing past their quota while no combine chunk is ready
+    int kinds;            // bit mask of the plan kinds the cost model may choose (bit kPlanSplit, ...)
     int withhold_mb;      // test hook: this m-block's "dispatched" flag is never published (-1 = off)
     int c_min, c_max, c_step;
     float alpha;
@@ -198,7 +208,7 @@ __device__ __noinline__ void give_up(Ctl *ctl, int where)
 
 // Optional timeline: one 16-byte record {start ns, end ns, kind<<24 | id, extra} per event, per CTA.
 enum { kEvRoute = 1, kEvSetup = 2, kEvFixup = 3, kEvDispatch = 4, kEvGemmLoad = 5, kEvGemmEpi = 6,
-       kEvCombine = 7, kEvWaitChunk = 8, kEvBarrier = 9, kEvDepWait = 10, kEvMma = 11 };
+       kEvCombine = 7, kEvWaitChunk = 8, kEvBarrier = 9, kEvMma = 11 };
 __device__ __forceinline__ void trace_ev(const KParams &p, SmemTail &S, int kind, unsigned id,
                                          unsigned long long t0, unsigned long long t1, unsigned extra)
 {
@@ -254,6 +264,13 @@ __device__ __forceinline__ bool flag_wait_ge(const unsigned *flag, unsigned targ
         }
     }
     return true;
+}
+
+__device__ __forceinline__ void linger_after_abort()
+{
+    // lets copies and MMAs that are already in flight land before this CTA can leave
+    const unsigned long long t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 50000ull) __nanosleep(1000);
 }
 
 // All CTAs are co-resident (cooperative launch); arrivals accumulate over the barriers of a launch.
@@ -471,6 +488,26 @@ __device__ __forceinline__ float model_t_total(const KParams &p, float bw, float
     return fmaxf(__fadd_rn(t_comp, t_tail), t_comm);
 }
 
+// Plan kind "dispatch on all SMs, then split": W_disp / BW(N), then Eq. 15 with only the combine left as
+// communication.  bw_n = BW(N).
+__device__ __forceinline__ float model_t_dispatch_all(const KParams &p, float bw, float tf, float bw_n, int ki, float w_comp,
+                                                      float w_disp, float w_comb)
+{
+    const float Kf = (float)(1 << ki);
+    const float t_disp = __fdiv_rn(w_disp, bw_n);
+    const float t_comp = __fdiv_rn(w_comp, __fmul_rn(tf, p.eff[ki]));
+    const float t_tail = __fmul_rn(__fsub_rn(1.0f, p.alpha), __fdiv_rn(w_comb, __fmul_rn(bw, Kf)));
+    const float t_comb = __fdiv_rn(w_comb, bw);
+    return __fadd_rn(t_disp, fmaxf(__fadd_rn(t_comp, t_tail), t_comb));
+}
+
+// Plan kind "phased": dispatch, GEMMs and combine one after the other, each on all N SMs.
+__device__ __forceinline__ float model_t_phased(const KParams &p, float bw_n, float tf_n, float w_comp, float w_disp, float w_comb)
+{
+    return __fadd_rn(__fadd_rn(__fdiv_rn(w_disp, bw_n), __fdiv_rn(w_comp, tf_n)),
+                     __fmul_rn(__fsub_rn(1.0f, p.alpha), __fdiv_rn(w_comb, bw_n)));
+}
+
 // Eq. 11-14 with W_tile = W_comp / n_tiles (the mean GEMM tile of this layer).
 __device__ __forceinline__ int model_n_steal(int n_sm, float bw, float tf, float w_comp, float w_disp,
                                              float w_comb, int n_tiles)
@@ -685,6 +722,9 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
             M.mv[b].d = 2;
             mbar_arrive(&S.dv_full[b]);
         }
+        // a wait gave up (or the abort word was seen): copies this warp issued may still be landing in
+        // this CTA's buffers; let them land before the CTA can leave
+        if (!ok && lane == 0) linger_after_abort();
         __syncwarp();
     } else if (warp == 1) {
         // ---- storer: one bulk store per buffer.  A buffer is handed back as soon as the store has
@@ -846,6 +886,7 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uin
             M.mv[b].d = 2;
             mbar_arrive(&S.cb_full[b]);
         }
+        if (!ok && lane == 0) linger_after_abort();      // as in the dispatch loader
         __syncwarp();
     } else if (warp >= 2) {
         // ---- reducers
@@ -925,13 +966,6 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity
         }
     }
     return true;
-}
-
-__device__ __forceinline__ void linger_after_abort()
-{
-    // lets copies and MMAs that are already in flight land before this CTA can leave
-    const unsigned long long t0 = globaltimer_ns();
-    while (globaltimer_ns() - t0 < 50000ull) __nanosleep(1000);
 }
 
 // 32 rows x 32 columns of bf16 held one row per thread (16 packed words each) go out through the
@@ -1453,8 +1487,9 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
     // entries before the barrier, so that their latency is spent waiting there.
     const int cm_ki = tid & 3, cm_c = p.c_min + (tid >> 2) * p.c_step;
     const bool cm_ok = p.mode == kModeAuto && cm_c >= 2 && cm_c <= p.c_max && cm_c <= n_sm - 2 && (EE << cm_ki) <= kMaxSeg;
-    float cm_bw = 0.f, cm_tf = 0.f;
+    float cm_bw = 0.f, cm_tf = 0.f, cm_bw_n = 0.f, cm_tf_n = 0.f;
     if (cm_ok) { cm_bw = p.bw[cm_c]; cm_tf = p.tf[n_sm - cm_c]; }
+    if (p.mode == kModeAuto) { cm_bw_n = p.bw[n_sm]; cm_tf_n = p.tf[n_sm]; }
     const unsigned long long tk1 = trace_now(p);
     bool alive = grid_barrier(p, S, (unsigned)n_sm, 1);
     const unsigned long long tk2 = trace_now(p);
@@ -1481,7 +1516,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
     const unsigned ep_xl = alive ? __ldcg(&p.ctl->x_local) : 0u, ep_xi = alive ? __ldcg(&p.ctl->x_in) : 0u,
                    ep_xu = alive ? __ldcg(&p.ctl->x_in_uniq) : 0u;
     if (blockIdx.x == 0 && tid == 0) { p.ctl->ep_x_local = ep_xl; p.ctl->ep_x_in = ep_xi; p.ctl->ep_x_in_uniq = ep_xu; }
-    int plan_c, plan_ki, plan_steal;
+    int plan_c, plan_ki, plan_steal, plan_kind = kPlanSplit;
     float plan_t = 0.f;
     if (p.mode == kModeAuto) {
         // Eq. 1-3 (single-GPU reading: every pair moves through HBM), then Eq. 16 over the grid
@@ -1498,9 +1533,19 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
             w_disp = __fmul_rn((float)(p.T + P), B);
             w_comb = __fmul_rn((float)(P + p.T), B);
         }
+        // candidate order = (kind, c ascending, K ascending), index = kind * 256 + thread; the phased plan
+        // is index 512; ties go to the smaller index
         float t = __int_as_float(0x7f800000);
-        if (cm_ok) t = model_t_total(p, cm_bw, cm_tf, cm_ki, w_comp, w_disp, w_comb);
-        int bi = tid;       // candidate order = (c ascending, K ascending): ties go to the smaller index
+        int bi = tid;
+        if (cm_ok && (p.kinds & (1 << kPlanSplit))) t = model_t_total(p, cm_bw, cm_tf, cm_ki, w_comp, w_disp, w_comb);
+        if (cm_ok && (p.kinds & (1 << kPlanDispatchAll))) {
+            const float t1 = model_t_dispatch_all(p, cm_bw, cm_tf, cm_bw_n, cm_ki, w_comp, w_disp, w_comb);
+            if (t1 < t) { t = t1; bi = kThreads + tid; }
+        }
+        if (tid == 0 && (p.kinds & (1 << kPlanPhased))) {
+            const float t2 = model_t_phased(p, cm_bw_n, cm_tf_n, w_comp, w_disp, w_comb);
+            if (t2 < t) { t = t2; bi = 2 * kThreads; }
+        }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             const float ot = __shfl_xor_sync(0xffffffffu, t, o);
@@ -1515,13 +1560,15 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
             const int oi = S.red_i[w][0];
             if (ot < t || (ot == t && oi < bi)) { t = ot; bi = oi; }
         }
-        plan_c = p.c_min + (bi >> 2) * p.c_step;
-        plan_ki = bi & 3;
+        plan_kind = bi / kThreads;
+        const int bt = bi % kThreads;      // the thread that evaluated the winner
+        plan_c = plan_kind == kPlanPhased ? n_sm : p.c_min + (bt >> 2) * p.c_step;
+        plan_ki = plan_kind == kPlanPhased ? 0 : (bt & 3);
         plan_t = t;
         // the winner hands its two table entries to everybody; the pair tiles (256 rows) of the layer at
         // the chosen K are counted meanwhile (a segment = one expert's rows inside one chunk; its last
         // pair tile may be half empty)
-        if (tid == bi) { S.red_i[0][1] = __float_as_int(cm_bw); S.red_i[0][2] = __float_as_int(cm_tf); }
+        if (tid == bt) { S.red_i[0][1] = __float_as_int(cm_bw); S.red_i[0][2] = __float_as_int(cm_tf); }
         {
             const int Kc = 1 << plan_ki, g = kFine / Kc;
             int acc = 0;
@@ -1539,8 +1586,11 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
         int n_tiles = 0;
         for (int w = 0; w < kThreads / 32; ++w) n_tiles += S.red_i[w][3];
         n_tiles *= p.nt0 + p.nt1;
-        plan_steal = model_n_steal(n_sm, __int_as_float(S.red_i[0][1]), __int_as_float(S.red_i[0][2]), w_comp, w_disp, w_comb,
-                                   n_tiles);   // per CTA pair
+        // the steal quota of Eq. 11-14 belongs to the paper's plan kind; in the other kinds the movement
+        // SMs have nothing to wait out (they take GEMM tiles while no combine chunk is ready)
+        plan_steal = plan_kind == kPlanSplit ? model_n_steal(n_sm, __int_as_float(S.red_i[0][1]), __int_as_float(S.red_i[0][2]),
+                                                            w_comp, w_disp, w_comb, n_tiles)   // per CTA pair
+                                             : 0;
         __syncthreads();
     } else if (p.mode == kModeFixed) {
         plan_c = max(2, min((p.fixed_c + 1) & ~1, n_sm - 2));     // whole CTA pairs
@@ -1551,6 +1601,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
         plan_c = n_sm;
         plan_ki = 0;
         plan_steal = 0;
+        plan_kind = kPlanPhased;
     }
     const int K = 1 << plan_ki;
     {
@@ -1603,6 +1654,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
             if (blockIdx.x == 0) {
                 p.ctl->plan_c = plan_c; p.ctl->plan_K = K; p.ctl->plan_steal = plan_steal; p.ctl->plan_t = plan_t;
                 p.ctl->plan_nmb = mb_base; p.ctl->plan_ngemm = pt_base * (p.nt0 + p.nt1);
+                p.ctl->plan_kind = plan_kind;
             }
         }
     }
@@ -1667,9 +1719,11 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
             // m-block too, so that the first wave of GEMM tiles does not wait for a handful of movers
             // (the mirror image of the final combine on all SMs); the forced "no temporal
             // scheduling" ablation keeps the two groups apart
-            const int dmax = mover ? 0x7fffffff : (p.elastic_steal ? 1 : 0);
+            // (plan kinds beyond the paper's: every CTA works through the dispatch queue first; in the
+            // phased plan every CTA is a "mover" without a steal limit)
+            const int dmax = (mover || plan_kind != kPlanSplit) ? 0x7fffffff : (p.elastic_steal ? 1 : 0);
             if (dmax > 0) dispatch_phase(p, S, stages, dmax);
-            const int budget = mover ? plan_steal : 0x7fffffff;
+            const int budget = (mover && plan_kind != kPlanPhased) ? plan_steal : 0x7fffffff;
             if (budget > 0 || p.elastic_steal) gemm_phase(p, S, stages, tmem_base, &tm, budget, ps);
             combine_phase(p, S, stages);
         }

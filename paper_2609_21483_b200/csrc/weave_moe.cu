@@ -104,6 +104,10 @@ struct weave_moe {
     int last_T;
     cudaStream_t last_stream;
     int last_cuda_error;
+    int last_timeout_where;
+    int kinds;         // plan kinds AUTO may choose (bit mask)
+    int elastic;       // -1 = on under AUTO only, 0 = off, 1 = on
+    const float *bw_dev, *tf_dev;     // cost tables on the device (in the workspace unless set otherwise)
     void *trace;
     int trace_cap;
     int ep_rank, ep_size;
@@ -234,6 +238,11 @@ int weave_moe_create(const weave_moe_config *cfg, weave_moe_t *out)
     h->last_T = 0;
     h->last_stream = nullptr;
     h->last_cuda_error = 0;
+    h->last_timeout_where = 0;
+    h->kinds = 7;
+    h->elastic = -1;
+    h->bw_dev = reinterpret_cast<const float *>(h->ws + L.bw);
+    h->tf_dev = reinterpret_cast<const float *>(h->ws + L.tf);
     h->trace = nullptr;
     h->trace_cap = 0;
     h->ep_rank = 0;
@@ -300,7 +309,8 @@ int weave_moe_forward(weave_moe_t h, const void *x, const float *logits, void *o
     p.nt1 = (c.hidden + 255) / 256;
     p.nmb_max = L.nmb_max;
     p.withhold_mb = h->withhold_mb;
-    p.elastic_steal = (h->mode == WEAVE_SCHED_AUTO) ? 1 : 0;
+    p.elastic_steal = h->elastic < 0 ? ((h->mode == WEAVE_SCHED_AUTO) ? 1 : 0) : h->elastic;
+    p.kinds = h->kinds;
     p.c_min = h->c_min; p.c_max = h->c_max; p.c_step = h->c_step;
     p.alpha = h->alpha;
     for (int i = 0; i < 4; ++i) p.eff[i] = h->eff[i];
@@ -323,8 +333,8 @@ int weave_moe_forward(weave_moe_t h, const void *x, const float *logits, void *o
     p.y = reinterpret_cast<__nv_bfloat16 *>(ws + L.y);
     p.xe_ready = reinterpret_cast<unsigned *>(ws + L.xe_ready);
     p.h_ready = reinterpret_cast<unsigned *>(ws + L.h_ready);
-    p.bw = reinterpret_cast<const float *>(ws + L.bw);
-    p.tf = reinterpret_cast<const float *>(ws + L.tf);
+    p.bw = h->bw_dev;
+    p.tf = h->tf_dev;
     p.ep_rank = h->ep_rank;
     p.ep_size = h->ep_size;
     p.ep_tshard = (T + h->ep_size - 1) / h->ep_size;
@@ -460,7 +470,7 @@ int weave_moe_set_cost_tables(weave_moe_t h, const float *bw, const float *tflop
     if (!h || !bw || !tflops || !eff_chunk) return WEAVE_ERR_INVALID_ARG;
     if (!(alpha >= 0.f && alpha < 1.f) || c_min < 2 || c_step < 2 || c_max < c_min) return WEAVE_ERR_INVALID_ARG;
     if ((c_min & 1) || (c_step & 1)) return WEAVE_ERR_INVALID_ARG;     // movement SMs come in CTA pairs
-    if ((c_max - c_min) / c_step + 1 > 64) return WEAVE_ERR_INVALID_ARG;
+    if ((c_max - c_min) / c_step + 1 > 64) return WEAVE_ERR_INVALID_ARG;      // one candidate c per four threads
     for (int i = 1; i <= h->n_sm; ++i)
         if (!(bw[i] > 0.f) || !(tflops[i] > 0.f)) return WEAVE_ERR_INVALID_ARG;
     for (int i = 0; i < 4; ++i)
@@ -485,6 +495,26 @@ int weave_moe_get_plan(weave_moe_t h, int *c, int *K, int *n_steal, float *t_tot
     if (K) *K = ctl.plan_K;
     if (n_steal) *n_steal = ctl.plan_steal;
     if (t_total_us) *t_total_us = ctl.plan_t;
+    return WEAVE_OK;
+}
+
+int weave_moe_get_plan_kind(weave_moe_t h, int *kind)
+{
+    if (!h || !kind) return WEAVE_ERR_INVALID_ARG;
+    cudaError_t e = cudaStreamSynchronize(h->last_stream);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    Ctl ctl;
+    e = cudaMemcpy(&ctl, h->ws + h->L.ctl, sizeof(Ctl), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    *kind = ctl.plan_kind;
+    return WEAVE_OK;
+}
+
+int weave_moe_set_model_options(weave_moe_t h, int kinds_mask, int elastic)
+{
+    if (!h || (kinds_mask & 7) == 0 || (kinds_mask & ~7) || elastic < -1 || elastic > 1) return WEAVE_ERR_INVALID_ARG;
+    h->kinds = kinds_mask;
+    h->elastic = elastic;
     return WEAVE_OK;
 }
 
@@ -540,7 +570,9 @@ int weave_moe_status(weave_moe_t h)
         if (e != cudaSuccess) return cuda_fail(h, e);
         e = cudaDeviceSynchronize();
         if (e != cudaSuccess) return cuda_fail(h, e);
-        h->last_cuda_error = ctl.timeout_where;   // where the first wait gave up (diagnostic)
+        h->last_timeout_where = st == WEAVE_ERR_TIMEOUT ? ctl.timeout_where : 0;
+    } else {
+        h->last_timeout_where = 0;
     }
     return st;
 }
@@ -601,6 +633,8 @@ int weave_moe_set_trace(weave_moe_t h, void *buf, int events_per_cta)
 
 int weave_moe_last_cuda_error(weave_moe_t h) { return h ? h->last_cuda_error : 0; }
 
+int weave_moe_last_timeout_where(weave_moe_t h) { return h ? h->last_timeout_where : 0; }
+
 int weave_moe_debug_gemm_queue(const int32_t *rows, int num_segments, int num_chunks, int nt0, int nt1, int32_t *out,
                                int max_tiles)
 {
@@ -655,10 +689,14 @@ namespace {
 
 constexpr size_t kStaticScratchBytes = 64ull << 20;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+// the default cost tables BW(i), TFLOPS(i), i <= 1023: they depend on the device only and are
+// written once per device, at set-up
+static __device__ __align__(256) float g_static_tables[2][1024];
 
 struct StaticDevice {
     bool ready;
     uint8_t *base;        // device address of g_static_scratch on this device, rounded up to 1024
+    const float *tables;  // device address of g_static_tables on this device
     size_t usable;
     int n_sm;
     EncodeTiledFn encode;
@@ -685,6 +723,17 @@ int static_setup(int dev, StaticDevice **out)
         d.base = reinterpret_cast<uint8_t *>(a);
         d.usable = kStaticScratchBytes - (size_t)(a - (uintptr_t)sym);
         d.n_sm = prop.multiProcessorCount & ~1;
+        void *tsym = nullptr;
+        if (cudaGetSymbolAddress(&tsym, g_static_tables) != cudaSuccess || tsym == nullptr) return WEAVE_ERR_CUDA;
+        d.tables = static_cast<const float *>(tsym);
+        {
+            std::vector<float> bw, tf;      // host heap only; filled and copied once per device
+            default_tables(d.n_sm, bw, tf);
+            if (cudaMemcpy(tsym, bw.data(), sizeof(float) * (d.n_sm + 1), cudaMemcpyHostToDevice) != cudaSuccess ||
+                cudaMemcpy(static_cast<float *>(tsym) + 1024, tf.data(), sizeof(float) * (d.n_sm + 1),
+                           cudaMemcpyHostToDevice) != cudaSuccess)
+                return WEAVE_ERR_CUDA;
+        }
         if (cudaFuncSetAttribute(weave_moe_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) !=
             cudaSuccess)
             return WEAVE_ERR_CUDA;
@@ -743,27 +792,20 @@ int weave_moe_forward_static(int hidden, int ffn, int num_experts, int top_k, in
     h.withhold_mb = -1;
     h.ep_rank = 0;
     h.ep_size = 1;
+    h.kinds = 7;
+    h.elastic = -1;
+    h.bw_dev = sd->tables;
+    h.tf_dev = sd->tables + 1024;
     const int EE = num_experts + num_shared;
     int r = 0;
     r = encode_maps(sd->encode, &h.tm, h.ws + L.xe, h.ws + L.hbuf, gate_up, down, (uint64_t)L.p_max, (uint64_t)EE,
                     (uint64_t)hidden, (uint64_t)ffn);
     if (r) return WEAVE_ERR_CUDA;
 
-    // the array keeps whatever the last call left behind: zero the control words, refill the tables
+    // the array keeps whatever the last call left behind: zero the control words (the cost tables sit
+    // in their own array, written once at set-up), then the kernel; nothing else is enqueued
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     if (cudaMemsetAsync(h.ws, 0, L.zero_end, st) != cudaSuccess) return WEAVE_ERR_CUDA;
-    float bw[1024], tf[1024];
-    {
-        for (int i = 1; i <= h.n_sm; ++i) {
-            bw[i] = 42.0e3f * (float)i;
-            tf[i] = 1.30e9f * sqrtf((float)i / (float)h.n_sm);
-        }
-        bw[0] = bw[1]; tf[0] = tf[1];
-    }
-    if (cudaMemcpyAsync(h.ws + L.bw, bw, sizeof(float) * (h.n_sm + 1), cudaMemcpyHostToDevice, st) != cudaSuccess)
-        return WEAVE_ERR_CUDA;
-    if (cudaMemcpyAsync(h.ws + L.tf, tf, sizeof(float) * (h.n_sm + 1), cudaMemcpyHostToDevice, st) != cudaSuccess)
-        return WEAVE_ERR_CUDA;
     return weave_moe_forward(&h, x, router_logits, out, T, cuda_stream);
 }
 

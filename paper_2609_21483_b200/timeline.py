@@ -197,6 +197,8 @@ def run(cfg, sched="auto", layer=0, events_per_cta=16384):
     moe = pk.WeaveMoE(as_bf16(inp.gate_up), as_bf16(inp.down), cfg.E, cfg.k, cfg.S, max_tokens=cfg.T)
     if sched == "serial":
         moe.set_schedule(pk.SCHED_SERIAL)
+    elif sched == "split":          # AUTO restricted to the paper's plan kind (a spatial split)
+        moe.set_model_options(1 << pk.PLAN_SPLIT, -1)
     elif sched.startswith("fixed"):
         _, c, K, s = sched.split(":")
         moe.set_schedule(pk.SCHED_FIXED, int(c), int(K), int(s))
@@ -219,7 +221,7 @@ def main(argv=None):
     import workloads as wl
     ap = argparse.ArgumentParser(description=__doc__.split("\n")[0])
     ap.add_argument("--config", default="c4_dsv2lite_T1024")
-    ap.add_argument("--sched", default="auto")
+    ap.add_argument("--sched", default="auto", help="auto | split | serial | fixed:c:K:steal")
     ap.add_argument("--ascii", default=None, help="write the per-CTA text timeline to this file")
     a = ap.parse_args(argv)
     rep, trace = run(wl.CONFIGS[a.config], a.sched)

@@ -114,6 +114,38 @@ def test_multi_rank_aggregation_over_gloo(tmp_path):
     assert "rank0-ok" in r.stdout and "rank1-ok" in r.stdout
 
 
+def test_bench_starts_its_own_ranks_for_gpus_n():
+    """`python bench.py --gpus 2 ...` as a user types it (no torchrun in front): the script starts two
+    ranks of itself, they meet over gloo (CPU stand-in for the NCCL replicas), the slowest rank's time
+    decides and only rank 0 prints a line."""
+    import json
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "10", "--launcher-selftest"]
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    r = subprocess.run(cmd, capture_output=True, text=True, timeout=300, env=env)
+    assert r.returncode == 0, r.stdout + r.stderr
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = lines[0]
+    assert d["launcher_selftest"] and d["n_gpus"] == 2 and d["max_seconds"] == 2.0
+    assert abs(d["value"] - 4096 * 10 * 2 / 2.0) < 1e-9
+
+
+def test_roofline_windows_use_their_own_peaks():
+    """A burst-window time is held against the burst bf16 peak and a sustained-run time against the
+    sustained one; the bound (tensor or HBM) is decided with the same window's peak."""
+    import bench
+    import workloads as wl
+    peaks = {"hbm_gbs": 6500.0, "bf16_tflops": 1600.0, "bf16_tflops_sustained": 1400.0, "source": "test"}
+    w = bench.layer_work(wl.CONFIGS["c2_mixtral"])
+    b = bench.roofline_of(w, 2.0e-3, peaks, "burst")
+    s = bench.roofline_of(w, 2.5e-3, peaks, "sustained")
+    assert b["bound"] == s["bound"] == "tensor" and b["peak"] == 1600.0 and s["peak"] == 1400.0
+    assert np.isclose(b["frac"], w["flops"] / 2.0e-3 / 1600e12) and np.isclose(s["frac"], w["flops"] / 2.5e-3 / 1400e12)
+    w4 = bench.layer_work(wl.CONFIGS["c4_dsv2lite_T64"])
+    h = bench.roofline_of(w4, 200e-6, peaks, "burst")
+    assert h["bound"] == "hbm" and h["unit"] == "GB/s" and np.isclose(h["frac"], w4["bytes"] / 200e-6 / 6500e9)
+
+
 def test_layer_work_formulas():
     """FLOPs per launch = P * 6HI (Eq. 1); bytes of config 2 match the hand-computed roofline table."""
     import bench

@@ -9,7 +9,7 @@ import oracle
 from oracle import cost_model as cm
 import workloads as wl
 import paper_2609_21483_b200 as pk
-from parity import bf16_to_np, check_values, to_dev
+from parity import bf16_to_np, check_values, coverage_token_sample, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -104,10 +104,14 @@ def test_plan_uses_the_paper_s_workload_terms_in_ep_mode():
         g = 8 // K
         tiles.append(sum(int(((fine[j * g:(j + 1) * g].sum(0) + geo["gemm_tile_m"] - 1) // geo["gemm_tile_m"]).sum())
                          for j in range(K)) * nt)
-    tab = cm.CostTables(N, bw, tf, eff, 0.7, 2, N // 2, 2, steal_workers=N // 2)
-    want = cm.plan(tab, cfg.T, 0, cfg.H, cfg.I, tiles, w=cm.workloads_ep(xl, xi, xu, cfg.H, cfg.I))
-    got = moe.plan()
-    assert (got["c"], got["K"], got["n_steal"]) == (want.c, want.K, want.n_steal), (got, want)
+    for kinds in (7, 1):      # all plan kinds (the default), then the paper's split alone
+        moe.set_model_options(kinds, -1)
+        moe.forward(x, lg)
+        moe.check()
+        tab = cm.CostTables(N, bw, tf, eff, 0.7, 2, N // 2, 2, steal_workers=N // 2, max_segments=1024, kinds=kinds)
+        want = cm.plan(tab, cfg.T, 0, cfg.H, cfg.I, tiles, w=cm.workloads_ep(xl, xi, xu, cfg.H, cfg.I), n_experts=cfg.E)
+        got = moe.plan()
+        assert (got["kind"], got["c"], got["K"], got["n_steal"]) == (want.kind, want.c, want.K, want.n_steal), (got, want)
     moe.close()
 
 
@@ -122,7 +126,11 @@ def test_c5_shaped_rank_share_sampled():
     moe.check()
     _, (xl, xi, xu) = _check_rank(moe, inp, 0, 4)
     assert xu <= xi and xl + xi > 0
-    toks = wl.stratified_token_sample(cfg.T, 8, seed=5)
+    # a sample that reaches every local expert's first and last row and every local m-block
+    toks, cov = coverage_token_sample(oracle.routing_ep(inp.logits, cfg.k, 0, 4), cfg, 8, None,
+                                      moe.geometry()["block_m"], seed=5)
+    print(f"[coverage] c5 rank 0 of 4: {cov}")
+    assert cov["experts"] == cov["experts_nonempty"] and cov["m_blocks"] == cov["m_blocks_total"], cov
     ref = oracle.moe_tokens_ep(inp.x, inp.logits, inp.gate_up, inp.down, cfg.k, toks, 0, 4)
     check_values(bf16_to_np(out[torch.from_numpy(toks).long().cuda()]), ref, "c5 rank 0")
     moe.close()

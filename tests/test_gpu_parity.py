@@ -43,11 +43,12 @@ def test_c1_tiny_every_schedule_matches_oracle_and_each_other():
     moe.close()
 
 
-@pytest.mark.parametrize("name,n_sample", [("c4_dsv2lite_T64", None), ("c4_dsv2lite_T256", 48),
+@pytest.mark.parametrize("name,n_sample", [("c4_dsv2lite_T64", None), ("c4_dsv2lite_T256", None),
                                            ("c4_dsv2lite_T1024", 32)])
 def test_c4_decode_like_with_shared_experts(name, n_sample):
+    """T = 64 and 256 in full; T = 1024 on a sample that reaches every expert and every m-block."""
     cfg = wl.CONFIGS[name]
-    moe, _, _ = run_case(cfg, n_sample=n_sample)
+    moe, _, _ = run_case(cfg, n_sample=n_sample, require_full_coverage=True)
     moe.close()
 
 
@@ -56,7 +57,9 @@ def test_c3_skewed_routing_sampled():
     cfg = wl.CONFIGS["c3_qwen3_30b"]
     inp = wl.make_inputs(cfg)
     dev = to_dev(inp)
-    moe, out0, _ = run_case(cfg, n_sample=24, inp=inp, dev_tensors=dev)
+    # the sample comes from the oracle's routing: first and last row of each of the ~126 non-empty
+    # experts (69 of them have at most 32 rows) and a row in each of the ~605 m-blocks
+    moe, out0, _ = run_case(cfg, n_sample=32, inp=inp, dev_tensors=dev, require_full_coverage=True)
     bits = out0.view(torch.int16).clone()
     # chunking multiplies the (chunk, expert) segments and with them the unpaired, swapped-operand
     # tiles; every schedule, repeated, must reproduce the same bits
@@ -72,18 +75,19 @@ def test_c3_skewed_routing_sampled():
 
 def test_c2_mixtral_shaped_sampled():
     cfg = wl.CONFIGS["c2_mixtral"]
-    moe, _, _ = run_case(cfg, n_sample=12)
+    moe, _, _ = run_case(cfg, n_sample=200, require_full_coverage=True)     # ~270 tokens, every m-block
     moe.close()
 
 
-def test_c5_qwen3_235b_shaped_two_layers_sampled():
-    """Two layers of the 24-layer stack (same weights, fresh skew per layer) on one handle."""
+def test_c5_qwen3_235b_shaped_three_layers_sampled():
+    """Three layers of the 24-layer stack (same weights, fresh skew per layer) on one handle, each on
+    a sample that reaches every expert and every one of its ~1100 m-blocks."""
     cfg = wl.CONFIGS["c5_qwen3_235b"]
     weights = wl.make_weights(cfg)
     moe = None
     dev_w = None
     plans = []
-    for layer in (0, 7):
+    for layer in (0, 7, 23):
         inp = wl.make_inputs(cfg, layer, weights)
         if dev_w is None:
             dev = to_dev(inp)
@@ -91,17 +95,22 @@ def test_c5_qwen3_235b_shaped_two_layers_sampled():
         else:
             x = torch.from_numpy(inp.x.view(np.int16)).view(torch.bfloat16).cuda()
             dev = (x, torch.from_numpy(inp.logits).cuda()) + dev_w
-        moe, _, _ = run_case(cfg, n_sample=6, inp=inp, dev_tensors=dev, moe=moe)
+        moe, _, _ = run_case(cfg, n_sample=16, layer=layer, inp=inp, dev_tensors=dev, moe=moe, require_full_coverage=True)
         plans.append(moe.plan())
     moe.close()
 
 
-@pytest.mark.parametrize("name", ["t1_dsv3_T2048", "t1_phi35_T2048", "t1_qwen35_35b_T2048", "t1_dsv2_T2048",
-                                  "t1_qwen35_35b_T16384"])
-def test_remaining_table1_shapes_sampled(name):
+@pytest.mark.parametrize("name,budget", [("t1_dsv3_T2048", 40), ("t1_dsv3_T8192", 40), ("t1_phi35_T2048", None),
+                                         ("t1_qwen35_35b_T2048", None), ("t1_qwen35_35b_T8192", None),
+                                         ("t1_dsv2_T2048", 64), ("t1_qwen35_35b_T16384", 256)])
+def test_remaining_table1_shapes_sampled(name, budget):
     """The Table 1 rows that are not among the five configs of record (256 experts, H = 7168 / 5120,
-    I = 512 ... 6400), mildly skewed routing, four sampled tokens each."""
-    moe, _, _ = run_case_streamed(wl.CONFIGS[name], n_sample=4)
+    I = 512 ... 6400), mildly skewed routing.  Shapes whose weights fit the host are checked on a
+    sample that reaches every expert and every m-block; for the 20 GB and 7 GB layers the sample is
+    cut to `budget` tokens, smallest experts first (their oracle weights are generated in groups)."""
+    cfg = wl.CONFIGS[name]
+    moe, _, _ = run_case_streamed(cfg, n_sample=8, budget=budget,
+                                  max_experts_per_group=64 if cfg.H * cfg.I > 4 << 20 else 256)
     moe.close()
 
 
@@ -266,7 +275,7 @@ def test_short_tiles_back_to_back_launches_keep_their_bits():
     cfg = _small("short_tiles", 4096, 512, 256, 64, 4, zipf=1.0, cfg_id=93)
     inp = wl.make_inputs(cfg)
     dev = to_dev(inp)
-    moe, out0, _ = run_case(cfg, n_sample=32, inp=inp, dev_tensors=dev)
+    moe, out0, _ = run_case(cfg, n_sample=32, inp=inp, dev_tensors=dev, budget=96)
     bits = out0.view(torch.int16).clone()
     for s in [(pk.SCHED_AUTO, 0, 1, 0), (pk.SCHED_FIXED, 16, 2, 8), (pk.SCHED_SERIAL, 0, 1, 0)]:
         moe.set_schedule(*s)
@@ -375,37 +384,54 @@ def _fine_counts(ref, cfg, geo):
     return fine
 
 
-@pytest.mark.parametrize("name", ["c1_tiny", "c4_dsv2lite_T256"])
-def test_device_plan_equals_cpu_cost_model(name):
-    """AUTO's (c*, K*, n_steal) must equal the CPU restatement of Eq. 1-16 fed the same tables."""
+@pytest.mark.parametrize("name,kinds,c_step", [("c1_tiny", 1, 2), ("c1_tiny", 7, 2), ("c4_dsv2lite_T256", 7, 2),
+                                               ("c4_dsv2lite_T256", 1, 4), ("t1_qwen35_35b_T2048", 7, 4),
+                                               ("t1_qwen35_35b_T2048", 3, 2)])
+def test_device_plan_equals_cpu_cost_model(name, kinds, c_step):
+    """AUTO's plan (kind, c*, K*, n_steal) must equal the CPU restatement of Eq. 1-16 fed the same
+    tables: with the paper's plan kind alone (kinds = 1) and with the added kinds, on a candidate grid
+    with steps of 2 and of 4, and on a 256-expert shape, where K = 8 is not a candidate on either
+    side (K * (E+S) > 1024 segments)."""
     from oracle import cost_model as cm
     cfg = wl.CONFIGS[name]
-    inp = wl.make_inputs(cfg)
-    x, lg, gu, dn = to_dev(inp)
+    x_h, lg_h = wl.make_x(cfg), wl.make_logits(cfg)
+    x = torch.from_numpy(x_h.view(np.int16)).view(torch.bfloat16).cuda()
+    lg = torch.from_numpy(lg_h).cuda()
+    EE = cfg.E + cfg.S
+    # the plan does not depend on the weights' values: any finite ones do
+    gu = torch.zeros((EE, 2 * cfg.I, cfg.H), dtype=torch.bfloat16, device="cuda")
+    dn = torch.zeros((EE, cfg.H, cfg.I), dtype=torch.bfloat16, device="cuda")
     moe = pk.WeaveMoE(gu, dn, cfg.E, cfg.k, cfg.S, max_tokens=cfg.T)
     geo = moe.geometry()
     N = geo["n_sm"]
-    ref = oracle.routing(inp.logits, cfg.k, cfg.S)
+    ref = oracle.routing(lg_h, cfg.k, cfg.S)
     fine = _fine_counts(ref, cfg, geo)
     nt = _n_tiles_of_K(fine, geo, cfg.H, cfg.I)
-    rng = np.random.default_rng(5)
-    for trial in range(6):
+    rng = np.random.default_rng(5 + kinds + 10 * c_step)
+    seen = set()
+    for trial in range(8):
         idx = np.arange(N + 1, dtype=np.float64)
-        b, f = 10 ** rng.uniform(3.5, 5.5), 10 ** rng.uniform(6, 7.5)
+        b, f = 10 ** rng.uniform(3.0, 5.5), 10 ** rng.uniform(6, 8.0)
         bw = (b * np.minimum(idx, rng.uniform(20, 148))).astype(np.float32)
-        tf = (f * idx ** rng.uniform(0.7, 1.0)).astype(np.float32)
+        tf = (f * idx ** rng.uniform(0.5, 1.0)).astype(np.float32)
         bw[0], tf[0] = bw[1], tf[1]
-        eff = np.array([1.0, rng.uniform(.8, 1), rng.uniform(.6, .9), rng.uniform(.4, .8)], np.float32)
+        eff = np.array([1.0, rng.uniform(.8, 1), rng.uniform(.6, 1), rng.uniform(.4, 1)], np.float32)
         alpha = float(rng.uniform(0, 0.95))
-        tab = cm.CostTables(N, bw, tf, eff, alpha, c_min=2, c_max=N // 2, c_step=2, steal_workers=N // 2)
-        want = cm.plan(tab, cfg.T, cfg.P, cfg.H, cfg.I, nt)
-        moe.set_cost_tables(bw, tf, eff, alpha, 2, N // 2, 2)
+        c_min = 2 if c_step == 2 else 4
+        tab = cm.CostTables(N, bw, tf, eff, alpha, c_min=c_min, c_max=N // 2, c_step=c_step, steal_workers=N // 2,
+                            max_segments=1024, kinds=kinds)
+        want = cm.plan(tab, cfg.T, cfg.P, cfg.H, cfg.I, nt, n_experts=EE)
+        moe.set_cost_tables(bw, tf, eff, alpha, c_min, N // 2, c_step)
+        moe.set_model_options(kinds, -1)
         moe.set_schedule(pk.SCHED_AUTO)
         moe.forward(x, lg)
         moe.check()
         got = moe.plan()
-        assert (got["c"], got["K"], got["n_steal"]) == (want.c, want.K, want.n_steal), (trial, got, want)
+        assert (got["kind"], got["c"], got["K"], got["n_steal"]) == (want.kind, want.c, want.K, want.n_steal), (trial, got, want)
         assert abs(got["t_total_us"] - want.t_total) <= 1e-6 * want.t_total
+        assert EE * got["K"] <= 1024
+        seen.add(got["kind"])
+    assert seen <= {k for k in range(3) if (kinds >> k) & 1}
     moe.close()
 
 

@@ -72,19 +72,46 @@ def test_calibration_produces_usable_tables_and_auto_follows_them():
     moe.set_cost_tables(tab["bw"], tab["tflops"], tab["eff_chunk"], tab["alpha"], tab["c_min"], tab["c_max"],
                         tab["c_step"])
     moe.set_schedule(pk.SCHED_AUTO)
+    moe.set_model_options(1 << pk.PLAN_SPLIT, -1)         # the paper's plan kind alone
     moe.forward(x, lg)
     moe.check()
     p = moe.plan()
+    assert p["kind"] == pk.PLAN_SPLIT
     assert 2 <= p["c"] <= n // 2 and p["c"] % 2 == 0 and p["K"] in (1, 2, 4, 8) and p["t_total_us"] > 0
+    moe.set_model_options(7, -1)                          # every kind: the phased plan reports c = n_sm
+    moe.forward(x, lg)
+    moe.check()
+    q = moe.plan()
+    assert q["t_total_us"] <= p["t_total_us"] and (q["c"] == n) == (q["kind"] == pk.PLAN_PHASED)
+    moe.close()
+
+
+def test_grid_sweep_compares_the_model_s_pick_with_the_forced_grid():
+    """The (c, K) sweep of the accuracy experiment (Section 5.5) on a small shape: every grid point is
+    the paper's split forced to one (c, K) with the steal count Eq. 11-14 give at that c; the model's
+    own pick must be one of the candidates and its gap to the measured optimum finite."""
+    from paper_2609_21483_b200 import calibrate
+    cfg = wl.CONFIGS["c4_dsv2lite_T256"]
+    moe, xl, tab = calibrate.calibrate(cfg, verbose=False)
+    rep = calibrate.grid_sweep(moe, xl, cfg, tab, verbose=False, c_points=(4, 16, 48), reps=2)
+    assert rep["grid_points"] == 3 * 4
+    assert rep["plan"]["kind"] == pk.PLAN_SPLIT and 2 <= rep["plan"]["c"] <= tab["n_sm"] // 2
+    assert np.isfinite(rep["selection_gap"]) and rep["selection_gap"] >= 0.0
+    assert rep["best_us"] > 0 and rep["pick_us"] >= rep["best_us"] * 0.999
+    # the steal quota moves with c: fewer movement SMs finish later, so less is left to steal
+    steals = {c: rep["steal_of"][f"{c},1"] for c in (4, 16, 48)}
+    assert steals[4] <= steals[16] <= steals[48]
+    assert rep["auto_us"] > 0 and rep["serial_us"] > 0
     moe.close()
 
 
 @pytest.mark.gpu
 def test_utilisation_report_from_the_kernel_timeline():
-    """AUTO overlaps movement with tensor-core work; with barriers between the phases nothing overlaps."""
+    """The paper's spatial split overlaps movement with tensor-core work; with barriers between the
+    phases nothing overlaps."""
     from paper_2609_21483_b200 import timeline
     cfg = wl.CONFIGS["c3_qwen3_30b"].with_T(4096)
-    auto, trace = timeline.run(cfg, "auto")
+    auto, trace = timeline.run(cfg, "split")
     serial, _ = timeline.run(cfg, "serial")
     for rep in (auto, serial):
         assert 0.0 < rep["sm_busy"] <= 1.0 and 0.0 < rep["tensor_active"] <= 1.0

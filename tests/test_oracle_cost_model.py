@@ -117,3 +117,90 @@ def test_more_movement_cost_never_lowers_c(T, P, H, I):
         p = cm.plan(_toy(b=b, f=8e6, eff=(1, .9, .8, .7)), T, P, H, I, [64] * 4)
         assert p.c >= last
         last = p.c
+
+
+def test_steal_count_with_pair_workers():
+    """A build whose GEMM worker is an SM pair divides W_steal among N/2 workers and counts pair
+    tiles (Eq. 14 with N = pairs).  Closed forms: infinitely fast movement leaves all of W_comp to
+    share, so every worker gets n_tiles / (N/2) tiles; when W_partial is exactly half of W_comp the
+    quota is half of that; the pair quota is twice the per-SM quota for the same tile count."""
+    N = 148
+    T, P, H, I = 4096, 8192, 4096, 14336
+    w = cm.workloads(T, P, H, I)
+    n_tiles = 7400                       # 100 per pair
+    assert cm.n_steal(_toy(b=1e20, steal_workers=N // 2), 10, *w, n_tiles) == n_tiles // (N // 2) == 100
+    assert cm.n_steal(_toy(b=1e20), 10, *w, n_tiles) == n_tiles // N == 50
+    f = 10.0e6
+    t_half = float(w[0]) / 2 / (f * (N - 10))
+    b = float(w[1] + w[2]) / t_half / 10
+    assert abs(cm.n_steal(_toy(b=b, f=f, steal_workers=N // 2), 10, *w, n_tiles) - 50) <= 1
+    # slow movement: nothing is left to steal, whatever the worker count
+    assert cm.n_steal(_toy(b=1e-3, steal_workers=N // 2), 10, *w, n_tiles) == 0
+    # a non-integer share rounds to nearest: 7437 / 74 = 100.5 -> 101 (floor(x + 0.5)), 7436 / 74 = 100.49 -> 100
+    assert cm.n_steal(_toy(b=1e20, steal_workers=N // 2), 10, *w, 7437) == 101
+    assert cm.n_steal(_toy(b=1e20, steal_workers=N // 2), 10, *w, 7436) == 100
+
+
+def test_segment_table_bound_removes_large_chunk_counts():
+    """With a bound on (chunk, expert) segments, K * n_experts > bound is not a candidate: without a
+    chunking penalty the model wants K = 8, and gets the largest K that fits."""
+    T, P, H, I = 8192, 65536, 2048, 512
+    free = _toy(eff=(1, 1, 1, 1))
+    assert cm.plan(free, T, P, H, I, [10] * 4, n_experts=256).K == 8
+    bound = _toy(eff=(1, 1, 1, 1), max_segments=1024)
+    assert cm.plan(bound, T, P, H, I, [10] * 4, n_experts=256).K == 4      # 8 * 256 > 1024
+    assert cm.plan(bound, T, P, H, I, [10] * 4, n_experts=128).K == 8
+    assert cm.plan(bound, T, P, H, I, [10] * 4, n_experts=600).K == 1
+
+
+def test_phased_plan_wins_when_movement_is_cheap_by_the_gemm_rate_ratio():
+    """Movement -> 0: every kind's time is its GEMM time, W_comp / TFLOPS(n).  The phased plan runs
+    the GEMMs on all N SMs, the best split on N - c_min, so the phased plan wins and the ratio of
+    the two times is TFLOPS(N) / TFLOPS(N - c_min)."""
+    N = 148
+    T, P, H, I = 4096, 8192, 4096, 14336
+    split_only = _toy(N, b=1e15, f=1e6)
+    both = _toy(N, b=1e15, f=1e6, kinds=1 | 4)
+    p0 = cm.plan(split_only, T, P, H, I, [10] * 4)
+    p2 = cm.plan(both, T, P, H, I, [10] * 4)
+    assert (p0.kind, p0.c) == (cm.KIND_SPLIT, 2)
+    assert (p2.kind, p2.c, p2.K, p2.n_steal) == (cm.KIND_PHASED, N, 1, 0)
+    assert math.isclose(p0.t_total / p2.t_total, N / (N - 2), rel_tol=1e-5)      # toy TFLOPS(n) = f * n
+
+
+def test_phased_plan_loses_when_movement_dominates_and_overlaps():
+    """Linear toy curves, alpha = 0, K = 1 forced.  By hand: phased = W_disp/(bN) + A/N + W_comb/(bN)
+    with A = W_comp/f; the split at c takes max(A/(N-c) + W_comb/(bc), (W_disp+W_comb)/(bc)).  For
+    three bandwidths the plan must be the smaller of the hand-written phased time and the hand-written
+    minimum over c, and must say which kind it is."""
+    N = 148
+    T, P, H, I = 8192, 65536, 2048, 768
+    w_comp, w_disp, w_comb = (float(v) for v in cm.workloads(T, P, H, I))
+    f = 8.0e6
+    A = w_comp / f
+    for b in (2.0e3, 2.0e4, 2.0e5):
+        tab = _toy(N, b=b, f=f, eff=(1.0, 1e-3, 1e-3, 1e-3), kinds=1 | 4, c_min=2, c_max=N - 2, c_step=2)
+        hand_phased = w_disp / (b * N) + A / N + w_comb / (b * N)
+        hand_split = min(max(A / (N - c) + w_comb / (b * c), (w_disp + w_comb) / (b * c)) for c in range(2, N - 1, 2))
+        p = cm.plan(tab, T, P, H, I, [10] * 4)
+        assert math.isclose(p.t_total, min(hand_phased, hand_split), rel_tol=1e-5)
+        assert (p.kind == cm.KIND_PHASED) == (hand_phased < hand_split)
+
+
+def test_dispatch_all_kind_closed_form_and_tie_order():
+    """Kind 1 at (c, K): W_disp/BW(N) + max(T_comp + T_tail, W_comb/BW(c)).  With a huge GEMM rate
+    it is W_disp/(bN) + W_comb/(bc), minimal at c_max; the paper's kind gives (W_disp+W_comb)/(b c_max),
+    which is larger whenever c_max < N, so kind 1 wins; with identical times the paper's kind is kept."""
+    N = 148
+    T, P, H, I = 1000, 8000, 1024, 512
+    w_comp, w_disp, w_comb = (float(v) for v in cm.workloads(T, P, H, I))
+    b = 1.0e3
+    tab = _toy(N, b=b, f=1e30, kinds=1 | 2)
+    p = cm.plan(tab, T, P, H, I, [10] * 4)
+    assert (p.kind, p.c, p.n_steal) == (cm.KIND_DISPATCH_ALL, 74, 0)
+    assert math.isclose(p.t_total, w_disp / (b * N) + w_comb / (b * 74), rel_tol=1e-5)
+    # no movement cost at all and flat curves: every candidate of every kind ties -> paper's kind, c_min, K = 1
+    flat = np.full(N + 1, 5.0e6, np.float32)
+    tabf = cm.CostTables(N, np.full(N + 1, 1e30, np.float32), flat, np.ones(4, np.float32), 0.0, kinds=7)
+    pf = cm.plan(tabf, T, P, H, I, [10] * 4)
+    assert (pf.kind, pf.c, pf.K) == (cm.KIND_SPLIT, 2, 1)
