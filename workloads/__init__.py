@@ -95,6 +95,11 @@ CONFIGS: Dict[str, MoEConfig] = {
     # 24 Qwen3-235B-A22B-shaped layers, fresh skew per layer
     "c5_qwen3_235b": MoEConfig("c5_qwen3_235b", 5, T=16384, H=4096, I=1536, E=128, k=8,
                                zipf_range=(0.8, 1.6), layers=24),
+    # a quarter of one Qwen3-235B-shaped layer for profiler captures (the full layer holds 7.4 GB on the
+    # device): a quarter of the experts AND a quarter of the tokens, so the rows per expert, the tile mix
+    # and the bytes per token-expert pair stay those of the full layer while weights, activations and
+    # FLOPs are each exactly a quarter
+    "c5_quarter": MoEConfig("c5_quarter", 5, T=4096, H=4096, I=1536, E=32, k=8, zipf_range=(0.8, 1.6), layers=1),
 }
 
 # The other shapes of the paper's Table 1 (Qwen3-30B and DSv2-Lite are C3 / C4 above), at the
