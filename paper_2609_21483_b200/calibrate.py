@@ -177,20 +177,24 @@ def grid_sweep(moe, xl, cfg, tables, verbose=True, c_points=C_POINTS, reps=3):
     t_auto = time_it()
     plan_auto = moe.plan()
     moe.set_model_options(1 << pk.PLAN_SPLIT, 0)
-    t_pick = time_it(reps)
+    time_it(1)
     plan = moe.plan()
     n_sm = tables["n_sm"]
-    for c in c_points:
-        if c > n_sm - 2 or c % 2:
-            continue
-        for K in K_POINTS:
-            if K * (cfg.E + cfg.S) > 1024:
-                continue
+    # the model's own pick is a grid point like the others, measured in the same sweeps: two sweeps in
+    # opposite order, so that the clock state the previous points leave behind (a slow K = 8 point lets
+    # the part cool down) hits every point from both sides
+    cs = sorted({c for c in c_points if c <= n_sm - 2 and c % 2 == 0} | {plan["c"]})
+    pts = [(c, K) for c in cs for K in K_POINTS if K * (cfg.E + cfg.S) <= 1024]
+    acc = {pt: 0.0 for pt in pts}
+    for sweep in (pts, pts[::-1]):
+        for c, K in sweep:
             tables_for(c, c, 2, only_K=K)
-            res[(c, K)] = time_it(reps)
+            acc[(c, K)] += time_it(reps)
             got = moe.plan()
             assert (got["c"], got["K"]) == (c, K), (got, c, K)
             steal_of[f"{c},{K}"] = got["n_steal"]
+    res = {pt: v / 2 for pt, v in acc.items()}
+    t_pick = res[(plan["c"], plan["K"])]
     tables_for(tables["c_min"], tables["c_max"], tables["c_step"])
     best = min(res, key=res.get)
     moe.set_model_options(7, -1)
@@ -210,15 +214,15 @@ def grid_sweep(moe, xl, cfg, tables, verbose=True, c_points=C_POINTS, reps=3):
     moe.set_schedule(pk.SCHED_AUTO)
     if verbose:
         print("grid (us):")
-        for c in c_points:
+        for c in cs:
             print(f"  c={c:3d} " + " ".join(f"K={K}:{res.get((c, K), float('nan')):8.1f} (steal {steal_of.get(f'{c},{K}', '-')})"
                                             for K in K_POINTS))
         print(f"AUTO (all plan kinds) {plan_auto} -> {t_auto:.1f} us; measured optimum of the split grid {best} -> "
               f"{res[best]:.1f} us; AUTO vs that {100 * (t_auto / res[best] - 1):+.1f} %; SERIAL {t_serial:.1f} us")
-        print(f"model's split pick {plan}: {t_pick:.1f} us, selection gap inside the grid {100 * (t_pick / min(res[best], t_pick) - 1):.1f} %; "
+        print(f"model's split pick {plan}: {t_pick:.1f} us, selection gap inside the grid {100 * (t_pick / res[best] - 1):.1f} %; "
               f"set-up {su_auto:.2f} us with the search, {su_fixed:.2f} us without")
     return {"workload": cfg.name, "auto_us": t_auto, "plan_auto": plan_auto, "plan": plan, "best": list(best),
-            "best_us": min(res[best], t_pick), "pick_us": t_pick, "selection_gap": t_pick / min(res[best], t_pick) - 1,
+            "best_us": res[best], "pick_us": t_pick, "selection_gap": t_pick / res[best] - 1,
             "auto_vs_best": t_auto / res[best] - 1, "serial_us": t_serial, "setup_us_auto": su_auto,
             "setup_us_fixed": su_fixed, "grid_points": len(res), "steal_of": steal_of}
 

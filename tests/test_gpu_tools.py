@@ -94,10 +94,10 @@ def test_grid_sweep_compares_the_model_s_pick_with_the_forced_grid():
     cfg = wl.CONFIGS["c4_dsv2lite_T256"]
     moe, xl, tab = calibrate.calibrate(cfg, verbose=False)
     rep = calibrate.grid_sweep(moe, xl, cfg, tab, verbose=False, c_points=(4, 16, 48), reps=2)
-    assert rep["grid_points"] == 3 * 4
+    assert rep["grid_points"] in (3 * 4, 4 * 4)          # the model's pick joins the grid when it is not on it
     assert rep["plan"]["kind"] == pk.PLAN_SPLIT and 2 <= rep["plan"]["c"] <= tab["n_sm"] // 2
     assert np.isfinite(rep["selection_gap"]) and rep["selection_gap"] >= 0.0
-    assert rep["best_us"] > 0 and rep["pick_us"] >= rep["best_us"] * 0.999
+    assert rep["best_us"] > 0 and rep["pick_us"] >= rep["best_us"]
     # the steal quota moves with c: fewer movement SMs finish later, so less is left to steal
     steals = {c: rep["steal_of"][f"{c},1"] for c in (4, 16, 48)}
     assert steals[4] <= steals[16] <= steals[48]
