@@ -218,6 +218,18 @@ int weave_moe_status(weave_moe_t h);
  * Diagnostic only. */
 int weave_moe_last_timeout_where(weave_moe_t h);
 
+/* Post-mortem of the launch whose failure the last weave_moe_status() reported.  Every bounded wait
+ * that ended without success - its own limit ran out, or it saw the abort word another wait had raised -
+ * left a record in its warp's slot.  Copies up to max_records records of six ints to `out` (host):
+ * {CTA, warp, wait id (as weave_moe_last_timeout_where), the object waited on (for a shared-memory
+ * barrier its address, whose low 10 bits are the barrier's byte offset among the CTA's barriers; for
+ * a ready flag the low 32 bits of its device address), the parity or count waited for, 1 = this
+ * wait's limit ran out / 2 = cut short by the abort word}.  Returns the number of records there
+ * are (may exceed max_records), 0 when the last status was clean.  Diagnostic only: which warps
+ * waited for what when the launch stopped.  (A device-side wait that fails is the only failure
+ * injected or observed on the GPU; nothing traps or faults.) */
+int weave_moe_debug_wait_log(weave_moe_t h, int32_t *out, int max_records);
+
 /* Upper bound, in milliseconds, for any single in-kernel wait (grid barrier, ready flag,
  * mbarrier); after it the kernel records WEAVE_ERR_TIMEOUT and every CTA returns.  Default 4000. */
 int weave_moe_set_timeout_ms(weave_moe_t h, int ms);

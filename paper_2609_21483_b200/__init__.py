@@ -65,6 +65,7 @@ EXPORTS = [
     "weave_moe_set_expert_parallel", "weave_moe_get_ep_descriptors",
     "weave_moe_forward_host_pipelined", "weave_moe_host_wait", "weave_moe_debug_gemm_queue",
     "weave_moe_get_plan_kind", "weave_moe_set_model_options", "weave_moe_last_timeout_where",
+    "weave_moe_debug_wait_log",
 ]
 
 
@@ -105,6 +106,8 @@ def load():
     lib.weave_moe_set_model_options.argtypes = [vp, ci, ci]
     lib.weave_moe_last_timeout_where.restype = ci
     lib.weave_moe_last_timeout_where.argtypes = [vp]
+    lib.weave_moe_debug_wait_log.restype = ci
+    lib.weave_moe_debug_wait_log.argtypes = [vp, vp, ci]
     lib.weave_moe_get_geometry.restype = ci
     lib.weave_moe_get_geometry.argtypes = [vp, cip, cip, cip, cip, cip, cip, cip]
     lib.weave_moe_get_routing.restype = ci
@@ -316,6 +319,14 @@ class WeaveMoE:
     def last_timeout_where(self) -> int:
         return int(self._lib.weave_moe_last_timeout_where(self._h))
 
+    def wait_log(self):
+        """Records {cta, warp, wait id, object, wanted, how} of the waits that failed in the launch whose
+        failure the last status() reported."""
+        n = int(self._lib.weave_moe_debug_wait_log(self._h, None, 0))
+        buf = (ctypes.c_int32 * (6 * max(n, 1)))()
+        n = min(n, int(self._lib.weave_moe_debug_wait_log(self._h, buf, n)))
+        return [tuple(buf[6 * i:6 * i + 6]) for i in range(n)]
+
     def geometry(self):
         v = [ctypes.c_int() for _ in range(7)]
         _check(self._lib.weave_moe_get_geometry(self._h, *[ctypes.byref(a) for a in v]), "weave_moe_get_geometry")
@@ -366,7 +377,7 @@ class WeaveMoE:
     def check(self):
         st = self.status()
         if st != WEAVE_OK:
-            raise WeaveError(st, f"device status (wait id {self._lib.weave_moe_last_cuda_error(self._h)})")
+            raise WeaveError(st, f"device status (wait id {self._lib.weave_moe_last_timeout_where(self._h)})")
 
     def set_expert_parallel(self, ep_rank: int, ep_size: int):
         """Act as rank ep_rank of ep_size (see weave_moe_set_expert_parallel); ep_size = 1 = off."""

@@ -125,6 +125,7 @@ struct KParams {
     const float *tf;      // [n_sm+1] FLOP/us
     uint4 *trace;         // optional [n_sm][trace_cap] event records (nullptr = off)
     int trace_cap;
+    int4 *wait_log;       // [n_sm][8 warps]: written only by a wait that gives up or is cut short by the abort word
 };
 
 struct TileInfo {
@@ -206,6 +207,19 @@ __device__ __noinline__ void give_up(Ctl *ctl, int where)
     atomicExch(&ctl->abort, 1u);
 }
 
+// Post-mortem of a failed launch: every wait that ends without success (its own limit ran out, or it saw
+// the abort word another wait had raised) leaves {wait id, what it waited on (shared-memory address of the
+// barrier or low bits of the flag's address), the parity or target it waited for, 1 = timed out / 2 = cut
+// short} in its warp's slot (the warp's first such wait only).  Together the slots show who was waiting
+// for whom when the launch stopped.
+__device__ __noinline__ void note_failed_wait(int4 *log, int where, unsigned what, unsigned want, int how)
+{
+    // the first failed wait of a warp is the one that tells where it stood; what it runs into afterwards,
+    // on its way out with the abort word set, is not recorded
+    if (log && log[blockIdx.x * 8 + (threadIdx.x >> 5)].w == 0)
+        log[blockIdx.x * 8 + (threadIdx.x >> 5)] = make_int4(where, (int)what, (int)want, how);
+}
+
 // Optional timeline: one 16-byte record {start ns, end ns, kind<<24 | id, extra} per event, per CTA.
 enum { kEvRoute = 1, kEvSetup = 2, kEvFixup = 3, kEvDispatch = 4, kEvGemmLoad = 5, kEvGemmEpi = 6,
        kEvCombine = 7, kEvWaitChunk = 8, kEvBarrier = 9, kEvMma = 11 };
@@ -234,11 +248,12 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, const 
     unsigned it = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++it & 31u) == 0u) {
-            if (ld_relaxed_u32(&p.ctl->abort)) return false;
+            if (ld_relaxed_u32(&p.ctl->abort)) { note_failed_wait(p.wait_log, where, smem_u32(bar), parity, 2); return false; }
             const unsigned long long now = globaltimer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > p.timeout_ns) {
+            else if ((long long)(now - t0) > (long long)p.timeout_ns) {     // signed: a timer that steps back is not a time-out
                 give_up(p.ctl, where);
+                note_failed_wait(p.wait_log, where, smem_u32(bar), parity, 1);
                 return false;
             }
         }
@@ -254,11 +269,15 @@ __device__ __forceinline__ bool flag_wait_ge(const unsigned *flag, unsigned targ
     while (ld_acquire_u32(flag) < target) {
         __nanosleep(40);
         if ((++it & 31u) == 0u) {
-            if (ld_relaxed_u32(&p.ctl->abort)) return false;
+            if (ld_relaxed_u32(&p.ctl->abort)) {
+                note_failed_wait(p.wait_log, where, (unsigned)(size_t)flag, target, 2);
+                return false;
+            }
             const unsigned long long now = globaltimer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > p.timeout_ns) {
+            else if ((long long)(now - t0) > (long long)p.timeout_ns) {
                 give_up(p.ctl, where);
+                note_failed_wait(p.wait_log, where, (unsigned)(size_t)flag, target, 1);
                 return false;
             }
         }
@@ -948,6 +967,23 @@ __device__ __forceinline__ float silu_mul(float g, float u)
     return __fdividef(g, 1.0f + __expf(-g)) * u;
 }
 
+// A consumer of the tile-descriptor ring hands its slot back with a barrier arrival, after which the
+// scheduler (for the peer CTA: a thread of ANOTHER CTA, through remote stores) may overwrite the slot.
+// The copy of the descriptor must have LANDED in this thread's registers by then.  Program order alone
+// does not say so: the arrival has CTA scope (a cluster-scope release would wait for the thread's
+// global stores, ~1000 cycles) and no instruction reads the loaded words before it is issued, so the
+// shared-memory loads can still be in flight when the slot is rewritten.  Storing a fold of all eight
+// words to a scratch word makes the hardware wait for them here: a store cannot issue before its
+// operand has arrived, and the arrival is issued after the store.  (An empty asm statement that
+// merely names the words generates no instruction and therefore no wait.)
+// Seen without it, about once in 300 000 launches and only in the peer CTA: warps reading different
+// row counts for one swapped tile, the up/gate exchange of its epilogue running out of step, the
+// accumulator never handed back, a bounded wait running out.
+__device__ __forceinline__ void tile_info_landed(const TileInfo &ti, int *scratch)
+{
+    *reinterpret_cast<volatile int *>(scratch) = ti.type ^ ti.mb ^ ti.row0 ^ ti.nrows ^ ti.e ^ ti.n ^ ti.chunk ^ ti.nkb;
+}
+
 // bounded wait on a barrier whose guarded data may come from the peer CTA
 __device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity, const KParams &p, int where)
 {
@@ -956,11 +992,12 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity
     unsigned it = 0;
     while (!mbar_try_wait_cluster(bar, parity)) {
         if ((++it & 31u) == 0u) {
-            if (ld_relaxed_u32(&p.ctl->abort)) return false;
+            if (ld_relaxed_u32(&p.ctl->abort)) { note_failed_wait(p.wait_log, where, smem_u32(bar), parity, 2); return false; }
             const unsigned long long now = globaltimer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > p.timeout_ns) {
+            else if ((long long)(now - t0) > (long long)p.timeout_ns) {
                 give_up(p.ctl, where);
+                note_failed_wait(p.wait_log, where, smem_u32(bar), parity, 1);
                 return false;
             }
         }
@@ -1077,6 +1114,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
             if (lane == 0) ok = mbar_wait_cluster(&S.ti_full[ps.slot], ps.slot_phase, p, 35);
             if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
             const TileInfo ti = S.ti[ps.slot];
+            tile_info_landed(ti, &S.scan_w[warp]);
             __syncwarp();
             if (lane == 0) mbar_arrive_remote(mapa_u32(smem_u32(&S.ti_empty[ps.slot]), 0u));
             ps.next_slot();
@@ -1137,6 +1175,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
             if (lane == 0) ok = mbar_wait(&S.ti_full[ps.slot], ps.slot_phase, p, 40);
             if (!__all_sync(0xffffffffu, ok)) { dead = true; break; }
             const TileInfo ti = S.ti[ps.slot];
+            tile_info_landed(ti, &S.scan_w[warp]);
             __syncwarp();
             if (lane == 0) mbar_arrive(&S.ti_empty[ps.slot]);
             ps.next_slot();
@@ -1198,6 +1237,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
             dead = __any_sync(0xffffffffu, dead);
             if (dead) break;
             const TileInfo ti = S.ti[ps.slot];
+            tile_info_landed(ti, &S.scan_w[warp]);
             __syncwarp();
             if (lane == 0) mbar_arrive_remote(mapa_u32(smem_u32(&S.ti_empty[ps.slot]), 0u));
             ps.next_slot();
@@ -1374,6 +1414,8 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
             if (!mbar_wait(&S.rel_full[rs], rph, p, 57)) break;
             unsigned *flag = S.rel_flag[rs];
             const unsigned cnt = S.rel_cnt[rs];
+            // both words have landed before the slot goes back (see tile_info_landed)
+            *reinterpret_cast<volatile int *>(&S.scan_w[warp]) = (int)cnt ^ (int)(size_t)flag;
             __syncwarp();
             if (lane == 0) mbar_arrive(&S.rel_empty[rs]);
             if (cnt == kRelEnd) break;

@@ -20,8 +20,10 @@ namespace {
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+constexpr int kWaitLogSlots = 1024 * 8;      // one slot per warp of up to 1024 CTAs
+
 struct Layout {
-    size_t ctl, fcnt, xe_ready, h_ready, zero_end;       // [0, zero_end) is zeroed at create / recovery
+    size_t ctl, fcnt, xe_ready, h_ready, wait_log, zero_end;       // [0, zero_end) is zeroed at create / recovery
     size_t hist, topk, gates, row_of, token_of, counts, offsets, bw, tf, uniq_mask, xs;
     size_t xe, hbuf, y, st_x, st_logits, st_out, st2_x, st2_logits, st2_out, total;
     int nmb_max, nblk_max, p_max;
@@ -58,6 +60,7 @@ Layout make_layout(const weave_moe_config *c)
     L.fcnt = take(sizeof(unsigned) * kFine * kMaxEE, 256);
     L.xe_ready = take(sizeof(unsigned) * L.nmb_max, 256);
     L.h_ready = take(sizeof(unsigned) * L.nmb_max, 256);
+    L.wait_log = take(sizeof(int4) * kWaitLogSlots, 256);     // written by failed waits only, cleared by the host
     L.zero_end = align_up(o, 256);
     L.hist = take(sizeof(int) * (size_t)L.nblk_max * kMaxEE, 256);
     L.topk = take(sizeof(int) * T * c->top_k, 256);
@@ -105,6 +108,7 @@ struct weave_moe {
     cudaStream_t last_stream;
     int last_cuda_error;
     int last_timeout_where;
+    std::vector<int32_t> *wait_log;     // records of the last failed launch: {cta, warp, wait id, object, wanted, how}
     int kinds;         // plan kinds AUTO may choose (bit mask)
     int elastic;       // -1 = on under AUTO only, 0 = off, 1 = on
     const float *bw_dev, *tf_dev;     // cost tables on the device (in the workspace unless set otherwise)
@@ -239,6 +243,7 @@ int weave_moe_create(const weave_moe_config *cfg, weave_moe_t *out)
     h->last_stream = nullptr;
     h->last_cuda_error = 0;
     h->last_timeout_where = 0;
+    h->wait_log = new (std::nothrow) std::vector<int32_t>();
     h->kinds = 7;
     h->elastic = -1;
     h->bw_dev = reinterpret_cast<const float *>(h->ws + L.bw);
@@ -342,6 +347,7 @@ int weave_moe_forward(weave_moe_t h, const void *x, const float *logits, void *o
     p.uniq_mask = reinterpret_cast<unsigned long long *>(ws + L.uniq_mask);
     p.trace = reinterpret_cast<uint4 *>(h->trace);
     p.trace_cap = h->trace_cap;
+    p.wait_log = reinterpret_cast<int4 *>(ws + L.wait_log);
 
     void *args[] = {&p, &h->tm};
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -449,6 +455,7 @@ int weave_moe_destroy(weave_moe_t h)
         cudaStreamDestroy(h->pipe_h2d);
         cudaStreamDestroy(h->pipe_d2h);
     }
+    if (h) delete h->wait_log;
     delete h;
     return WEAVE_OK;
 }
@@ -565,6 +572,17 @@ int weave_moe_status(weave_moe_t h)
     if (e != cudaSuccess) return cuda_fail(h, e);
     int st = ctl.status;
     if (st != 0) {
+        // keep what the failed waits wrote down, for weave_moe_debug_wait_log()
+        if (h->wait_log) {
+            std::vector<int4> raw(kWaitLogSlots);
+            h->wait_log->clear();
+            if (cudaMemcpy(raw.data(), h->ws + h->L.wait_log, sizeof(int4) * kWaitLogSlots, cudaMemcpyDeviceToHost) == cudaSuccess)
+                for (int i = 0; i < kWaitLogSlots; ++i)
+                    if (raw[i].w != 0) {
+                        const int32_t rec[6] = {i / 8, i % 8, raw[i].x, raw[i].y, raw[i].z, raw[i].w};
+                        h->wait_log->insert(h->wait_log->end(), rec, rec + 6);
+                    }
+        }
         // a failed launch may have left flags behind: start from a clean slate
         e = cudaMemset(h->ws, 0, h->L.zero_end);
         if (e != cudaSuccess) return cuda_fail(h, e);
@@ -634,6 +652,16 @@ int weave_moe_set_trace(weave_moe_t h, void *buf, int events_per_cta)
 int weave_moe_last_cuda_error(weave_moe_t h) { return h ? h->last_cuda_error : 0; }
 
 int weave_moe_last_timeout_where(weave_moe_t h) { return h ? h->last_timeout_where : 0; }
+
+int weave_moe_debug_wait_log(weave_moe_t h, int32_t *out, int max_records)
+{
+    if (!h || max_records < 0 || (max_records > 0 && !out)) return WEAVE_ERR_INVALID_ARG;
+    if (!h->wait_log) return 0;
+    const int n = (int)(h->wait_log->size() / 6);
+    for (int i = 0; i < n && i < max_records; ++i)
+        for (int j = 0; j < 6; ++j) out[i * 6 + j] = (*h->wait_log)[(size_t)i * 6 + j];
+    return n;
+}
 
 int weave_moe_debug_gemm_queue(const int32_t *rows, int num_segments, int num_chunks, int nt0, int nt1, int32_t *out,
                                int max_tiles)

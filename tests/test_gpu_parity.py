@@ -466,6 +466,13 @@ def test_bounded_wait_gives_up_and_handle_recovers():
     moe.debug_withhold_flag(1)
     moe.forward(dev[0], dev[1])
     assert moe.status() == pk.ERR_TIMEOUT
+    # the post-mortem: the GEMM scheduler that waited for the m-block's rows (wait id 31) is in it, one
+    # wait ran out (not necessarily that one: a warp that idled behind it started its clock earlier)
+    # and the others were cut short by the abort word
+    log = moe.wait_log()
+    assert any(r[2] == 31 for r in log) and all(r[5] in (1, 2) for r in log)
+    assert sum(1 for r in log if r[5] == 1) >= 1 and moe.last_timeout_where() in {r[2] for r in log if r[5] == 1}
+    assert all(0 <= r[0] < moe.geometry()["n_sm"] and 0 <= r[1] < 8 for r in log)
     moe.debug_withhold_flag(-1)
     moe.set_timeout_ms(4000)
     run_case(cfg, inp=inp, dev_tensors=dev, moe=moe)
