@@ -307,7 +307,7 @@ class Layer:
     def schedules(self):
         pk = self.pk
         return {
-            "auto": ((pk.SCHED_AUTO, 0, 1, 0), 7, -1),                    # the model over every plan kind
+            "auto": ((pk.SCHED_AUTO, 0, 1, 0), 7, -1),                    # the model over its default plan kinds
             "auto_split": ((pk.SCHED_AUTO, 0, 1, 0), 1, -1),              # the paper's plan kind only
             "fixed": ((pk.SCHED_FIXED, self.fixed_c, 1, 0), 7, 0),        # static 15 % split, nothing else
             "fixed_elastic": ((pk.SCHED_FIXED, self.fixed_c, 1, 0), 7, 1),  # ... plus elastic stealing and the first dispatch wave
@@ -373,21 +373,24 @@ class Layer:
         clocks = sampler.stop()
         return sec / n / self.L, sec, clocks
 
-    def ablation(self, step_s, rounds=3):
-        """The schedules take turns (round robin, the order rotating from round to round), so that clock
-        and power drift over the run and whatever the previous schedule left in L2 hit them alike.  The
-        part runs under its power cap and the clock follows the last ~50 ms of load: each measurement is
-        preceded by that much of its own schedule."""
+    def ablation(self, step_s, rounds=4):
+        """The schedules take turns.  The part runs under its power cap and the clock follows the last
+        ~50 ms of load, so a schedule measured right after a slow (cool) one looks faster: each
+        measurement is preceded by ~50 ms of its own schedule, and the order changes from round to
+        round so that every schedule follows a different predecessor each time (round r walks the list
+        with stride r + 1: with five schedules the four strides give four different predecessors)."""
         names = list(self.schedules())
+        n = len(names)
         n_abl = max(2, min(5, int(0.25 / step_s) + 1))
         warm = max(1, min(20, int(0.05 / step_s) + 1))
-        tot = {n: 0.0 for n in names}
+        tot = {nm: 0.0 for nm in names}
         for r in range(rounds):
-            k = r % len(names)
-            for name in names[k:] + names[:k]:
+            stride = r % (n - 1) + 1
+            for j in range(n):
+                name = names[(2 * r + j * stride) % n]
                 self.set(name)
                 tot[name] += self.timed(self.step_dev, n_abl, warm)
-        res = {n + "_us_per_layer": s / (n_abl * rounds) / self.L * 1e6 for n, s in tot.items()}
+        res = {nm + "_us_per_layer": s / (n_abl * rounds) / self.L * 1e6 for nm, s in tot.items()}
         res["fixed_c"] = self.fixed_c
         self.set("auto")
         self.moe.check()

@@ -159,7 +159,7 @@ int weave_moe_get_plan(weave_moe_t h, int *c, int *K, int *n_steal, float *t_tot
 /* Plan kinds.  SPLIT is the paper's execution plan (Section 3.3, Eq. 15): c movement SMs next to
  * N - c GEMM SMs from the first tile on.  The paper's movement crosses NVLink; here it is a copy
  * inside one GPU's memory that all SMs can do at full speed, so AUTO's arg-min (Eq. 16) also ranges
- * over two kinds the paper has no use for, costed from the same tables BW(.), TFLOPS(.), eff_chunk,
+ * over three kinds the paper has no use for, costed from the same tables BW(.), TFLOPS(.), eff_chunk,
  * alpha:
  *   DISPATCH_ALL  every SM dispatches, then c SMs combine chunk by chunk while N - c run the GEMMs:
  *                 T = W_disp/BW(N) + max(T_comp(c,K) + T_tail(c,K), W_comb/BW(c))
@@ -167,16 +167,23 @@ int weave_moe_get_plan(weave_moe_t h, int *c, int *K, int *n_steal, float *t_tot
  *                 then combines (tile-level ready flags, no grid barrier between the phases):
  *                 T = W_disp/BW(N) + W_comp/TFLOPS(N) + (1-alpha) * W_comb/BW(N);  reported as
  *                 c = n_sm, K = 1, n_steal = 0.
- * Ties go to SPLIT, then to the smaller c, then to the smaller K.  The steal quota of Eq. 11-14
+ *   REJOIN        the split in which the c movement SMs return to the GEMM queue for good once the
+ *                 dispatch is done (they take GEMM tiles whenever no combine chunk is ready; no
+ *                 quota) and every GEMM CTA dispatches one m-block before its first tile; K = 1:
+ *                 t_d = W_disp/BW(c), W_during = min(t_d * TFLOPS(N-c), 2/3 W_comp)  (the work done
+ *                 meanwhile, as Eq. 12, capped at the gate/up tiles' share, which the queue runs first),
+ *                 T = t_d + max(0, W_comp - W_during)/TFLOPS(N) + (1-alpha) * W_comb/BW(N).
+ * Ties go to SPLIT, then DISPATCH_ALL, PHASED, REJOIN, then to the smaller c, then to the smaller K.  The steal quota of Eq. 11-14
  * belongs to SPLIT; the other kinds report n_steal = 0.  FIXED always runs SPLIT; SERIAL reports
  * PHASED (it is the same order of work with a grid barrier between the phases). */
-enum { WEAVE_PLAN_SPLIT = 0, WEAVE_PLAN_DISPATCH_ALL = 1, WEAVE_PLAN_PHASED = 2 };
+enum { WEAVE_PLAN_SPLIT = 0, WEAVE_PLAN_DISPATCH_ALL = 1, WEAVE_PLAN_PHASED = 2, WEAVE_PLAN_REJOIN = 3 };
 
 /* Kind of the plan of the most recent forward.  Synchronises the handle's last stream. */
 int weave_moe_get_plan_kind(weave_moe_t h, int *kind);
 
-/* kinds_mask: which plan kinds AUTO's arg-min may choose (bit 1 << WEAVE_PLAN_*; default all
- * three; 1 = the paper's split only; must be non-zero).  elastic: whether movement SM pairs keep
+/* kinds_mask: which plan kinds AUTO's arg-min may choose (bit 1 << WEAVE_PLAN_*; default 7 = SPLIT,
+ * DISPATCH_ALL and PHASED; 15 adds REJOIN, which measured no better than PHASED on this hardware;
+ * 1 = the paper's split only; must be non-zero).  elastic: whether movement SM pairs keep
  * taking GEMM tiles beyond their steal quota while no combine chunk is ready, and GEMM CTAs
  * dispatch one m-block before their first GEMM tile: 1 = on, 0 = off, -1 = the default (on under
  * AUTO, off under FIXED, so that FIXED is the plain static split of the paper's ablation).

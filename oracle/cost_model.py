@@ -20,8 +20,14 @@ them; on one GPU, where movement is an HBM copy that all SMs can do at full spee
             T = W_disp/BW(N) + max(T_comp(c,K) + T_tail(c,K), W_comb/BW(c))
     kind 2, "phased": all SMs per phase, no spatial split (the paper's "w/o S+T" ablation as a
             candidate):  T = W_disp/BW(N) + W_comp/TFLOPS(N) + (1-alpha) * W_comb/BW(N)
+    kind 3, "split with rejoin" (K = 1): c SMs dispatch while N-c run GEMM tiles; when the dispatch
+            is done the c SMs join the GEMM queue for good; the final combine runs on all SMs:
+            t_d = W_disp/BW(c),  W_during = min(t_d * TFLOPS(N-c), 2/3 W_comp)  (as Eq. 12; the 2/3 are
+            the gate/up FLOPs, 4HI of 6HI per row, which the queue runs first: a dispatch that outlasts
+            them holds the GEMM SMs up),
+            T = t_d + max(0, W_comp - W_during)/TFLOPS(N) + (1-alpha) * W_comb/BW(N)
 They take part in the arg-min only when CostTables.kinds has their bit set; ties go to the
-paper's kind, then to the smaller c, then to the smaller K.
+paper's kind, then kinds 1, 2, 3 in that order, then to the smaller c, then to the smaller K.
 
 Units: work in FLOPs / bytes, rates in FLOP/us and byte/us, times in us.
 Parity: pinned by closed forms in tests/test_oracle_cost_model.py.  The values
@@ -38,7 +44,7 @@ import numpy as np
 
 f32 = np.float32
 K_CANDIDATES = (1, 2, 4, 8)
-KIND_SPLIT, KIND_DISPATCH_ALL, KIND_PHASED = 0, 1, 2
+KIND_SPLIT, KIND_DISPATCH_ALL, KIND_PHASED, KIND_REJOIN = 0, 1, 2, 3
 
 
 @dataclass
@@ -57,7 +63,7 @@ class CostTables:
     max_segments: int = 0    # a build that keeps a table of (chunk, expert) segments bounds the chunk
                              # count: candidates with K * n_experts > max_segments are skipped (0 = no bound)
     kinds: int = 1           # bit mask of the plan kinds in the arg-min: 1 = the paper's split (Eq. 15),
-                             # 2 = dispatch on all SMs then split, 4 = phased
+                             # 2 = dispatch on all SMs then split, 4 = phased, 8 = split with rejoin
 
 
 @dataclass
@@ -119,6 +125,15 @@ def t_total_phased(tab: CostTables, w_comp, w_disp, w_comb) -> np.float32:
     return (w_disp / bw + w_comp / tf) + (f32(1.0) - f32(tab.alpha)) * (w_comb / bw)
 
 
+def t_total_rejoin(tab: CostTables, c: int, w_comp, w_disp, w_comb) -> np.float32:
+    """Kind 3 (K = 1): the GEMM SMs' work during the dispatch as in Eq. 12, the rest on all N SMs."""
+    n = tab.n_sm
+    t_disp = w_disp / f32(tab.bw[c])
+    w_during = np.minimum(t_disp * f32(tab.tflops[n - c]), w_comp * f32(0.6666667))
+    w_rest = np.maximum(f32(0.0), w_comp - w_during)
+    return (t_disp + w_rest / f32(tab.tflops[n])) + (f32(1.0) - f32(tab.alpha)) * (w_comb / f32(tab.bw[n]))
+
+
 def candidates(tab: CostTables):
     c = tab.c_min
     while c <= tab.c_max and c <= tab.n_sm - 1:
@@ -171,6 +186,11 @@ def plan(tab: CostTables, T: int, P: int, H: int, I: int, n_tiles_of_K: Sequence
         t = t_total_phased(tab, w_comp, w_disp, w_comb)
         if best is None or t < best[0]:
             best = (t, tab.n_sm, 0, KIND_PHASED)
+    if (tab.kinds >> KIND_REJOIN) & 1:
+        for c in candidates(tab):
+            t = t_total_rejoin(tab, c, w_comp, w_disp, w_comb)
+            if best is None or t < best[0]:
+                best = (t, c, 0, KIND_REJOIN)
     t, c, ki, kind = best
     steal = n_steal(tab, c, w_comp, w_disp, w_comb, n_tiles_of_K[ki]) if kind == KIND_SPLIT else 0
     return Plan(c, K_CANDIDATES[ki], steal, float(t), kind)

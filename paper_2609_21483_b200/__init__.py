@@ -19,7 +19,7 @@ _SOURCES = ["weave_moe.cu", "weave_kernel.cuh", "weave_ptx.cuh"]
 WEAVE_OK = 0
 WEAVE_ERR_INVALID_ARG = -1
 SCHED_AUTO, SCHED_FIXED, SCHED_SERIAL = 0, 1, 2
-PLAN_SPLIT, PLAN_DISPATCH_ALL, PLAN_PHASED = 0, 1, 2
+PLAN_SPLIT, PLAN_DISPATCH_ALL, PLAN_PHASED, PLAN_REJOIN = 0, 1, 2, 3
 ERR_NONFINITE_LOGITS, ERR_TIMEOUT = -5, -6
 
 _lib = None
@@ -312,7 +312,7 @@ class WeaveMoE:
         return {"c": c.value, "K": K.value, "n_steal": s.value, "t_total_us": t.value, "kind": kind.value}
 
     def set_model_options(self, kinds_mask: int = 7, elastic: int = -1):
-        """Plan kinds AUTO may choose (bit 0 the paper's split, bit 1 dispatch-all, bit 2 phased) and
+        """Plan kinds AUTO may choose (bit 0 the paper's split, bit 1 dispatch-all, bit 2 phased, bit 3 rejoin) and
         the elastic-stealing switch (-1 = on under AUTO only)."""
         _check(self._lib.weave_moe_set_model_options(self._h, kinds_mask, elastic), "weave_moe_set_model_options")
 

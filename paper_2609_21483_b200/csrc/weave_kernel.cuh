@@ -83,8 +83,10 @@ constexpr int kCtlZeroWords = 24;
 // SMs can do at full speed: kPlanDispatchAll lets every SM dispatch before the roles split (only the
 // combine is left to the movement SMs), kPlanPhased has no roles at all (every SM dispatches, then
 // runs GEMM tiles until the queue is empty, then combines; the ready flags still order the tiles,
-// no grid barrier separates the phases).
-enum { kPlanSplit = 0, kPlanDispatchAll = 1, kPlanPhased = 2 };
+// no grid barrier separates the phases).  kPlanRejoin is the split in which the movement SMs come back to
+// the GEMM queue for good once the dispatch is done (no steal quota: they take GEMM tiles whenever no
+// combine chunk is ready) and every GEMM CTA dispatches one m-block before its first tile; K = 1.
+enum { kPlanSplit = 0, kPlanDispatchAll = 1, kPlanPhased = 2, kPlanRejoin = 3 };
 
 struct KParams {
     int T, H, I, E, S, k, EE;
@@ -169,6 +171,7 @@ struct SmemTail {
     int scan_w[8];
     int scan_total;
     int c, K, steal, nmb, n_gemm, n_comb;
+    int elastic;                 // this launch: movement pairs take GEMM tiles beyond their quota, GEMM CTAs dispatch one m-block first
     int comb_tok;                // tokens per combine tile of this launch: 16, 8, 4, 2 or 1
     unsigned trace_n;
     int chunk_mb0[kFine + 1];
@@ -524,6 +527,21 @@ __device__ __forceinline__ float model_t_dispatch_all(const KParams &p, float bw
 __device__ __forceinline__ float model_t_phased(const KParams &p, float bw_n, float tf_n, float w_comp, float w_disp, float w_comb)
 {
     return __fadd_rn(__fadd_rn(__fdiv_rn(w_disp, bw_n), __fdiv_rn(w_comp, tf_n)),
+                     __fmul_rn(__fsub_rn(1.0f, p.alpha), __fdiv_rn(w_comb, bw_n)));
+}
+
+// Plan kind "split with rejoin": while c SMs dispatch (W_disp / BW(c)), N - c SMs run GEMM tiles (the work
+// done meanwhile as in Eq. 12, but no more than the gate/up tiles of the layer, 4HI of the 6HI FLOPs per
+// row: the queue runs them first and a down tile needs its m-block's gate/up tiles, so a dispatch that
+// outlasts them holds the GEMM SMs up); what is left then runs on all N SMs; the final combine is on all
+// N SMs.
+__device__ __forceinline__ float model_t_rejoin(const KParams &p, float bw, float tf, float bw_n, float tf_n, float w_comp,
+                                                float w_disp, float w_comb)
+{
+    const float t_disp = __fdiv_rn(w_disp, bw);
+    const float w_during = fminf(__fmul_rn(t_disp, tf), __fmul_rn(w_comp, 0.6666667f));
+    const float w_rest = fmaxf(0.0f, __fsub_rn(w_comp, w_during));
+    return __fadd_rn(__fadd_rn(t_disp, __fdiv_rn(w_rest, tf_n)),
                      __fmul_rn(__fsub_rn(1.0f, p.alpha), __fdiv_rn(w_comb, bw_n)));
 }
 
@@ -1052,7 +1070,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
         // kTinfo tiles ahead of the MMAs, so claim and flag latencies stay off the critical path.
         if (lane == 0) {
             int taken = 0;
-            int g_next = (budget > 0 || p.elastic_steal) ? (int)atomicAdd(&p.ctl->q_gemm, 1u) : 0x7fffffff;
+            int g_next = (budget > 0 || S.elastic) ? (int)atomicAdd(&p.ctl->q_gemm, 1u) : 0x7fffffff;
             for (;;) {
                 const int g = g_next;
                 const unsigned long long tp0 = trace_now(p);
@@ -1070,7 +1088,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                 if (tl.type != 2) {
                     ++taken;
                     bool more = taken < budget;
-                    if (!more && p.elastic_steal) {
+                    if (!more && S.elastic) {
                         // the steal quota is used up: keep taking GEMM tiles for as long as the next
                         // combine chunk has not been produced yet (nothing else to do meanwhile)
                         const unsigned qc = ld_relaxed_u32(&p.ctl->q_comb);
@@ -1285,6 +1303,9 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                             const uint4 t4 = ld_shared_v4(xs + (uint32_t)(lane * 64 + i * 16));
                             u[4 * i] = t4.x; u[4 * i + 1] = t4.y; u[4 * i + 2] = t4.z; u[4 * i + 3] = t4.w;
                         }
+                        // the four vector loads have landed before the region is handed back to the up warp
+                        // (see tile_info_landed: the values are not used until after the arrival)
+                        *reinterpret_cast<volatile int *>(&S.scan_w[warp]) = (int)(u[0] ^ u[4] ^ u[8] ^ u[12]);
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&S.xg_empty);
 #pragma unroll
@@ -1576,7 +1597,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
             w_comb = __fmul_rn((float)(P + p.T), B);
         }
         // candidate order = (kind, c ascending, K ascending), index = kind * 256 + thread; the phased plan
-        // is index 512; ties go to the smaller index
+        // is index 512, the rejoin plans follow it; ties go to the smaller index
         float t = __int_as_float(0x7f800000);
         int bi = tid;
         if (cm_ok && (p.kinds & (1 << kPlanSplit))) t = model_t_total(p, cm_bw, cm_tf, cm_ki, w_comp, w_disp, w_comb);
@@ -1587,6 +1608,10 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
         if (tid == 0 && (p.kinds & (1 << kPlanPhased))) {
             const float t2 = model_t_phased(p, cm_bw_n, cm_tf_n, w_comp, w_disp, w_comb);
             if (t2 < t) { t = t2; bi = 2 * kThreads; }
+        }
+        if (cm_ok && cm_ki == 0 && (p.kinds & (1 << kPlanRejoin))) {      // K = 1 only
+            const float t3 = model_t_rejoin(p, cm_bw, cm_tf, cm_bw_n, cm_tf_n, w_comp, w_disp, w_comb);
+            if (t3 < t) { t = t3; bi = 3 * kThreads + tid; }
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
@@ -1646,6 +1671,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
         plan_kind = kPlanPhased;
     }
     const int K = 1 << plan_ki;
+    if (tid == 0) S.elastic = (p.elastic_steal || plan_kind == kPlanRejoin) ? 1 : 0;
     {
         const int g = kFine / K;
         int run_row = tid < EE ? off : 0;
@@ -1763,10 +1789,11 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
             // scheduling" ablation keeps the two groups apart
             // (plan kinds beyond the paper's: every CTA works through the dispatch queue first; in the
             // phased plan every CTA is a "mover" without a steal limit)
-            const int dmax = (mover || plan_kind != kPlanSplit) ? 0x7fffffff : (p.elastic_steal ? 1 : 0);
+            const bool two_roles = plan_kind == kPlanSplit || plan_kind == kPlanRejoin;
+            const int dmax = (mover || !two_roles) ? 0x7fffffff : (S.elastic ? 1 : 0);
             if (dmax > 0) dispatch_phase(p, S, stages, dmax);
             const int budget = (mover && plan_kind != kPlanPhased) ? plan_steal : 0x7fffffff;
-            if (budget > 0 || p.elastic_steal) gemm_phase(p, S, stages, tmem_base, &tm, budget, ps);
+            if (budget > 0 || S.elastic) gemm_phase(p, S, stages, tmem_base, &tm, budget, ps);
             combine_phase(p, S, stages);
         }
     }

@@ -244,7 +244,7 @@ int weave_moe_create(const weave_moe_config *cfg, weave_moe_t *out)
     h->last_cuda_error = 0;
     h->last_timeout_where = 0;
     h->wait_log = new (std::nothrow) std::vector<int32_t>();
-    h->kinds = 7;
+    h->kinds = 7;       // split, dispatch-all, phased; the rejoin kind is opt-in (weave_moe_set_model_options)
     h->elastic = -1;
     h->bw_dev = reinterpret_cast<const float *>(h->ws + L.bw);
     h->tf_dev = reinterpret_cast<const float *>(h->ws + L.tf);
@@ -519,7 +519,7 @@ int weave_moe_get_plan_kind(weave_moe_t h, int *kind)
 
 int weave_moe_set_model_options(weave_moe_t h, int kinds_mask, int elastic)
 {
-    if (!h || (kinds_mask & 7) == 0 || (kinds_mask & ~7) || elastic < -1 || elastic > 1) return WEAVE_ERR_INVALID_ARG;
+    if (!h || (kinds_mask & 15) == 0 || (kinds_mask & ~15) || elastic < -1 || elastic > 1) return WEAVE_ERR_INVALID_ARG;
     h->kinds = kinds_mask;
     h->elastic = elastic;
     return WEAVE_OK;

@@ -104,7 +104,7 @@ def test_plan_uses_the_paper_s_workload_terms_in_ep_mode():
         g = 8 // K
         tiles.append(sum(int(((fine[j * g:(j + 1) * g].sum(0) + geo["gemm_tile_m"] - 1) // geo["gemm_tile_m"]).sum())
                          for j in range(K)) * nt)
-    for kinds in (7, 1):      # all plan kinds (the default), then the paper's split alone
+    for kinds in (7, 15, 1):      # the default kinds, all four, the paper's split alone
         moe.set_model_options(kinds, -1)
         moe.forward(x, lg)
         moe.check()

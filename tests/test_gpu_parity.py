@@ -384,9 +384,10 @@ def _fine_counts(ref, cfg, geo):
     return fine
 
 
-@pytest.mark.parametrize("name,kinds,c_step", [("c1_tiny", 1, 2), ("c1_tiny", 7, 2), ("c4_dsv2lite_T256", 7, 2),
-                                               ("c4_dsv2lite_T256", 1, 4), ("t1_qwen35_35b_T2048", 7, 4),
-                                               ("t1_qwen35_35b_T2048", 3, 2)])
+@pytest.mark.parametrize("name,kinds,c_step", [("c1_tiny", 1, 2), ("c1_tiny", 15, 2), ("c4_dsv2lite_T256", 7, 2),
+                                               ("c4_dsv2lite_T256", 1, 4), ("c4_dsv2lite_T256", 9, 2),
+                                               ("t1_qwen35_35b_T2048", 15, 4), ("t1_qwen35_35b_T2048", 3, 2),
+                                               ("t1_qwen35_35b_T2048", 8, 2)])
 def test_device_plan_equals_cpu_cost_model(name, kinds, c_step):
     """AUTO's plan (kind, c*, K*, n_steal) must equal the CPU restatement of Eq. 1-16 fed the same
     tables: with the paper's plan kind alone (kinds = 1) and with the added kinds, on a candidate grid
@@ -431,7 +432,7 @@ def test_device_plan_equals_cpu_cost_model(name, kinds, c_step):
         assert abs(got["t_total_us"] - want.t_total) <= 1e-6 * want.t_total
         assert EE * got["K"] <= 1024
         seen.add(got["kind"])
-    assert seen <= {k for k in range(3) if (kinds >> k) & 1}
+    assert seen <= {k for k in range(4) if (kinds >> k) & 1}
     moe.close()
 
 

@@ -78,7 +78,7 @@ def test_calibration_produces_usable_tables_and_auto_follows_them():
     p = moe.plan()
     assert p["kind"] == pk.PLAN_SPLIT
     assert 2 <= p["c"] <= n // 2 and p["c"] % 2 == 0 and p["K"] in (1, 2, 4, 8) and p["t_total_us"] > 0
-    moe.set_model_options(7, -1)                          # every kind: the phased plan reports c = n_sm
+    moe.set_model_options(7, -1)                          # the default kinds: the phased plan reports c = n_sm
     moe.forward(x, lg)
     moe.check()
     q = moe.plan()

@@ -204,3 +204,46 @@ def test_dispatch_all_kind_closed_form_and_tie_order():
     tabf = cm.CostTables(N, np.full(N + 1, 1e30, np.float32), flat, np.ones(4, np.float32), 0.0, kinds=7)
     pf = cm.plan(tabf, T, P, H, I, [10] * 4)
     assert (pf.kind, pf.c, pf.K) == (cm.KIND_SPLIT, 2, 1)
+
+
+def test_rejoin_kind_closed_forms():
+    """Kind 3: t_d = W_disp/BW(c); the N-c GEMM SMs do t_d*TFLOPS(N-c) meanwhile; the rest runs on N SMs.
+    (a) With LINEAR curves the time does not depend on c and equals the phased time: by hand
+        t_d + (A*f - f*(N-c)*t_d)/(f*N) = A/N + t_d*c/N = A/N + W_disp/(b*N), A = W_comp/f.  Phased comes
+        first in the candidate order, so it keeps the tie.
+    (b) With a concave GEMM curve, TFLOPS(n) = F*sqrt(n/N), the time is t_d*(1 - sqrt((N-c)/N)) + W_comp/F
+        + tail while the GEMMs outlast the dispatch: less than the phased time, minimal at some c that
+        the hand formula gives.
+    (c) Slow dispatch: only the gate/up tiles (2/3 of the FLOPs) can run meanwhile; T = t_d + the down tiles
+        on N SMs + the combine tail."""
+    N = 148
+    T, P, H, I = 8192, 65536, 2048, 768
+    w_comp, w_disp, w_comb = (float(v) for v in cm.workloads(T, P, H, I))
+    b, f = 40.0e3, 8.0e6
+    lin = _toy(N, b, f, kinds=8)
+    A = w_comp / f
+    for c in (24, 32, 74):        # (with these the dispatch ends before 2/3 of the GEMM work is done: c/(N-c) > 0.147)
+        t = float(cm.t_total_rejoin(lin, c, *cm.workloads(T, P, H, I)))
+        assert math.isclose(t, A / N + w_disp / (b * N) + w_comb / (b * N), rel_tol=1e-5)
+    # two dispatch SMs: only the gate/up tiles (2/3 of the work) can run meanwhile, the down tiles follow on N SMs
+    t2 = float(cm.t_total_rejoin(lin, 2, *cm.workloads(T, P, H, I)))
+    assert math.isclose(t2, w_disp / (b * 2) + (A / 3) / N + w_comb / (b * N), rel_tol=1e-5)
+    both = _toy(N, b, f, kinds=4 | 8)
+    assert cm.plan(both, T, P, H, I, [10] * 4).kind == cm.KIND_PHASED
+    # (b) TFLOPS(n) = F * sqrt(n / N)
+    idx = np.arange(N + 1, dtype=np.float64)
+    F = 1.2e9
+    conc = cm.CostTables(N, (b * idx).astype(np.float32), (F * np.sqrt(idx / N)).astype(np.float32),
+                         np.ones(4, np.float32), 0.0, kinds=4 | 8)
+    p = cm.plan(conc, T, P, H, I, [10] * 4)
+    assert p.kind == cm.KIND_REJOIN and p.K == 1 and p.n_steal == 0
+    hand = lambda c: (w_disp / (b * c)) * (1.0 - math.sqrt((N - c) / N)) + w_comp / F + w_comb / (b * N) \
+        if (w_disp / (b * c)) * F * math.sqrt((N - c) / N) < 2 * w_comp / 3 else w_disp / (b * c) + w_comp / (3 * F) + w_comb / (b * N)
+    best_c = min(range(2, 75, 2), key=hand)
+    assert math.isclose(p.t_total, hand(best_c), rel_tol=1e-4) and abs(p.c - best_c) <= 2
+    phased = w_disp / (b * N) + w_comp / F + w_comb / (b * N)
+    assert p.t_total < phased
+    # (c) two dispatch SMs at a crawl: the other 146 finish the GEMMs long before
+    slow = _toy(N, b=10.0, f=1e9, kinds=8, c_min=2, c_max=2)
+    p = cm.plan(slow, T, P, H, I, [10] * 4)
+    assert math.isclose(p.t_total, w_disp / 20.0 + (w_comp / 3) / (1e9 * N) + w_comb / (10.0 * N), rel_tol=1e-5)
