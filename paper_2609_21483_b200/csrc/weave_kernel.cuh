@@ -362,9 +362,9 @@ __device__ __forceinline__ int block_excl_scan(int v, SmemTail &S, int &total)
 // Four threads route one token, so a CTA's 256 threads take a whole 64-token block at once and no
 // lane idles.  The block's logits are staged in shared memory (row stride = 4 mod 32 words, so the
 // 32 lanes of a warp - eight tokens x four threads - hit 32 different banks).  Thread q of a quad
-// scans experts q, q+4, ... in ascending order and keeps its KC >= k best in a sorted register list;
-// the four lists are then merged k times through two shuffle steps.  Order: larger logit first,
-// equal logits by lower expert index (-0 == +0); gates = softmax over the selected k.
+// holds experts q, q+4, ... as order keys in registers; the k selections are k rounds of arg-max over
+// the quad (see route_block_rounds).  Order: larger logit first, equal logits by lower expert index
+// (-0 == +0); gates = softmax over the selected k.
 
 // fp32 -> uint32 that orders like the float (finite values; -0 has been folded into +0)
 __device__ __forceinline__ unsigned float_order_key(float v)
@@ -386,16 +386,30 @@ __device__ __forceinline__ void stage_logits(const KParams &p, int b, float *lg_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ntok = min(kRouteBlock, p.T - b * kRouteBlock);
     const int stride = route_row_stride(p.E);
-    for (int r = warp; r < ntok; r += kThreads / 32) {
-        const float *src = p.logits + (size_t)(b * kRouteBlock + r) * p.E;
-        for (int c = lane; c < p.E; c += 32) cp_async_4(smem_u32(lg_s + r * stride + c), src + c);
+    if ((p.E & 3) == 0) {      // rows are 16-byte multiples: both sides of every copy are 16-byte aligned
+        const int per_row = p.E >> 2;
+        for (int i = threadIdx.x; i < ntok * per_row; i += kThreads) {
+            const int r = i / per_row, c = (i - r * per_row) << 2;
+            cp_async_16(smem_u32(lg_s + r * stride + c), p.logits + (size_t)(b * kRouteBlock + r) * p.E + c);
+        }
+    } else {
+        for (int r = warp; r < ntok; r += kThreads / 32) {
+            const float *src = p.logits + (size_t)(b * kRouteBlock + r) * p.E;
+            for (int c = lane; c < p.E; c += 32) cp_async_4(smem_u32(lg_s + r * stride + c), src + c);
+        }
     }
     cp_async_wait_all();
 }
 
-template <int KC>
-__device__ __forceinline__ void route_block_quads(const KParams &p, int b, const float *lg_s, unsigned long long *r_mask,
-                                                  int *r_idx, int *r_cnt)
+// Top-k selection by k rounds of arg-max, four threads (a quad) per token.  Thread q of a quad holds
+// the order keys of experts q, q+4, ... in NPT registers and knows its own best (largest key, lowest expert index among equals).  A round:
+// the quad's best of the four bests (two shuffle steps; equal keys go to the lower expert index) is
+// slot j; its owner clears it and rescans its registers (two independent chains, so that the compare
+// latencies overlap).  No sorted lists, no divergent inserts.  r_p: [64][16] floats of scratch for the
+// exponentials (the sum is only known after the last round).
+template <int NPT>
+__device__ __forceinline__ void route_block_rounds(const KParams &p, int b, const float *lg_s, unsigned long long *r_mask,
+                                                   int *r_idx, int *r_cnt, float *r_p)
 {
     static_assert(kThreads == 4 * kRouteBlock, "four threads per token of a routing block");
     const int tl = threadIdx.x >> 2, q = threadIdx.x & 3;
@@ -405,85 +419,80 @@ __device__ __forceinline__ void route_block_quads(const KParams &p, int b, const
     const int e_lo = p.ep_size > 1 ? p.ep_rank * (p.E / p.ep_size) : 0;
     const int e_hi = p.ep_size > 1 ? e_lo + p.E / p.ep_size : p.E;
 
-    // keys: 0 = empty slot; every finite logit maps to a key >= 1 that orders like the float
-    unsigned key[KC];
-    int idx[KC];
-#pragma unroll
-    for (int j = 0; j < KC; ++j) { key[j] = 0u; idx[j] = 0x7fffffff; }
+    // keys: 0 = nothing there; every finite logit maps to a key >= 1 that orders like the float
+    unsigned key[NPT];
     bool bad = false;
-    if (valid) {
-        for (int e = q; e < p.E; e += 4) {
+#pragma unroll
+    for (int i = 0; i < NPT; ++i) {
+        const int e = q + 4 * i;
+        unsigned c = 0u;
+        if (valid && e < p.E) {
             float x = lg_s[tl * stride + e];
             if (!(fabsf(x) <= 3.402823466e38f)) {   // NaN or +-inf: flag it, keep indices in range
                 bad = true;
                 x = -3.402823466e38f;
             }
             x = __fadd_rn(x, 0.0f);                  // folds -0 into +0, leaves everything else alone
-            const unsigned c = float_order_key(x);
-            if (c > key[KC - 1]) {
-                // insert behind every entry that is >= c (they have lower indices): from the bottom,
-                // an entry smaller than c moves down one slot, and c lands above the first such entry
-#pragma unroll
-                for (int j = KC - 1; j >= 1; --j) {
-                    if (c > key[j - 1]) { key[j] = key[j - 1]; idx[j] = idx[j - 1]; }
-                    else if (c > key[j]) { key[j] = c; idx[j] = e; }
-                }
-                if (c > key[0]) { key[0] = c; idx[0] = e; }
-            }
+            c = float_order_key(x);
         }
+        key[i] = c;
     }
     if (__any_sync(0xffffffffu, bad) && (threadIdx.x & 31) == 0) atomicCAS(&p.ctl->status, 0, kErrNonFinite);
 
-    // merge: slot j = the best head of the quad's four lists; its owner pops it
-    unsigned sel_key[KC];
-    int sel_idx[KC];
+    // this thread's best: two chains over the even and the odd registers, strict '>' keeps the lower index
+    auto rescan = [&](unsigned &bk, int &bi) {
+        unsigned k0 = key[0], k1 = NPT > 1 ? key[1] : 0u;
+        int i0 = 0, i1 = 1;
 #pragma unroll
-    for (int j = 0; j < KC; ++j) {
-        sel_key[j] = 0u; sel_idx[j] = 0;
-        if (j < p.k) {
-            unsigned hk = key[0];
-            int hi = idx[0];
+        for (int i = 2; i < NPT; i += 2) {
+            if (key[i] > k0) { k0 = key[i]; i0 = i; }
+            if (i + 1 < NPT && key[i + 1] > k1) { k1 = key[i + 1]; i1 = i + 1; }
+        }
+        const bool odd = k1 > k0 || (k1 == k0 && i1 < i0);
+        bk = odd ? k1 : k0;
+        bi = odd ? i1 : i0;
+    };
+    unsigned bk;
+    int bi;
+    rescan(bk, bi);
+
+    float vmax = 0.f, sum = 0.f;
+    int nloc = 0;
+    for (int j = 0; j < p.k; ++j) {
+        unsigned hk = bk;
+        int hi = bk ? q + 4 * bi : 0x7fffffff;
 #pragma unroll
-            for (int o = 1; o <= 2; o <<= 1) {
-                const unsigned ok = __shfl_xor_sync(0xffffffffu, hk, o);
-                const int oi = __shfl_xor_sync(0xffffffffu, hi, o);
-                if (ok > hk || (ok == hk && oi < hi)) { hk = ok; hi = oi; }
-            }
-            sel_key[j] = hk; sel_idx[j] = hi;
-            if (hi == idx[0]) {
+        for (int o = 1; o <= 2; o <<= 1) {
+            const unsigned ok = __shfl_xor_sync(0xffffffffu, hk, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, hi, o);
+            if (ok > hk || (ok == hk && oi < hi)) { hk = ok; hi = oi; }
+        }
+        // every thread of the quad knows slot j now; thread j mod 4 writes it down
+        const float v = float_from_order_key(hk);
+        if (j == 0) vmax = v;
+        const float pj = expf(v - vmax);
+        sum += pj;                                   // slot order
+        // expert-parallel share: only the experts hosted here get rows; the gates stay normalised over
+        // all k selected experts
+        const bool local = hi >= e_lo && hi < e_hi;
+        nloc += local ? 1 : 0;
+        if (valid && (j & 3) == q) {
+            p.topk_idx[(size_t)t * p.k + j] = hi;
+            r_p[tl * kMaxTopK + j] = pj;
+            r_idx[tl * kMaxTopK + j] = local ? hi : -1;
+            if (local) atomicOr(reinterpret_cast<unsigned *>(&r_mask[hi]) + (tl >> 5), 1u << (tl & 31));
+        }
+        // the owner takes its winner out and looks for its next best
+        if ((hi & 3) == q && hk != 0u) {
 #pragma unroll
-                for (int i = 0; i + 1 < KC; ++i) { key[i] = key[i + 1]; idx[i] = idx[i + 1]; }
-                key[KC - 1] = 0u; idx[KC - 1] = 0x7fffffff;
-            }
+            for (int i = 0; i < NPT; ++i)
+                if (i == bi) key[i] = 0u;
+            rescan(bk, bi);
         }
     }
-
+    __syncwarp();
     if (valid) {
-        // every thread of the quad holds all k selections; thread q writes slots q, q+4, ...
-        const float vmax = float_from_order_key(sel_key[0]);
-        float pj[KC];
-        float sum = 0.f;
-#pragma unroll
-        for (int j = 0; j < KC; ++j) {
-            pj[j] = 0.f;
-            if (j < p.k) { pj[j] = expf(float_from_order_key(sel_key[j]) - vmax); sum += pj[j]; }   // slot order
-        }
-        int nloc = 0;
-#pragma unroll
-        for (int j = 0; j < KC; ++j) {
-            if (j < p.k) {
-                // expert-parallel share: only the experts hosted here get rows; the gates stay
-                // normalised over all k selected experts
-                const bool local = sel_idx[j] >= e_lo && sel_idx[j] < e_hi;
-                nloc += local ? 1 : 0;
-                if ((j & 3) == q) {
-                    p.topk_idx[(size_t)t * p.k + j] = sel_idx[j];
-                    p.gates[(size_t)t * p.k + j] = __fdiv_rn(pj[j], sum);
-                    r_idx[tl * kMaxTopK + j] = local ? sel_idx[j] : -1;
-                    if (local) atomicOr(reinterpret_cast<unsigned *>(&r_mask[sel_idx[j]]) + (tl >> 5), 1u << (tl & 31));
-                }
-            }
-        }
+        for (int j = q; j < p.k; j += 4) p.gates[(size_t)t * p.k + j] = __fdiv_rn(r_p[tl * kMaxTopK + j], sum);
         if (p.ep_size > 1 && q == 0 && nloc) {
             if (t / p.ep_tshard == p.ep_rank) atomicAdd(&r_cnt[0], nloc);
             else {
@@ -653,7 +662,9 @@ __device__ __forceinline__ unsigned y_done_target(const SmemTail &S, const KPara
 // writes each full buffer to its (contiguous) destination rows with one bulk store.  About 96 KB
 // of loads and as much of stores are in flight per SM.  The m-block's ready flag is released once
 // its last store has completed.
-__device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, uint8_t *stages, int max_tiles)
+// n_disp = number of CTAs that take part in the dispatch of this launch: CTA i's first tile is m-block i
+// (no queue round trip before the first copy), later claims go through the queue, which starts at n_disp.
+__device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, uint8_t *stages, int max_tiles, int n_disp)
 {
     MoveScratch &M = move_scratch(stages);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -723,10 +734,12 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
             ph = __shfl_sync(0xffffffffu, ph, 0);
         }
         for (int taken = 0; ok && taken < max_tiles; ++taken) {
-            int mb = 0;
-            if (lane == 0) mb = (int)atomicAdd(&p.ctl->q_disp, 1u);
-            mb = __shfl_sync(0xffffffffu, mb, 0);
-            if (mb >= S.nmb) break;
+            int mb = (int)blockIdx.x;
+            if (taken > 0) {
+                if (lane == 0) mb = n_disp + (int)atomicAdd(&p.ctl->q_disp, 1u);
+                mb = __shfl_sync(0xffffffffu, mb, 0);
+            }
+            if (mb >= S.nmb) { if (taken > 0) break; else continue; }
             int row0, nrows;
             decode_mblock(S, p.EE, mb, row0, nrows);
             for (int i = lane; i < nrows; i += 32) M.tok[i] = __ldcg(p.token_of + row0 + i);
@@ -1508,6 +1521,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
     int *r_base = reinterpret_cast<int *>(stages + 2048 + 64 + kRouteBlock * kMaxTopK * 4);    // [256]
     int *r_cnt = r_base + kMaxEE;                                                          // [2] local / remote pairs
     float *lg_s = reinterpret_cast<float *>(stages + 8192);                                // [64][route_row_stride(E)]
+    float *r_p = reinterpret_cast<float *>(stages + 80 * 1024);                            // [64][16] exponentials of the selected logits
 
     // ================= phase R: routing
     for (int b = blockIdx.x; b < p.nblk; b += n_sm) {
@@ -1516,10 +1530,10 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
         __syncthreads();
         stage_logits(p, b, lg_s);
         __syncthreads();
-        if (p.k <= 2) route_block_quads<2>(p, b, lg_s, r_mask, r_idx, r_cnt);
-        else if (p.k <= 4) route_block_quads<4>(p, b, lg_s, r_mask, r_idx, r_cnt);
-        else if (p.k <= 8) route_block_quads<8>(p, b, lg_s, r_mask, r_idx, r_cnt);
-        else route_block_quads<16>(p, b, lg_s, r_mask, r_idx, r_cnt);
+        if (p.E <= 16) route_block_rounds<4>(p, b, lg_s, r_mask, r_idx, r_cnt, r_p);
+        else if (p.E <= 64) route_block_rounds<16>(p, b, lg_s, r_mask, r_idx, r_cnt, r_p);
+        else if (p.E <= 128) route_block_rounds<32>(p, b, lg_s, r_mask, r_idx, r_cnt, r_p);
+        else route_block_rounds<64>(p, b, lg_s, r_mask, r_idx, r_cnt, r_p);
         __syncthreads();
         // in-block rank of each (token, slot): tokens before it in the block that chose the same expert
         for (int pi = tid; pi < kRouteBlock * p.k; pi += kThreads) {
@@ -1566,6 +1580,10 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
         cf[f] = (alive && tid < EE) ? (int)__ldcg(p.fcnt + f * kMaxEE + tid) : 0;
         cnt += cf[f];
     }
+    // (asked for together with the counts: one L2 round trip instead of two)
+    const bool ep_on = alive && p.ep_size > 1;
+    const unsigned ep_xl = ep_on ? __ldcg(&p.ctl->x_local) : 0u, ep_xi = ep_on ? __ldcg(&p.ctl->x_in) : 0u,
+                   ep_xu = ep_on ? __ldcg(&p.ctl->x_in_uniq) : 0u;
     int total_rows;
     const int off = block_excl_scan(cnt, S, total_rows);
     if (tid < EE) S.offsets[tid] = off;
@@ -1576,8 +1594,6 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
         if (tid == 0) p.offsets[EE] = total_rows;
     }
     const int P = p.T * (p.k + p.S);
-    const unsigned ep_xl = alive ? __ldcg(&p.ctl->x_local) : 0u, ep_xi = alive ? __ldcg(&p.ctl->x_in) : 0u,
-                   ep_xu = alive ? __ldcg(&p.ctl->x_in_uniq) : 0u;
     if (blockIdx.x == 0 && tid == 0) { p.ctl->ep_x_local = ep_xl; p.ctl->ep_x_in = ep_xi; p.ctl->ep_x_in_uniq = ep_xu; }
     int plan_c, plan_ki, plan_steal, plan_kind = kPlanSplit;
     float plan_t = 0.f;
@@ -1733,6 +1749,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
     // ================= permutation fix-up: in-block rank + rows of earlier blocks + expert offset
     if (alive) {
         int fixed = 0;
+        const bool one_block = p.nblk <= n_sm;
         for (int b = blockIdx.x; b < p.nblk; b += n_sm) {
             const int f = (b * kFine) / p.nblk;
             const int bstart = (f * p.nblk + kFine - 1) / kFine;
@@ -1748,8 +1765,11 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
                 const int tl = pi / p.k, j = pi - tl * p.k;
                 const int t = b * kRouteBlock + tl;
                 if (t < p.T) {
-                    const int e = __ldcg(p.topk_idx + (size_t)t * p.k + j);
-                    const int rk = __ldcg(p.row_of + (size_t)t * p.k + j);
+                    // with at most one routing block per CTA the block's selections and masks are still in
+                    // shared memory (one L2 round trip less on the way to the first dispatch tile)
+                    const int e = one_block ? r_idx[tl * kMaxTopK + j] : __ldcg(p.topk_idx + (size_t)t * p.k + j);
+                    const int rk = one_block ? (e >= 0 ? __popcll(r_mask[e] & ((1ull << tl) - 1ull)) : -1)
+                                             : __ldcg(p.row_of + (size_t)t * p.k + j);
                     if (rk >= 0) {
                         const int r = rk + r_base[e];
                         p.row_of[(size_t)t * p.k + j] = r;
@@ -1776,7 +1796,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
     PipeState ps;
     if (alive) {
         if (p.mode == kModeSerial) {
-            dispatch_phase(p, S, stages, 0x7fffffff);
+            dispatch_phase(p, S, stages, 0x7fffffff, n_sm);
             alive = grid_barrier(p, S, 2u * n_sm, 2);
             if (alive) gemm_phase(p, S, stages, tmem_base, &tm, 0x7fffffff, ps);
             alive = alive && grid_barrier(p, S, 3u * n_sm, 3);
@@ -1791,7 +1811,8 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
             // phased plan every CTA is a "mover" without a steal limit)
             const bool two_roles = plan_kind == kPlanSplit || plan_kind == kPlanRejoin;
             const int dmax = (mover || !two_roles) ? 0x7fffffff : (S.elastic ? 1 : 0);
-            if (dmax > 0) dispatch_phase(p, S, stages, dmax);
+            const int n_disp = (!two_roles || S.elastic) ? n_sm : plan_c;       // who dispatches at all
+            if (dmax > 0) dispatch_phase(p, S, stages, dmax, n_disp);
             const int budget = (mover && plan_kind != kPlanPhased) ? plan_steal : 0x7fffffff;
             if (budget > 0 || S.elastic) gemm_phase(p, S, stages, tmem_base, &tm, budget, ps);
             combine_phase(p, S, stages);
