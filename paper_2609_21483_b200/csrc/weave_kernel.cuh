@@ -34,6 +34,7 @@ constexpr int kStageB = 128 * kBK * 2;                  // 16 KB: this CTA's hal
 constexpr int kStageBytes = kStageA + kStageB;          // 32 KB
 constexpr int kEpiStageBytes = 4 * 2 * 32 * 64;         // epilogue staging: per warp two buffers of 32 rows x 64 bytes
 constexpr int kRouteBlock = 64;  // tokens per routing block (one 64-bit mask per expert)
+constexpr int kLocalBlocks = 2;  // a batch of at most this many routing blocks is routed by every CTA for itself
 constexpr int kCombTile = 16;    // tokens per combine tile (fewer when the batch would give fewer tiles than SMs)
 constexpr int kMaxEE = 256;      // routed + shared experts
 constexpr int kMaxTopK = 16;
@@ -194,6 +195,8 @@ struct MoveScratch {
     float cgate[kCombTile][kMaxTopK + 8];
 };
 static_assert(sizeof(MoveScratch) <= kEpiStageBytes / 2, "movement scratch must fit half of the staging area");
+static_assert(kLocalBlocks * (kMaxEE + 1) * 8 <= kEpiStageBytes / 2, "the routing masks must fit the other half");
+static_assert(kFine == 8, "chunk of a fine chunk = f >> (3 - log2 K)");
 __device__ __forceinline__ MoveScratch &move_scratch(uint8_t *stages)
 {
     return *reinterpret_cast<MoveScratch *>(stages + kStages * kStageBytes + kEpiStageBytes / 2);
@@ -238,6 +241,11 @@ __device__ __forceinline__ void trace_ev(const KParams &p, SmemTail &S, int kind
 __device__ __forceinline__ unsigned long long trace_now(const KParams &p)
 {
     return p.trace ? globaltimer_ns() : 0ull;
+}
+// the same for the CTA-wide phases, whose records thread 0 writes: the other threads do not read the timer
+__device__ __forceinline__ unsigned long long trace_now_t0(const KParams &p)
+{
+    return (p.trace && threadIdx.x == 0) ? globaltimer_ns() : 0ull;
 }
 
 // Every wait is bounded: it polls the global abort word and a wall-clock limit, and returns false
@@ -359,12 +367,13 @@ __device__ __forceinline__ int block_excl_scan(int v, SmemTail &S, int &total)
 
 // ------------------------------------------------------------------------------------ phase R
 
-// Four threads route one token, so a CTA's 256 threads take a whole 64-token block at once and no
-// lane idles.  The block's logits are staged in shared memory (row stride = 4 mod 32 words, so the
-// 32 lanes of a warp - eight tokens x four threads - hit 32 different banks).  Thread q of a quad
-// holds experts q, q+4, ... as order keys in registers; the k selections are k rounds of arg-max over
-// the quad (see route_block_rounds).  Order: larger logit first, equal logits by lower expert index
-// (-0 == +0); gates = softmax over the selected k.
+// Four threads route one token, so a CTA's 256 threads take a whole 64-token block at once and every
+// warp instruction serves eight tokens (a prologue of eight warps per SM is bound by the instructions each
+// warp has to issue, not by their latencies).  The block's logits are staged in shared memory (row stride
+// = 4 mod 32 words, so the 32 lanes of a warp - eight tokens x four threads - hit 32 different banks).
+// Thread q of a quad holds experts q, q+4, ... as order keys in registers; the k selections are k rounds of
+// arg-max over the quad.  Order: larger logit first, equal logits by lower expert index (-0 == +0);
+// gates = softmax over the selected k.
 
 // fp32 -> uint32 that orders like the float (finite values; -0 has been folded into +0)
 __device__ __forceinline__ unsigned float_order_key(float v)
@@ -379,9 +388,10 @@ __device__ __forceinline__ float float_from_order_key(unsigned k)
 
 __device__ __forceinline__ int route_row_stride(int E) { return ((E + 27) / 32) * 32 + 4; }
 
-// cooperative copy of the block's logit rows into shared memory, a warp per row, coalesced; all copies
-// are in flight together (one memory round trip); the caller's __syncthreads() publishes them
-__device__ __forceinline__ void stage_logits(const KParams &p, int b, float *lg_s)
+// cooperative copy of the block's logit rows into shared memory, coalesced; all copies are in flight
+// together (one memory round trip).  The caller waits (cp_async_wait_all) and publishes them
+// (__syncthreads) when it needs them, and may do other work in between.
+__device__ __forceinline__ void stage_logits_issue(const KParams &p, int b, float *lg_s)
 {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ntok = min(kRouteBlock, p.T - b * kRouteBlock);
@@ -398,19 +408,36 @@ __device__ __forceinline__ void stage_logits(const KParams &p, int b, float *lg_
             for (int c = lane; c < p.E; c += 32) cp_async_4(smem_u32(lg_s + r * stride + c), src + c);
         }
     }
-    cp_async_wait_all();
 }
 
-// Top-k selection by k rounds of arg-max, four threads (a quad) per token.  Thread q of a quad holds
-// the order keys of experts q, q+4, ... in NPT registers and knows its own best (largest key, lowest expert index among equals).  A round:
-// the quad's best of the four bests (two shuffle steps; equal keys go to the lower expert index) is
-// slot j; its owner clears it and rescans its registers (two independent chains, so that the compare
-// latencies overlap).  No sorted lists, no divergent inserts.  r_p: [64][16] floats of scratch for the
-// exponentials (the sum is only known after the last round).
+// Top-k selection of routing block b by k rounds of arg-max.  Thread q of a quad holds the order keys of
+// experts q, q+4, ... in NPT registers and knows its own best (largest key, lowest expert index among
+// equals).  A round: the quad's best of the four bests (two shuffle steps; equal keys go to the lower expert
+// index) is slot j; its owner clears it and rescans its registers.  The scratch arrays come as 32-bit
+// shared-memory addresses.  r_mask[e] (64 bits): bit tl set when token tl of the block selected expert e
+// (an expert hosted here); r_idx[tl][j]: the expert of slot j, -1 when another rank hosts it; r_cnt: local /
+// remote (token, expert) pairs of the block (expert-parallel share only); r_p: [64][16] floats of scratch
+// for the exponentials (the sum is only known after the last round).  write_out: this CTA is the one that
+// writes the block's selections and gates to global memory (every CTA routes a small batch for itself, one
+// of them writes it down).
+// Not inlined: its registers (64 keys per thread at E = 256) stay out of the kernel's own allocation.  What it
+// needs of the kernel's parameters comes by value (a reference would turn every use into a load through
+// the generic window onto the parameter bank), and its shared-memory accesses name the shared space
+// (generic atomics that land in shared memory take a slow path).
+struct RouteArgs {
+    int T, E, k, ep_size, ep_rank, ep_tshard;
+    int *status;
+    int *topk_idx;
+    float *gates;
+};
 template <int NPT>
-__device__ __forceinline__ void route_block_rounds(const KParams &p, int b, const float *lg_s, unsigned long long *r_mask,
-                                                   int *r_idx, int *r_cnt, float *r_p)
+__device__ __noinline__ void route_block_quads(int T, int E, int k, int ep_size, int ep_rank, int ep_tshard, int *status,
+                                               int *topk_idx, float *gates, int b, uint32_t lg_s, uint32_t r_mask,
+                                               uint32_t r_idx, uint32_t r_cnt, uint32_t r_p, bool write_out)
 {
+    RouteArgs p;      // (scalars in the call: a structure would travel through local memory)
+    p.T = T; p.E = E; p.k = k; p.ep_size = ep_size; p.ep_rank = ep_rank; p.ep_tshard = ep_tshard;
+    p.status = status; p.topk_idx = topk_idx; p.gates = gates;
     static_assert(kThreads == 4 * kRouteBlock, "four threads per token of a routing block");
     const int tl = threadIdx.x >> 2, q = threadIdx.x & 3;
     const int t = b * kRouteBlock + tl;
@@ -420,24 +447,21 @@ __device__ __forceinline__ void route_block_rounds(const KParams &p, int b, cons
     const int e_hi = p.ep_size > 1 ? e_lo + p.E / p.ep_size : p.E;
 
     // keys: 0 = nothing there; every finite logit maps to a key >= 1 that orders like the float
+    // (rows of tokens past the end and columns past E hold stale values: read, then masked)
     unsigned key[NPT];
     bool bad = false;
 #pragma unroll
     for (int i = 0; i < NPT; ++i) {
         const int e = q + 4 * i;
-        unsigned c = 0u;
-        if (valid && e < p.E) {
-            float x = lg_s[tl * stride + e];
-            if (!(fabsf(x) <= 3.402823466e38f)) {   // NaN or +-inf: flag it, keep indices in range
-                bad = true;
-                x = -3.402823466e38f;
-            }
-            x = __fadd_rn(x, 0.0f);                  // folds -0 into +0, leaves everything else alone
-            c = float_order_key(x);
-        }
-        key[i] = c;
+        float x = ld_shared_f32(lg_s + 4u * (uint32_t)(tl * stride + min(e, p.E - 1)));
+        const bool there = valid && e < p.E;
+        const bool nf = !(fabsf(x) <= 3.402823466e38f);      // NaN or +-inf: flag it, keep indices in range
+        bad = bad || (there && nf);
+        x = nf ? -3.402823466e38f : x;
+        x = __fadd_rn(x, 0.0f);                              // folds -0 into +0, leaves everything else alone
+        key[i] = there ? float_order_key(x) : 0u;
     }
-    if (__any_sync(0xffffffffu, bad) && (threadIdx.x & 31) == 0) atomicCAS(&p.ctl->status, 0, kErrNonFinite);
+    if (__any_sync(0xffffffffu, bad) && (threadIdx.x & 31) == 0) atomicCAS(p.status, 0, kErrNonFinite);
 
     // this thread's best: two chains over the even and the odd registers, strict '>' keeps the lower index
     auto rescan = [&](unsigned &bk, int &bi) {
@@ -458,7 +482,7 @@ __device__ __forceinline__ void route_block_rounds(const KParams &p, int b, cons
 
     float vmax = 0.f, sum = 0.f;
     int nloc = 0;
-    for (int j = 0; j < p.k; ++j) {
+    for (int j = 0; j < k; ++j) {
         unsigned hk = bk;
         int hi = bk ? q + 4 * bi : 0x7fffffff;
 #pragma unroll
@@ -477,10 +501,12 @@ __device__ __forceinline__ void route_block_rounds(const KParams &p, int b, cons
         const bool local = hi >= e_lo && hi < e_hi;
         nloc += local ? 1 : 0;
         if (valid && (j & 3) == q) {
-            p.topk_idx[(size_t)t * p.k + j] = hi;
-            r_p[tl * kMaxTopK + j] = pj;
-            r_idx[tl * kMaxTopK + j] = local ? hi : -1;
-            if (local) atomicOr(reinterpret_cast<unsigned *>(&r_mask[hi]) + (tl >> 5), 1u << (tl & 31));
+            st_shared_u32(r_p + 4u * (uint32_t)(tl * kMaxTopK + j), __float_as_uint(pj));
+            if (write_out) {
+                p.topk_idx[(size_t)t * k + j] = hi;
+                st_shared_u32(r_idx + 4u * (uint32_t)(tl * kMaxTopK + j), (uint32_t)(local ? hi : -1));
+            }
+            if (local) red_shared_or_u32(r_mask + 8u * (uint32_t)hi + 4u * (uint32_t)(tl >> 5), 1u << (tl & 31));
         }
         // the owner takes its winner out and looks for its next best
         if ((hi & 3) == q && hk != 0u) {
@@ -492,12 +518,14 @@ __device__ __forceinline__ void route_block_rounds(const KParams &p, int b, cons
     }
     __syncwarp();
     if (valid) {
-        for (int j = q; j < p.k; j += 4) p.gates[(size_t)t * p.k + j] = __fdiv_rn(r_p[tl * kMaxTopK + j], sum);
+        if (write_out)
+            for (int j = q; j < k; j += 4)
+                p.gates[(size_t)t * k + j] = __fdiv_rn(__uint_as_float(ld_shared_u32(r_p + 4u * (uint32_t)(tl * kMaxTopK + j))), sum);
         if (p.ep_size > 1 && q == 0 && nloc) {
-            if (t / p.ep_tshard == p.ep_rank) atomicAdd(&r_cnt[0], nloc);
+            if (t / p.ep_tshard == p.ep_rank) red_shared_add_u32(r_cnt, (uint32_t)nloc);
             else {
-                atomicAdd(&r_cnt[1], nloc);
-                atomicOr(reinterpret_cast<unsigned *>(&r_mask[kMaxEE]) + (tl >> 5), 1u << (tl & 31));
+                red_shared_add_u32(r_cnt + 4u, (uint32_t)nloc);
+                red_shared_or_u32(r_mask + 8u * (uint32_t)kMaxEE + 4u * (uint32_t)(tl >> 5), 1u << (tl & 31));
             }
         }
     }
@@ -509,7 +537,8 @@ __device__ __forceinline__ void route_block_rounds(const KParams &p, int b, cons
 // T_comp = W_comp / (TFLOPS(N-c) * eff_chunk(K))  (Eq. 9),  T_comm = (W_disp + W_comb) / BW(c)  (Eq. 5),
 // T_tail = (1 - alpha) * W_comb / (BW(c) * K)  (Eq. 10),  T_total = max(T_comp + T_tail, T_comm).
 // bw = BW(c), tf = TFLOPS(N - c): the candidate's two table entries
-__device__ __forceinline__ float model_t_total(const KParams &p, float bw, float tf, int ki, float w_comp, float w_disp,
+template <class PB>
+__device__ __forceinline__ float model_t_total(const PB &p, float bw, float tf, int ki, float w_comp, float w_disp,
                                                float w_comb)
 {
     const float Kf = (float)(1 << ki);
@@ -521,7 +550,8 @@ __device__ __forceinline__ float model_t_total(const KParams &p, float bw, float
 
 // Plan kind "dispatch on all SMs, then split": W_disp / BW(N), then Eq. 15 with only the combine left as
 // communication.  bw_n = BW(N).
-__device__ __forceinline__ float model_t_dispatch_all(const KParams &p, float bw, float tf, float bw_n, int ki, float w_comp,
+template <class PB>
+__device__ __forceinline__ float model_t_dispatch_all(const PB &p, float bw, float tf, float bw_n, int ki, float w_comp,
                                                       float w_disp, float w_comb)
 {
     const float Kf = (float)(1 << ki);
@@ -533,7 +563,8 @@ __device__ __forceinline__ float model_t_dispatch_all(const KParams &p, float bw
 }
 
 // Plan kind "phased": dispatch, GEMMs and combine one after the other, each on all N SMs.
-__device__ __forceinline__ float model_t_phased(const KParams &p, float bw_n, float tf_n, float w_comp, float w_disp, float w_comb)
+template <class PB>
+__device__ __forceinline__ float model_t_phased(const PB &p, float bw_n, float tf_n, float w_comp, float w_disp, float w_comb)
 {
     return __fadd_rn(__fadd_rn(__fdiv_rn(w_disp, bw_n), __fdiv_rn(w_comp, tf_n)),
                      __fmul_rn(__fsub_rn(1.0f, p.alpha), __fdiv_rn(w_comb, bw_n)));
@@ -544,7 +575,8 @@ __device__ __forceinline__ float model_t_phased(const KParams &p, float bw_n, fl
 // row: the queue runs them first and a down tile needs its m-block's gate/up tiles, so a dispatch that
 // outlasts them holds the GEMM SMs up); what is left then runs on all N SMs; the final combine is on all
 // N SMs.
-__device__ __forceinline__ float model_t_rejoin(const KParams &p, float bw, float tf, float bw_n, float tf_n, float w_comp,
+template <class PB>
+__device__ __forceinline__ float model_t_rejoin(const PB &p, float bw, float tf, float bw_n, float tf_n, float w_comp,
                                                 float w_disp, float w_comb)
 {
     const float t_disp = __fdiv_rn(w_disp, bw);
@@ -570,6 +602,58 @@ __device__ __forceinline__ int model_n_steal(int n_sm, float bw, float tf, float
     return max(0, min(r, n_tiles));
 }
 
+// Eq. 16: the arg-min of the modelled layer time over the candidate plans, evaluated by the whole CTA (every
+// CTA evaluates it for itself and gets the same answer).  Thread tid owns the split candidate
+// (c, K) = (c_min + (tid >> 2) * c_step, 1 << (tid & 3)) and its "dispatch on all SMs first" and "rejoin"
+// variants; thread 0 also owns the phased plan.  Candidate order = (kind, c ascending, K ascending),
+// index = kind * 256 + thread; the phased plan is index 512, the rejoin plans follow it; ties go to the
+// smaller index.  Contains one __syncthreads(); S.red_f and S.red_i[.][0] carry the reduction.
+struct PlanPick { int c, ki, kind; float t; };
+struct ModelArgs { float alpha, eff[4]; int kinds, c_min, c_step; };     // by value, see RouteArgs
+__device__ __noinline__ PlanPick model_pick(const ModelArgs p, SmemTail &S, int n_sm, float w_comp, float w_disp, float w_comb,
+                                            bool cm_ok, float cm_bw, float cm_tf, float cm_bw_n, float cm_tf_n)
+{
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int cm_ki = tid & 3;
+    float t = __int_as_float(0x7f800000);
+    int bi = tid;
+    if (cm_ok && (p.kinds & (1 << kPlanSplit))) t = model_t_total(p, cm_bw, cm_tf, cm_ki, w_comp, w_disp, w_comb);
+    if (cm_ok && (p.kinds & (1 << kPlanDispatchAll))) {
+        const float t1 = model_t_dispatch_all(p, cm_bw, cm_tf, cm_bw_n, cm_ki, w_comp, w_disp, w_comb);
+        if (t1 < t) { t = t1; bi = kThreads + tid; }
+    }
+    if (tid == 0 && (p.kinds & (1 << kPlanPhased))) {
+        const float t2 = model_t_phased(p, cm_bw_n, cm_tf_n, w_comp, w_disp, w_comb);
+        if (t2 < t) { t = t2; bi = 2 * kThreads; }
+    }
+    if (cm_ok && cm_ki == 0 && (p.kinds & (1 << kPlanRejoin))) {      // K = 1 only
+        const float t3 = model_t_rejoin(p, cm_bw, cm_tf, cm_bw_n, cm_tf_n, w_comp, w_disp, w_comb);
+        if (t3 < t) { t = t3; bi = 3 * kThreads + tid; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float ot = __shfl_xor_sync(0xffffffffu, t, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ot < t || (ot == t && oi < bi)) { t = ot; bi = oi; }
+    }
+    if (lane == 0) { S.red_f[warp] = t; S.red_i[warp][0] = bi; }
+    __syncthreads();
+    t = S.red_f[0]; bi = S.red_i[0][0];
+#pragma unroll
+    for (int w = 1; w < kThreads / 32; ++w) {
+        const float ot = S.red_f[w];
+        const int oi = S.red_i[w][0];
+        if (ot < t || (ot == t && oi < bi)) { t = ot; bi = oi; }
+    }
+    PlanPick r;
+    r.kind = bi / kThreads;
+    const int bt = bi % kThreads;      // the thread that evaluated the winner
+    r.c = r.kind == kPlanPhased ? n_sm : p.c_min + (bt >> 2) * p.c_step;
+    r.ki = r.kind == kPlanPhased ? 0 : (bt & 3);
+    r.t = t;
+    return r;
+}
+
 // ------------------------------------------------------------------------------------ tile decoding
 
 // largest s in [lo, hi) with (seg_mb0[s] - base) * mul <= key   (empty segments share a start)
@@ -582,9 +666,11 @@ __device__ __forceinline__ int seg_search(const SmemTail &S, int lo, int hi, int
     return lo;
 }
 
-__device__ __forceinline__ void decode_mblock(const SmemTail &S, int EE, int mb, int &row0, int &nrows)
+// m-block -> its rows; seg = the (chunk, expert) segment it belongs to (index chunk * EE + expert)
+__device__ __forceinline__ void decode_mblock(const SmemTail &S, int EE, int mb, int &row0, int &nrows, int &seg)
 {
     const int s = seg_search(S, 0, S.K * EE, 0, 1, mb);
+    seg = s;
     const int m = mb - S.seg_mb0[s];
     row0 = S.seg_row0[s] + m * kBM;
     nrows = min(kBM, S.seg_rows[s] - m * kBM);
@@ -664,8 +750,19 @@ __device__ __forceinline__ unsigned y_done_target(const SmemTail &S, const KPara
 // its last store has completed.
 // n_disp = number of CTAs that take part in the dispatch of this launch: CTA i's first tile is m-block i
 // (no queue round trip before the first copy), later claims go through the queue, which starts at n_disp.
-__device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, uint8_t *stages, int max_tiles, int n_disp)
+// local_route (a small batch that every CTA routed for itself): this CTA's copy of the routing blocks'
+// expert masks, [nblk][kMaxEE + 1], sits at the start of the epilogue staging area; the source tokens of a
+// tile are looked up there and nothing is read from the routing outputs in global memory.
+__device__ __forceinline__ int nth_set_bit(unsigned long long m, int r)
 {
+    const unsigned lo = (unsigned)m, hi = (unsigned)(m >> 32);
+    const int cl = __popc(lo);
+    return r < cl ? (int)__fns(lo, 0u, r + 1) : 32 + (int)__fns(hi, 0u, r - cl + 1);
+}
+__device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, uint8_t *stages, int max_tiles, int n_disp,
+                                               bool local_route)
+{
+    const unsigned long long *lmask = local_route ? reinterpret_cast<const unsigned long long *>(stages + kStages * kStageBytes) : nullptr;
     MoveScratch &M = move_scratch(stages);
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     fence_proxy_async();      // the buffers held routing scratch written with ordinary stores
@@ -677,7 +774,7 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
         int b = 0;
         uint32_t ph = 0;
         bool ok = true;
-        if (lane == 0) ok = flag_wait_ge(&p.ctl->fix_done, (unsigned)p.nblk, p, 10);
+        if (lane == 0 && lmask == nullptr) ok = flag_wait_ge(&p.ctl->fix_done, (unsigned)p.nblk, p, 10);
         ok = __shfl_sync(0xffffffffu, ok, 0);
         if (p.ep_size > 1) {
             // expert-parallel share: first every remote token that has an expert here is copied ONCE
@@ -689,7 +786,7 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
                 if (lane == 0) blk = (int)atomicAdd(&p.ctl->q_pull, 1u);
                 blk = __shfl_sync(0xffffffffu, blk, 0);
                 if (blk >= p.nblk) break;
-                const unsigned long long um = __ldcg(p.uniq_mask + blk);
+                const unsigned long long um = lmask ? lmask[blk * (kMaxEE + 1) + kMaxEE] : __ldcg(p.uniq_mask + blk);
                 const int n = __popcll(um);
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
@@ -740,9 +837,29 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
                 mb = __shfl_sync(0xffffffffu, mb, 0);
             }
             if (mb >= S.nmb) { if (taken > 0) break; else continue; }
-            int row0, nrows;
-            decode_mblock(S, p.EE, mb, row0, nrows);
-            for (int i = lane; i < nrows; i += 32) M.tok[i] = __ldcg(p.token_of + row0 + i);
+            int row0, nrows, seg;
+            decode_mblock(S, p.EE, mb, row0, nrows, seg);
+            if (lmask == nullptr) {
+                for (int i = lane; i < nrows; i += 32) M.tok[i] = __ldcg(p.token_of + row0 + i);
+            } else {
+                // row r of expert e = the r-th token that selected it, in token order; a shared expert's
+                // row r is token r
+                const int e = seg % p.EE;
+                for (int i = lane; i < nrows; i += 32) {
+                    int rank = row0 + i - S.offsets[e];
+                    int tok = rank;
+                    if (e < p.E) {
+                        tok = 0;
+                        for (int bb = 0; bb < p.nblk; ++bb) {
+                            const unsigned long long mk = lmask[bb * (kMaxEE + 1) + e];
+                            const int c = __popcll(mk);
+                            if (rank < c) { tok = bb * kRouteBlock + nth_set_bit(mk, rank); break; }
+                            rank -= c;
+                        }
+                    }
+                    M.tok[i] = tok;
+                }
+            }
             __syncwarp();
             for (int r0 = 0; r0 < nrows && ok; r0 += R) {
                 const int nr = min(R, nrows - r0);
@@ -1513,77 +1630,146 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
     tc_fence_after();
     const uint32_t tmem_base = S.tmem_base;
     if (tid == 0) S.trace_n = 0u;
-    const unsigned long long tk0 = trace_now(p);
+    const unsigned long long tk0 = trace_now_t0(p);
 
-    // routing scratch lives in the (not yet used) stage buffers
-    unsigned long long *r_mask = reinterpret_cast<unsigned long long *>(stages);          // [256] + 1 (remote tokens)
-    int *r_idx = reinterpret_cast<int *>(stages + 2048 + 64);                              // [64][16]
-    int *r_base = reinterpret_cast<int *>(stages + 2048 + 64 + kRouteBlock * kMaxTopK * 4);    // [256]
-    int *r_cnt = r_base + kMaxEE;                                                          // [2] local / remote pairs
-    float *lg_s = reinterpret_cast<float *>(stages + 8192);                                // [64][route_row_stride(E)]
-    float *r_p = reinterpret_cast<float *>(stages + 80 * 1024);                            // [64][16] exponentials of the selected logits
+    // Routing scratch.  The expert masks of the routing blocks sit in the first half of the epilogue staging
+    // area: a small batch's masks are still needed while its dispatch copies run through all the stage
+    // buffers.  Everything else lives in the (not yet used) stage buffers.
+    unsigned long long *lmask = reinterpret_cast<unsigned long long *>(stages + kStages * kStageBytes);   // [kLocalBlocks][256 + 1 (remote tokens)]
+    int *r_base = reinterpret_cast<int *>(stages);                                         // [256]
+    int *r_cnt = r_base + kMaxEE;                                                          // [kLocalBlocks][2] local / remote pairs
+    int *r_idx = reinterpret_cast<int *>(stages + 2048);                                   // [kLocalBlocks][64][16]
+    float *lg_s = reinterpret_cast<float *>(stages + 2048 + kLocalBlocks * kRouteBlock * kMaxTopK * 4);   // [64][route_row_stride(E)]
+    float *r_p = reinterpret_cast<float *>(stages + 96 * 1024);                            // [64][16] exponentials of the selected logits
 
-    // ================= phase R: routing
-    for (int b = blockIdx.x; b < p.nblk; b += n_sm) {
-        for (int e = tid; e < EE; e += kThreads) r_mask[e] = 0ull;
-        if (tid == 0) { r_mask[kMaxEE] = 0ull; r_cnt[0] = 0; r_cnt[1] = 0; }
-        __syncthreads();
-        stage_logits(p, b, lg_s);
-        __syncthreads();
-        if (p.E <= 16) route_block_rounds<4>(p, b, lg_s, r_mask, r_idx, r_cnt, r_p);
-        else if (p.E <= 64) route_block_rounds<16>(p, b, lg_s, r_mask, r_idx, r_cnt, r_p);
-        else if (p.E <= 128) route_block_rounds<32>(p, b, lg_s, r_mask, r_idx, r_cnt, r_p);
-        else route_block_rounds<64>(p, b, lg_s, r_mask, r_idx, r_cnt, r_p);
-        __syncthreads();
-        // in-block rank of each (token, slot): tokens before it in the block that chose the same expert
-        for (int pi = tid; pi < kRouteBlock * p.k; pi += kThreads) {
-            const int tl = pi / p.k, j = pi - tl * p.k;
-            const int t = b * kRouteBlock + tl;
-            if (t < p.T) {
-                const int e = r_idx[tl * kMaxTopK + j];     // -1: the expert lives on another rank
-                p.row_of[(size_t)t * p.k + j] = e >= 0 ? __popcll(r_mask[e] & ((1ull << tl) - 1ull)) : -1;
-            }
-        }
-        if (p.ep_size > 1 && tid == 0) {
-            const unsigned long long um = r_mask[kMaxEE];
-            p.uniq_mask[b] = um;
-            if (r_cnt[0]) atomicAdd(&p.ctl->x_local, (unsigned)r_cnt[0]);
-            if (r_cnt[1]) atomicAdd(&p.ctl->x_in, (unsigned)r_cnt[1]);
-            if (um) atomicAdd(&p.ctl->x_in_uniq, (unsigned)__popcll(um));
-        }
-        const int ntok = min(kRouteBlock, p.T - b * kRouteBlock);
-        const int f = (b * kFine) / p.nblk;
-        for (int e = tid; e < EE; e += kThreads) {
-            const int cnt = e < p.E ? __popcll(r_mask[e]) : ntok;
-            p.hist[(size_t)b * kMaxEE + e] = cnt;
-            if (cnt) atomicAdd(&p.fcnt[f * kMaxEE + e], (unsigned)cnt);
-        }
-        __syncthreads();
-    }
+    // A batch of at most kLocalBlocks routing blocks is routed by every CTA for itself: no grid barrier and
+    // no round trip through global memory stand between the logits and the first dispatch copy.  CTA b
+    // writes block b's results down for the combine and the host.  Larger batches: block b is routed by
+    // CTA b mod N, the counts meet in global memory behind a grid barrier.
+    const bool local_route = p.nblk <= kLocalBlocks;
+    const bool ep = p.ep_size > 1;
+
     // The cost tables do not depend on the routing: this thread's candidate (c, K) asks for its two
-    // entries before the barrier, so that their latency is spent waiting there.
+    // entries first of all, and (without an expert-parallel share, whose workload descriptors are counted
+    // while routing) the plan is chosen while the first block's logits are on their way.
     const int cm_ki = tid & 3, cm_c = p.c_min + (tid >> 2) * p.c_step;
     const bool cm_ok = p.mode == kModeAuto && cm_c >= 2 && cm_c <= p.c_max && cm_c <= n_sm - 2 && (EE << cm_ki) <= kMaxSeg;
     float cm_bw = 0.f, cm_tf = 0.f, cm_bw_n = 0.f, cm_tf_n = 0.f;
     if (cm_ok) { cm_bw = p.bw[cm_c]; cm_tf = p.tf[n_sm - cm_c]; }
     if (p.mode == kModeAuto) { cm_bw_n = p.bw[n_sm]; cm_tf_n = p.tf[n_sm]; }
-    const unsigned long long tk1 = trace_now(p);
-    bool alive = grid_barrier(p, S, (unsigned)n_sm, 1);
-    const unsigned long long tk2 = trace_now(p);
-    if (tid == 0) { trace_ev(p, S, kEvRoute, 0u, tk0, tk1, 0u); trace_ev(p, S, kEvBarrier, 1u, tk1, tk2, 0u); }
+    const int P = p.T * (p.k + p.S);
+    // Eq. 1-3 (single-GPU reading: every pair moves through HBM)
+    const float B = (float)(2 * p.H);
+    float w_comp = __fmul_rn(__fmul_rn(__fmul_rn((float)P, 6.0f), (float)p.H), (float)p.I);
+    float w_disp = __fmul_rn((float)(p.T + P), B);
+    float w_comb = __fmul_rn((float)(P + p.T), B);
+    ModelArgs ma;
+    ma.alpha = p.alpha; ma.eff[0] = p.eff[0]; ma.eff[1] = p.eff[1]; ma.eff[2] = p.eff[2]; ma.eff[3] = p.eff[3];
+    ma.kinds = p.kinds; ma.c_min = p.c_min; ma.c_step = p.c_step;
+    RouteArgs ra;
+    ra.T = p.T; ra.E = p.E; ra.k = p.k; ra.ep_size = p.ep_size; ra.ep_rank = p.ep_rank; ra.ep_tshard = p.ep_tshard;
+    ra.status = &p.ctl->status; ra.topk_idx = p.topk_idx; ra.gates = p.gates;
+    PlanPick pick;
+    pick.c = n_sm; pick.ki = 0; pick.kind = kPlanSplit; pick.t = 0.f;
+    bool picked = false;
+
+    // ================= phase R: routing
+    for (int it = 0;; ++it) {
+        const int b = local_route ? it : (int)blockIdx.x + it * n_sm;
+        if (b >= p.nblk) break;
+        const int slot = local_route ? b : 0;
+        unsigned long long *r_mask = lmask + slot * (kMaxEE + 1);
+        const bool writer = !local_route || b == (int)blockIdx.x;
+        for (int e = tid; e < EE; e += kThreads) r_mask[e] = 0ull;
+        if (tid == 0) { r_mask[kMaxEE] = 0ull; r_cnt[2 * slot] = 0; r_cnt[2 * slot + 1] = 0; }
+        stage_logits_issue(p, b, lg_s);
+        if (!picked && !ep && p.mode == kModeAuto) {
+            pick = model_pick(ma, S, n_sm, w_comp, w_disp, w_comb, cm_ok, cm_bw, cm_tf, cm_bw_n, cm_tf_n);
+            picked = true;
+        }
+        cp_async_wait_all();
+        __syncthreads();
+        int *idx_b = r_idx + slot * kRouteBlock * kMaxTopK;
+        {
+            const uint32_t a0 = smem_u32(lg_s), a1 = smem_u32(r_mask), a2 = smem_u32(idx_b), a3 = smem_u32(r_cnt + 2 * slot),
+                           a4 = smem_u32(r_p);
+            if (p.E <= 16) route_block_quads<4>(ra.T, ra.E, ra.k, ra.ep_size, ra.ep_rank, ra.ep_tshard, ra.status, ra.topk_idx, ra.gates, b, a0, a1, a2, a3, a4, writer);
+            else if (p.E <= 64) route_block_quads<16>(ra.T, ra.E, ra.k, ra.ep_size, ra.ep_rank, ra.ep_tshard, ra.status, ra.topk_idx, ra.gates, b, a0, a1, a2, a3, a4, writer);
+            else if (p.E <= 128) route_block_quads<32>(ra.T, ra.E, ra.k, ra.ep_size, ra.ep_rank, ra.ep_tshard, ra.status, ra.topk_idx, ra.gates, b, a0, a1, a2, a3, a4, writer);
+            else route_block_quads<64>(ra.T, ra.E, ra.k, ra.ep_size, ra.ep_rank, ra.ep_tshard, ra.status, ra.topk_idx, ra.gates, b, a0, a1, a2, a3, a4, writer);
+        }
+        __syncthreads();
+        if (p.nblk > n_sm) {
+            // this CTA routes several blocks and its scratch is reused: the in-block rank of each (token,
+            // slot) - tokens before it in the block that chose the same expert - goes out to global memory
+            for (int pi = tid; pi < kRouteBlock * p.k; pi += kThreads) {
+                const int tl = pi / p.k, j = pi - tl * p.k;
+                const int t = b * kRouteBlock + tl;
+                if (t < p.T) {
+                    const int e = idx_b[tl * kMaxTopK + j];     // -1: the expert lives on another rank
+                    p.row_of[(size_t)t * p.k + j] = e >= 0 ? __popcll(r_mask[e] & ((1ull << tl) - 1ull)) : -1;
+                }
+            }
+        }
+        if (ep && writer && tid == 0) p.uniq_mask[b] = r_mask[kMaxEE];
+        if (!local_route) {
+            if (ep && tid == 0) {
+                const unsigned long long um = r_mask[kMaxEE];
+                if (r_cnt[0]) atomicAdd(&p.ctl->x_local, (unsigned)r_cnt[0]);
+                if (r_cnt[1]) atomicAdd(&p.ctl->x_in, (unsigned)r_cnt[1]);
+                if (um) atomicAdd(&p.ctl->x_in_uniq, (unsigned)__popcll(um));
+            }
+            const int ntok = min(kRouteBlock, p.T - b * kRouteBlock);
+            const int f = (b * kFine) / p.nblk;
+            for (int e = tid; e < EE; e += kThreads) {
+                const int cnt = e < p.E ? __popcll(r_mask[e]) : ntok;
+                p.hist[(size_t)b * kMaxEE + e] = cnt;
+                if (cnt) atomicAdd(&p.fcnt[f * kMaxEE + e], (unsigned)cnt);
+            }
+            __syncthreads();      // the scratch is reused by this CTA's next block
+        }
+    }
+    if (!picked && !ep && p.mode == kModeAuto) {      // a CTA without a routing block
+        pick = model_pick(ma, S, n_sm, w_comp, w_disp, w_comb, cm_ok, cm_bw, cm_tf, cm_bw_n, cm_tf_n);
+        picked = true;
+    }
+    const unsigned long long tk1 = trace_now_t0(p);
+    bool alive = true;
+    // (arrivals accumulate over the grid barriers of a launch: the later ones count this one in)
+    if (!local_route) alive = grid_barrier(p, S, (unsigned)n_sm, 1);
+    const unsigned long long tk2 = trace_now_t0(p);
+    if (tid == 0) {
+        trace_ev(p, S, kEvRoute, 0u, tk0, tk1, 0u);
+        if (!local_route) trace_ev(p, S, kEvBarrier, 1u, tk1, tk2, 0u);
+    }
 
     // ================= set-up: counts, offsets, plan, segment tables (identical on every CTA)
     int cf[kFine];
     int cnt = 0;
+    unsigned ep_xl = 0u, ep_xi = 0u, ep_xu = 0u;
+    if (local_route) {
 #pragma unroll
-    for (int f = 0; f < kFine; ++f) {
-        cf[f] = (alive && tid < EE) ? (int)__ldcg(p.fcnt + f * kMaxEE + tid) : 0;
-        cnt += cf[f];
+        for (int f = 0; f < kFine; ++f) cf[f] = 0;
+        for (int bb = 0; bb < p.nblk; ++bb) {
+            const int fb = (bb * kFine) / p.nblk;
+            const int c = tid >= EE ? 0 : tid < p.E ? __popcll(lmask[bb * (kMaxEE + 1) + tid]) : min(kRouteBlock, p.T - bb * kRouteBlock);
+#pragma unroll
+            for (int f = 0; f < kFine; ++f) if (f == fb) cf[f] += c;
+            cnt += c;
+            if (ep) {
+                ep_xl += (unsigned)r_cnt[2 * bb]; ep_xi += (unsigned)r_cnt[2 * bb + 1];
+                ep_xu += (unsigned)__popcll(lmask[bb * (kMaxEE + 1) + kMaxEE]);
+            }
+        }
+    } else {
+#pragma unroll
+        for (int f = 0; f < kFine; ++f) {
+            cf[f] = (alive && tid < EE) ? (int)__ldcg(p.fcnt + f * kMaxEE + tid) : 0;
+            cnt += cf[f];
+        }
+        // (asked for together with the counts: one L2 round trip instead of two)
+        if (alive && ep) { ep_xl = __ldcg(&p.ctl->x_local); ep_xi = __ldcg(&p.ctl->x_in); ep_xu = __ldcg(&p.ctl->x_in_uniq); }
     }
-    // (asked for together with the counts: one L2 round trip instead of two)
-    const bool ep_on = alive && p.ep_size > 1;
-    const unsigned ep_xl = ep_on ? __ldcg(&p.ctl->x_local) : 0u, ep_xi = ep_on ? __ldcg(&p.ctl->x_in) : 0u,
-                   ep_xu = ep_on ? __ldcg(&p.ctl->x_in_uniq) : 0u;
     int total_rows;
     const int off = block_excl_scan(cnt, S, total_rows);
     if (tid < EE) S.offsets[tid] = off;
@@ -1593,88 +1779,43 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
         p.offsets[tid] = off;
         if (tid == 0) p.offsets[EE] = total_rows;
     }
-    const int P = p.T * (p.k + p.S);
     if (blockIdx.x == 0 && tid == 0) { p.ctl->ep_x_local = ep_xl; p.ctl->ep_x_in = ep_xi; p.ctl->ep_x_in_uniq = ep_xu; }
-    int plan_c, plan_ki, plan_steal, plan_kind = kPlanSplit;
+    int plan_c, plan_ki, plan_steal = 0, plan_kind = kPlanSplit;
     float plan_t = 0.f;
     if (p.mode == kModeAuto) {
-        // Eq. 1-3 (single-GPU reading: every pair moves through HBM), then Eq. 16 over the grid
-        const float B = (float)(2 * p.H);
-        float w_comp, w_disp, w_comb;
-        if (p.ep_size > 1) {
+        if (ep) {
             // Eq. 1-3 literally: X_local + X_in pairs are computed here, each unique remote token is
             // pulled once, one result goes back per remote pair
             w_comp = __fmul_rn(__fmul_rn(__fmul_rn((float)(ep_xl + ep_xi), 6.0f), (float)p.H), (float)p.I);
             w_disp = __fmul_rn((float)ep_xu, B);
             w_comb = __fmul_rn((float)ep_xi, B);
-        } else {
-            w_comp = __fmul_rn(__fmul_rn(__fmul_rn((float)P, 6.0f), (float)p.H), (float)p.I);
-            w_disp = __fmul_rn((float)(p.T + P), B);
-            w_comb = __fmul_rn((float)(P + p.T), B);
+            pick = model_pick(ma, S, n_sm, w_comp, w_disp, w_comb, cm_ok, cm_bw, cm_tf, cm_bw_n, cm_tf_n);
         }
-        // candidate order = (kind, c ascending, K ascending), index = kind * 256 + thread; the phased plan
-        // is index 512, the rejoin plans follow it; ties go to the smaller index
-        float t = __int_as_float(0x7f800000);
-        int bi = tid;
-        if (cm_ok && (p.kinds & (1 << kPlanSplit))) t = model_t_total(p, cm_bw, cm_tf, cm_ki, w_comp, w_disp, w_comb);
-        if (cm_ok && (p.kinds & (1 << kPlanDispatchAll))) {
-            const float t1 = model_t_dispatch_all(p, cm_bw, cm_tf, cm_bw_n, cm_ki, w_comp, w_disp, w_comb);
-            if (t1 < t) { t = t1; bi = kThreads + tid; }
-        }
-        if (tid == 0 && (p.kinds & (1 << kPlanPhased))) {
-            const float t2 = model_t_phased(p, cm_bw_n, cm_tf_n, w_comp, w_disp, w_comb);
-            if (t2 < t) { t = t2; bi = 2 * kThreads; }
-        }
-        if (cm_ok && cm_ki == 0 && (p.kinds & (1 << kPlanRejoin))) {      // K = 1 only
-            const float t3 = model_t_rejoin(p, cm_bw, cm_tf, cm_bw_n, cm_tf_n, w_comp, w_disp, w_comb);
-            if (t3 < t) { t = t3; bi = 3 * kThreads + tid; }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ot = __shfl_xor_sync(0xffffffffu, t, o);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-            if (ot < t || (ot == t && oi < bi)) { t = ot; bi = oi; }
-        }
-        if (lane == 0) { S.red_f[warp] = t; S.red_i[warp][0] = bi; }
-        __syncthreads();
-        t = S.red_f[0]; bi = S.red_i[0][0];
-        for (int w = 1; w < kThreads / 32; ++w) {
-            const float ot = S.red_f[w];
-            const int oi = S.red_i[w][0];
-            if (ot < t || (ot == t && oi < bi)) { t = ot; bi = oi; }
-        }
-        plan_kind = bi / kThreads;
-        const int bt = bi % kThreads;      // the thread that evaluated the winner
-        plan_c = plan_kind == kPlanPhased ? n_sm : p.c_min + (bt >> 2) * p.c_step;
-        plan_ki = plan_kind == kPlanPhased ? 0 : (bt & 3);
-        plan_t = t;
-        // the winner hands its two table entries to everybody; the pair tiles (256 rows) of the layer at
-        // the chosen K are counted meanwhile (a segment = one expert's rows inside one chunk; its last
-        // pair tile may be half empty)
-        if (tid == bt) { S.red_i[0][1] = __float_as_int(cm_bw); S.red_i[0][2] = __float_as_int(cm_tf); }
-        {
-            const int Kc = 1 << plan_ki, g = kFine / Kc;
+        plan_c = pick.c; plan_ki = pick.ki; plan_kind = pick.kind; plan_t = pick.t;
+        // the steal quota of Eq. 11-14 belongs to the paper's plan kind; in the other kinds the movement
+        // SMs have nothing to wait out (they take GEMM tiles while no combine chunk is ready)
+        if (plan_kind == kPlanSplit) {
+            const float bw_c = __ldg(p.bw + plan_c), tf_c = __ldg(p.tf + n_sm - plan_c);
+            // the pair tiles (256 rows) of the layer at the chosen K (a segment = one expert's rows inside
+            // one chunk; its last pair tile may be half empty)
+            const int Kc = 1 << plan_ki, sh = 3 - plan_ki;
             int acc = 0;
             for (int j = 0; j < Kc; ++j) {
                 int rows = 0;
 #pragma unroll
-                for (int f = 0; f < kFine; ++f) if (f / g == j) rows += cf[f];
+                for (int f = 0; f < kFine; ++f) if ((f >> sh) == j) rows += cf[f];
                 acc += (rows + 2 * kBM - 1) / (2 * kBM);
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
             if (lane == 0) S.red_i[warp][3] = acc;
+            __syncthreads();
+            int n_tiles = 0;
+#pragma unroll
+            for (int w = 0; w < kThreads / 32; ++w) n_tiles += S.red_i[w][3];
+            n_tiles *= p.nt0 + p.nt1;
+            plan_steal = model_n_steal(n_sm, bw_c, tf_c, w_comp, w_disp, w_comb, n_tiles);      // per CTA pair
         }
-        __syncthreads();
-        int n_tiles = 0;
-        for (int w = 0; w < kThreads / 32; ++w) n_tiles += S.red_i[w][3];
-        n_tiles *= p.nt0 + p.nt1;
-        // the steal quota of Eq. 11-14 belongs to the paper's plan kind; in the other kinds the movement
-        // SMs have nothing to wait out (they take GEMM tiles while no combine chunk is ready)
-        plan_steal = plan_kind == kPlanSplit ? model_n_steal(n_sm, __int_as_float(S.red_i[0][1]), __int_as_float(S.red_i[0][2]),
-                                                            w_comp, w_disp, w_comb, n_tiles)   // per CTA pair
-                                             : 0;
-        __syncthreads();
     } else if (p.mode == kModeFixed) {
         plan_c = max(2, min((p.fixed_c + 1) & ~1, n_sm - 2));     // whole CTA pairs
         plan_ki = p.fixed_K >= 8 ? 3 : p.fixed_K >= 4 ? 2 : p.fixed_K >= 2 ? 1 : 0;
@@ -1689,13 +1830,13 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
     const int K = 1 << plan_ki;
     if (tid == 0) S.elastic = (p.elastic_steal || plan_kind == kPlanRejoin) ? 1 : 0;
     {
-        const int g = kFine / K;
+        const int sh = 3 - plan_ki;      // fine chunks per chunk = kFine >> plan_ki
         int run_row = tid < EE ? off : 0;
         int mb_base = 0, pt_base = 0;
         for (int j = 0; j < K; ++j) {
             int rows = 0;
 #pragma unroll
-            for (int f = 0; f < kFine; ++f) if (f / g == j) rows += cf[f];
+            for (int f = 0; f < kFine; ++f) if ((f >> sh) == j) rows += cf[f];
             const int mbs = (rows + kBM - 1) / kBM;
             // m-blocks, pair tiles and unpaired m-blocks of the experts before this one: one packed scan
             unsigned long long tot3;
@@ -1730,9 +1871,9 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
             S.n_gemm = pt_base * (p.nt0 + p.nt1);
             // a small batch is cut into smaller combine tiles (powers of two, so that a tile never
             // straddles two chunks) until every SM has one: its final combine is a latency chain
-            // per tile, not a bandwidth problem
+            // per tile, not a bandwidth problem  (ceil(T / ct) < N  <=>  T <= (N - 1) * ct)
             int ct = kCombTile;
-            while (ct > 1 && (p.T + ct - 1) / ct < n_sm) ct >>= 1;
+            while (ct > 1 && p.T <= (n_sm - 1) * ct) ct >>= 1;
             S.comb_tok = ct;
             S.n_comb = (p.T + ct - 1) / ct;
             if (blockIdx.x == 0) {
@@ -1744,20 +1885,27 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
     }
     __syncthreads();
 
-    const unsigned long long tk3 = trace_now(p);
+    const unsigned long long tk3 = trace_now_t0(p);
     if (tid == 0) trace_ev(p, S, kEvSetup, 0u, tk2, tk3, 0u);
     // ================= permutation fix-up: in-block rank + rows of earlier blocks + expert offset
     if (alive) {
         int fixed = 0;
-        const bool one_block = p.nblk <= n_sm;
+        const bool from_smem = p.nblk <= n_sm;      // this CTA's block is still in its shared memory
         for (int b = blockIdx.x; b < p.nblk; b += n_sm) {
-            const int f = (b * kFine) / p.nblk;
-            const int bstart = (f * p.nblk + kFine - 1) / kFine;
+            const int slot = local_route ? b : 0;
+            const unsigned long long *r_mask = lmask + slot * (kMaxEE + 1);
+            const int *idx_b = r_idx + slot * kRouteBlock * kMaxTopK;
             if (tid < EE) {
                 int base = off;
+                if (local_route) {
+                    for (int bb = 0; bb < b; ++bb) base += __popcll(lmask[bb * (kMaxEE + 1) + tid]);
+                } else {
+                    const int f = (b * kFine) / p.nblk;
+                    const int bstart = (f * p.nblk + kFine - 1) / kFine;
 #pragma unroll
-                for (int ff = 0; ff < kFine; ++ff) if (ff < f) base += cf[ff];
-                for (int bb = bstart; bb < b; ++bb) base += __ldcg(p.hist + (size_t)bb * kMaxEE + tid);
+                    for (int ff = 0; ff < kFine; ++ff) if (ff < f) base += cf[ff];
+                    for (int bb = bstart; bb < b; ++bb) base += __ldcg(p.hist + (size_t)bb * kMaxEE + tid);
+                }
                 r_base[tid] = base;
             }
             __syncthreads();
@@ -1765,15 +1913,15 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
                 const int tl = pi / p.k, j = pi - tl * p.k;
                 const int t = b * kRouteBlock + tl;
                 if (t < p.T) {
-                    // with at most one routing block per CTA the block's selections and masks are still in
-                    // shared memory (one L2 round trip less on the way to the first dispatch tile)
-                    const int e = one_block ? r_idx[tl * kMaxTopK + j] : __ldcg(p.topk_idx + (size_t)t * p.k + j);
-                    const int rk = one_block ? (e >= 0 ? __popcll(r_mask[e] & ((1ull << tl) - 1ull)) : -1)
+                    const int e = from_smem ? idx_b[tl * kMaxTopK + j] : __ldcg(p.topk_idx + (size_t)t * p.k + j);
+                    const int rk = from_smem ? (e >= 0 ? __popcll(r_mask[e] & ((1ull << tl) - 1ull)) : -1)
                                              : __ldcg(p.row_of + (size_t)t * p.k + j);
                     if (rk >= 0) {
                         const int r = rk + r_base[e];
                         p.row_of[(size_t)t * p.k + j] = r;
                         p.token_of[r] = t;
+                    } else if (from_smem) {
+                        p.row_of[(size_t)t * p.k + j] = -1;
                     }
                 }
             }
@@ -1796,10 +1944,11 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
     PipeState ps;
     if (alive) {
         if (p.mode == kModeSerial) {
-            dispatch_phase(p, S, stages, 0x7fffffff, n_sm);
-            alive = grid_barrier(p, S, 2u * n_sm, 2);
+            dispatch_phase(p, S, stages, 0x7fffffff, n_sm, p.nblk <= kLocalBlocks);
+            const unsigned bar0 = p.nblk <= kLocalBlocks ? 0u : (unsigned)n_sm;      // no routing barrier in a small batch
+            alive = grid_barrier(p, S, bar0 + (unsigned)n_sm, 2);
             if (alive) gemm_phase(p, S, stages, tmem_base, &tm, 0x7fffffff, ps);
-            alive = alive && grid_barrier(p, S, 3u * n_sm, 3);
+            alive = alive && grid_barrier(p, S, (p.nblk <= kLocalBlocks ? 0u : (unsigned)n_sm) + 2u * n_sm, 3);
             if (alive) combine_phase(p, S, stages);
         } else {
             const bool mover = (int)blockIdx.x < plan_c;      // role from c* and the block index
@@ -1812,7 +1961,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
             const bool two_roles = plan_kind == kPlanSplit || plan_kind == kPlanRejoin;
             const int dmax = (mover || !two_roles) ? 0x7fffffff : (S.elastic ? 1 : 0);
             const int n_disp = (!two_roles || S.elastic) ? n_sm : plan_c;       // who dispatches at all
-            if (dmax > 0) dispatch_phase(p, S, stages, dmax, n_disp);
+            if (dmax > 0) dispatch_phase(p, S, stages, dmax, n_disp, p.nblk <= kLocalBlocks);
             const int budget = (mover && plan_kind != kPlanPhased) ? plan_steal : 0x7fffffff;
             if (budget > 0 || S.elastic) gemm_phase(p, S, stages, tmem_base, &tm, budget, ps);
             combine_phase(p, S, stages);

@@ -165,3 +165,29 @@ def test_random_groups_shapes_and_ranks(seed):
     else:
         assert bool((out == 0).all())
     moe.close()
+
+
+@pytest.mark.parametrize("T", [50, 64, 128])
+def test_small_batch_every_rank_routing_descriptors_and_output(T):
+    """A batch of one or two routing blocks (routed by every CTA for itself, remote tokens staged from the
+    masks in shared memory): permutation, workload descriptors and partial output of every rank of a group
+    of 4, in every schedule."""
+    cfg = wl.MoEConfig(f"ep_small_batch_T{T}", 95, T=T, H=256, I=384, E=16, k=4, zipf_s=1.0)
+    inp = wl.make_inputs(cfg)
+    x, lg, gu, dn = to_dev(inp)
+    moe = pk.WeaveMoE(gu, dn, cfg.E, cfg.k, cfg.S, max_tokens=cfg.T)
+    R = 4
+    toks = np.arange(cfg.T, dtype=np.int32)
+    for r in range(R):
+        moe.set_expert_parallel(r, R)
+        ref = oracle.moe_tokens_ep(inp.x, inp.logits, inp.gate_up, inp.down, cfg.k, toks, r, R)
+        for sched in [(pk.SCHED_AUTO, 0, 1, 0), (pk.SCHED_SERIAL, 0, 1, 0), (pk.SCHED_FIXED, 12, 2, 3)]:
+            moe.set_schedule(*sched)
+            out = moe.forward(x, lg)
+            moe.check()
+            _check_rank(moe, inp, r, R)
+            if np.abs(ref).max() > 0:
+                check_values(bf16_to_np(out), ref, f"T {T} rank {r} schedule {sched}")
+            else:
+                assert bool((out == 0).all())
+    moe.close()
