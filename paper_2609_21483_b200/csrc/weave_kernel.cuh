@@ -34,7 +34,8 @@ constexpr int kStageB = 128 * kBK * 2;                  // 16 KB: this CTA's hal
 constexpr int kStageBytes = kStageA + kStageB;          // 32 KB
 constexpr int kEpiStageBytes = 4 * 2 * 32 * 64;         // epilogue staging: per warp two buffers of 32 rows x 64 bytes
 constexpr int kRouteBlock = 64;  // tokens per routing block (one 64-bit mask per expert)
-constexpr int kLocalBlocks = 2;  // a batch of at most this many routing blocks is routed by every CTA for itself
+constexpr int kLocalBlocks = 1;  // a batch of at most this many routing blocks is routed by every CTA for itself
+                                 // (measured at two blocks: routing both in every CTA costs more than the grid barrier saves)
 constexpr int kCombTile = 16;    // tokens per combine tile (fewer when the batch would give fewer tiles than SMs)
 constexpr int kMaxEE = 256;      // routed + shared experts
 constexpr int kMaxTopK = 16;
@@ -328,6 +329,21 @@ __device__ __forceinline__ unsigned long long block_excl_scan_packed(unsigned lo
     return wbase + inc - v;
 }
 
+// the two halves of a grid barrier, for a caller that has work to do between arriving and waiting
+__device__ __forceinline__ void grid_barrier_arrive(const KParams &p)
+{
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        red_release_add_u32(&p.ctl->bar_count, 1u);
+    }
+}
+__device__ __forceinline__ bool grid_barrier_wait(const KParams &p, SmemTail &S, unsigned target, int where)
+{
+    if (threadIdx.x == 0) S.bcast[2] = flag_wait_ge(&p.ctl->bar_count, target, p, where) ? 1 : 0;
+    __syncthreads();
+    return S.bcast[2] != 0;
+}
 __device__ __forceinline__ bool grid_barrier(const KParams &p, SmemTail &S, unsigned target, int where)
 {
     __syncthreads();
@@ -1651,7 +1667,8 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
 
     // The cost tables do not depend on the routing: this thread's candidate (c, K) asks for its two
     // entries first of all, and (without an expert-parallel share, whose workload descriptors are counted
-    // while routing) the plan is chosen while the first block's logits are on their way.
+    // while routing) the plan is chosen where it costs nothing: behind the grid barrier's latency, or, in a
+    // batch that has no barrier, while the logits are on their way.
     const int cm_ki = tid & 3, cm_c = p.c_min + (tid >> 2) * p.c_step;
     const bool cm_ok = p.mode == kModeAuto && cm_c >= 2 && cm_c <= p.c_max && cm_c <= n_sm - 2 && (EE << cm_ki) <= kMaxSeg;
     float cm_bw = 0.f, cm_tf = 0.f, cm_bw_n = 0.f, cm_tf_n = 0.f;
@@ -1683,7 +1700,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
         for (int e = tid; e < EE; e += kThreads) r_mask[e] = 0ull;
         if (tid == 0) { r_mask[kMaxEE] = 0ull; r_cnt[2 * slot] = 0; r_cnt[2 * slot + 1] = 0; }
         stage_logits_issue(p, b, lg_s);
-        if (!picked && !ep && p.mode == kModeAuto) {
+        if (local_route && !ep && p.mode == kModeAuto) {      // (no barrier to hide it behind: the logits' way in will do)
             pick = model_pick(ma, S, n_sm, w_comp, w_disp, w_comb, cm_ok, cm_bw, cm_tf, cm_bw_n, cm_tf_n);
             picked = true;
         }
@@ -1729,14 +1746,19 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
             __syncthreads();      // the scratch is reused by this CTA's next block
         }
     }
-    if (!picked && !ep && p.mode == kModeAuto) {      // a CTA without a routing block
-        pick = model_pick(ma, S, n_sm, w_comp, w_disp, w_comb, cm_ok, cm_bw, cm_tf, cm_bw_n, cm_tf_n);
-        picked = true;
-    }
     const unsigned long long tk1 = trace_now_t0(p);
     bool alive = true;
     // (arrivals accumulate over the grid barriers of a launch: the later ones count this one in)
-    if (!local_route) alive = grid_barrier(p, S, (unsigned)n_sm, 1);
+    if (!local_route) {
+        // the plan is chosen between arriving at the barrier and waiting on it: the arrival's way to L2 and
+        // the wait for the slowest routing CTA hide it
+        grid_barrier_arrive(p);
+        if (!picked && !ep && p.mode == kModeAuto) {
+            pick = model_pick(ma, S, n_sm, w_comp, w_disp, w_comb, cm_ok, cm_bw, cm_tf, cm_bw_n, cm_tf_n);
+            picked = true;
+        }
+        alive = grid_barrier_wait(p, S, (unsigned)n_sm, 1);
+    }
     const unsigned long long tk2 = trace_now_t0(p);
     if (tid == 0) {
         trace_ev(p, S, kEvRoute, 0u, tk0, tk1, 0u);

@@ -169,9 +169,9 @@ def test_random_groups_shapes_and_ranks(seed):
 
 @pytest.mark.parametrize("T", [50, 64, 128])
 def test_small_batch_every_rank_routing_descriptors_and_output(T):
-    """A batch of one or two routing blocks (routed by every CTA for itself, remote tokens staged from the
-    masks in shared memory): permutation, workload descriptors and partial output of every rank of a group
-    of 4, in every schedule."""
+    """Batches on both sides of the limit below which every CTA routes the batch for itself (remote tokens
+    are then staged from the masks in shared memory): permutation, workload descriptors and partial output
+    of every rank of a group of 4, in every schedule."""
     cfg = wl.MoEConfig(f"ep_small_batch_T{T}", 95, T=T, H=256, I=384, E=16, k=4, zipf_s=1.0)
     inp = wl.make_inputs(cfg)
     x, lg, gu, dn = to_dev(inp)

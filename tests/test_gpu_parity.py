@@ -520,9 +520,9 @@ def test_argument_errors_at_the_boundary():
 @pytest.mark.parametrize("T", [40, 64, 100, 128, 129])
 @pytest.mark.parametrize("sched", ["auto", "serial", "fixed_k2"])
 def test_small_batches_on_both_sides_of_the_every_cta_routing_limit(T, sched):
-    """Batches of one or two 64-token routing blocks are routed by every CTA for itself (no grid barrier,
-    dispatch sources looked up in shared memory); T = 129 takes the path through global memory.  Shared
-    experts, 64 routed experts, every schedule; whole output against the oracle."""
+    """A batch of one 64-token routing block is routed by every CTA for itself (no grid barrier, dispatch
+    sources looked up in shared memory); larger ones take the path through global memory.  Shared experts,
+    64 routed experts, every schedule; whole output against the oracle."""
     cfg = _small(f"small_T{T}_{sched}", T, 512, 384, 64, 6, 2, zipf=1.0, cfg_id=900 + T)
     s = {"auto": None, "serial": (pk.SCHED_SERIAL, 0, 1, 0), "fixed_k2": (pk.SCHED_FIXED, 24, 2, 3)}[sched]
     moe, _, _ = run_case(cfg, sched=s)
