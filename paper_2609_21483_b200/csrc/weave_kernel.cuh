@@ -1965,29 +1965,26 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
     // ================= main phases
     PipeState ps;
     if (alive) {
-        if (p.mode == kModeSerial) {
-            dispatch_phase(p, S, stages, 0x7fffffff, n_sm, p.nblk <= kLocalBlocks);
-            const unsigned bar0 = p.nblk <= kLocalBlocks ? 0u : (unsigned)n_sm;      // no routing barrier in a small batch
-            alive = grid_barrier(p, S, bar0 + (unsigned)n_sm, 2);
-            if (alive) gemm_phase(p, S, stages, tmem_base, &tm, 0x7fffffff, ps);
-            alive = alive && grid_barrier(p, S, (p.nblk <= kLocalBlocks ? 0u : (unsigned)n_sm) + 2u * n_sm, 3);
-            if (alive) combine_phase(p, S, stages);
-        } else {
-            const bool mover = (int)blockIdx.x < plan_c;      // role from c* and the block index
-            // movement CTAs work through the dispatch queue; every GEMM CTA first dispatches one
-            // m-block too, so that the first wave of GEMM tiles does not wait for a handful of movers
-            // (the mirror image of the final combine on all SMs); the forced "no temporal
-            // scheduling" ablation keeps the two groups apart
-            // (plan kinds beyond the paper's: every CTA works through the dispatch queue first; in the
-            // phased plan every CTA is a "mover" without a steal limit)
-            const bool two_roles = plan_kind == kPlanSplit || plan_kind == kPlanRejoin;
-            const int dmax = (mover || !two_roles) ? 0x7fffffff : (S.elastic ? 1 : 0);
-            const int n_disp = (!two_roles || S.elastic) ? n_sm : plan_c;       // who dispatches at all
-            if (dmax > 0) dispatch_phase(p, S, stages, dmax, n_disp, p.nblk <= kLocalBlocks);
-            const int budget = (mover && plan_kind != kPlanPhased) ? plan_steal : 0x7fffffff;
-            if (budget > 0 || S.elastic) gemm_phase(p, S, stages, tmem_base, &tm, budget, ps);
-            combine_phase(p, S, stages);
-        }
+        // The serial schedule is the phased plan with a grid barrier between the phases (one copy of each
+        // phase's code serves both).
+        const bool serial = p.mode == kModeSerial;
+        const unsigned bar0 = p.nblk <= kLocalBlocks ? 0u : (unsigned)n_sm;      // no routing barrier in a small batch
+        const bool mover = (int)blockIdx.x < plan_c;      // role from c* and the block index
+        // movement CTAs work through the dispatch queue; every GEMM CTA first dispatches one
+        // m-block too, so that the first wave of GEMM tiles does not wait for a handful of movers
+        // (the mirror image of the final combine on all SMs); the forced "no temporal
+        // scheduling" ablation keeps the two groups apart
+        // (plan kinds beyond the paper's: every CTA works through the dispatch queue first; in the
+        // phased plan every CTA is a "mover" without a steal limit)
+        const bool two_roles = plan_kind == kPlanSplit || plan_kind == kPlanRejoin;
+        const int dmax = (mover || !two_roles) ? 0x7fffffff : (S.elastic ? 1 : 0);
+        const int n_disp = (!two_roles || S.elastic) ? n_sm : plan_c;       // who dispatches at all
+        if (dmax > 0) dispatch_phase(p, S, stages, dmax, n_disp, p.nblk <= kLocalBlocks);
+        if (serial) alive = grid_barrier(p, S, bar0 + (unsigned)n_sm, 2);
+        const int budget = (mover && plan_kind != kPlanPhased) ? plan_steal : 0x7fffffff;
+        if (alive && (budget > 0 || S.elastic)) gemm_phase(p, S, stages, tmem_base, &tm, budget, ps);
+        if (serial) alive = alive && grid_barrier(p, S, bar0 + 2u * (unsigned)n_sm, 3);
+        if (alive) combine_phase(p, S, stages);
     }
 
     // ================= leave: free TMEM; the last CTA out re-zeroes the control words
