@@ -1622,6 +1622,14 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
         return;
     }
 
+    // The logits of this CTA's first routing block start on their way before anything else: the copy needs
+    // no barrier, and the set-up of the barriers and of tensor memory (~1 us) hides part of its latency.
+    float *lg_s = reinterpret_cast<float *>(stages + 2048 + kLocalBlocks * kRouteBlock * kMaxTopK * 4);   // [64][route_row_stride(E)]
+    {
+        const int b_first = p.nblk <= kLocalBlocks ? 0 : (int)blockIdx.x;
+        if (b_first < p.nblk) stage_logits_issue(p, b_first, lg_s);
+    }
+
     if (tid == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(&S.full[i], 1); mbar_init(&S.empty[i], 1); }
         // accumulator free: 4 epilogue warps in each CTA of the pair arrive on the leader's barrier
@@ -1654,8 +1662,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
     unsigned long long *lmask = reinterpret_cast<unsigned long long *>(stages + kStages * kStageBytes);   // [kLocalBlocks][256 + 1 (remote tokens)]
     int *r_base = reinterpret_cast<int *>(stages);                                         // [256]
     int *r_cnt = r_base + kMaxEE;                                                          // [kLocalBlocks][2] local / remote pairs
-    int *r_idx = reinterpret_cast<int *>(stages + 2048);                                   // [kLocalBlocks][64][16]
-    float *lg_s = reinterpret_cast<float *>(stages + 2048 + kLocalBlocks * kRouteBlock * kMaxTopK * 4);   // [64][route_row_stride(E)]
+    int *r_idx = reinterpret_cast<int *>(stages + 2048);                                   // [kLocalBlocks][64][16]; the logits follow (lg_s)
     float *r_p = reinterpret_cast<float *>(stages + 96 * 1024);                            // [64][16] exponentials of the selected logits
 
     // A batch of at most kLocalBlocks routing blocks is routed by every CTA for itself: no grid barrier and
@@ -1699,7 +1706,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
         const bool writer = !local_route || b == (int)blockIdx.x;
         for (int e = tid; e < EE; e += kThreads) r_mask[e] = 0ull;
         if (tid == 0) { r_mask[kMaxEE] = 0ull; r_cnt[2 * slot] = 0; r_cnt[2 * slot + 1] = 0; }
-        stage_logits_issue(p, b, lg_s);
+        if (it > 0) stage_logits_issue(p, b, lg_s);      // (the first block's copy was issued at kernel entry)
         if (local_route && !ep && p.mode == kModeAuto) {      // (no barrier to hide it behind: the logits' way in will do)
             pick = model_pick(ma, S, n_sm, w_comp, w_disp, w_comb, cm_ok, cm_bw, cm_tf, cm_bw_n, cm_tf_n);
             picked = true;
