@@ -255,12 +255,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, const 
 {
     if (mbar_try_wait(bar, parity)) return true;
     // the clock is read only every 32 polls (the first reading starts the limit): a reading costs far
-    // more than a poll, and most waits end within a few polls
+    // more than a poll, and most waits end within a few polls.  The abort word is looked at one round
+    // late: its load (an L2 round trip on a line that every SM's queue claims hit) is issued here and its
+    // value used 32 polls later, so the waiting thread is never stalled on it when the barrier completes.
     unsigned long long t0 = 0;
     unsigned it = 0;
+    unsigned ab = 0u;
     while (!mbar_try_wait(bar, parity)) {
         if ((++it & 31u) == 0u) {
-            if (ld_relaxed_u32(&p.ctl->abort)) { note_failed_wait(p.wait_log, where, smem_u32(bar), parity, 2); return false; }
+            if (ab) { note_failed_wait(p.wait_log, where, smem_u32(bar), parity, 2); return false; }
+            ab = ld_relaxed_u32(&p.ctl->abort);
             const unsigned long long now = globaltimer_ns();
             if (t0 == 0) t0 = now;
             else if ((long long)(now - t0) > (long long)p.timeout_ns) {     // signed: a timer that steps back is not a time-out
@@ -1154,9 +1158,11 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t *bar, uint32_t parity
     if (mbar_try_wait_cluster(bar, parity)) return true;
     unsigned long long t0 = 0;
     unsigned it = 0;
+    unsigned ab = 0u;      // looked at one round late, see mbar_wait
     while (!mbar_try_wait_cluster(bar, parity)) {
         if ((++it & 31u) == 0u) {
-            if (ld_relaxed_u32(&p.ctl->abort)) { note_failed_wait(p.wait_log, where, smem_u32(bar), parity, 2); return false; }
+            if (ab) { note_failed_wait(p.wait_log, where, smem_u32(bar), parity, 2); return false; }
+            ab = ld_relaxed_u32(&p.ctl->abort);
             const unsigned long long now = globaltimer_ns();
             if (t0 == 0) t0 = now;
             else if ((long long)(now - t0) > (long long)p.timeout_ns) {
