@@ -253,7 +253,8 @@ int weave_moe_debug_withhold_flag(weave_moe_t h, int m_block);
  * holds the number written.  Kinds: 1 routing, 2 set-up, 3 permutation fix-up, 4 dispatch tile,
  * 5 GEMM tile scheduled (claim until its inputs were ready), 6 GEMM tile epilogue (id = m-block,
  * extra = type << 16 | ns spent before the release), 7 combine tile, 8 wait for a chunk's gemm1,
- * 9 grid barrier, 11 GEMM tile main loop on the MMA issuer (id = type << 16 | rows, extra = ns spent
+ * 9 grid barrier (the one behind the routing; a batch of at most 64 tokens is routed by every CTA for itself
+ * and has none), 11 GEMM tile main loop on the MMA issuer (id = type << 16 | rows, extra = ns spent
  * waiting for a free accumulator). */
 int weave_moe_set_trace(weave_moe_t h, void *buf, int events_per_cta);
 
