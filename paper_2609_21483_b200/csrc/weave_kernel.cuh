@@ -1002,6 +1002,7 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uin
         int b = 0;
         uint32_t ph = 0;
         int ready_upto = -1;     // chunks [0, ready_upto] are known complete
+        bool perm_final = false; // the permutation's rows (row_of, gates) are known final
         bool ok = true;
         for (;;) {
             int q = 0;
@@ -1010,10 +1011,24 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uin
             if (q >= S.n_comb) break;
             const int t0 = q * S.comb_tok;
             const int chunk = (((t0 / kRouteBlock) * kFine) / p.nblk) / g;
+            const int ntok = min(S.comb_tok, p.T - t0);
+            // the tile's rows and gates are final once the permutation is; they are fetched before the wait for
+            // the chunk's last GEMM tile, so that only the row copies themselves follow that wait
+            if (!perm_final) {
+                if (lane == 0) ok = flag_wait_ge(&p.ctl->fix_done, (unsigned)p.nblk, p, 20);
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) break;
+                perm_final = true;
+            }
+            for (int i = lane; i < ntok * kk; i += 32) {
+                const int tt = i / kk, j = i - tt * kk, t = t0 + tt;
+                M.crow[tt][j] = j < p.k ? __ldcg(p.row_of + (size_t)t * p.k + j) : S.offsets[p.E + (j - p.k)] + t;
+                M.cgate[tt][j] = j < p.k ? __ldcg(p.gates + (size_t)t * p.k + j) : 1.0f;
+            }
+            __syncwarp();
             if (chunk > ready_upto) {
                 if (lane == 0) {
                     const unsigned long long tw0 = trace_now(p);
-                    ok = flag_wait_ge(&p.ctl->fix_done, (unsigned)p.nblk, p, 20);
                     for (int j = ready_upto + 1; ok && j <= chunk; ++j) {
                         ok = flag_wait_ge(&p.ctl->y_done[j], y_done_target(S, p, j), p, 21);
                     }
@@ -1024,13 +1039,6 @@ __device__ __forceinline__ void combine_phase(const KParams &p, SmemTail &S, uin
                 ready_upto = chunk;
             }
             const unsigned long long tc0 = trace_now(p);
-            const int ntok = min(S.comb_tok, p.T - t0);
-            for (int i = lane; i < ntok * kk; i += 32) {
-                const int tt = i / kk, j = i - tt * kk, t = t0 + tt;
-                M.crow[tt][j] = j < p.k ? __ldcg(p.row_of + (size_t)t * p.k + j) : S.offsets[p.E + (j - p.k)] + t;
-                M.cgate[tt][j] = j < p.k ? __ldcg(p.gates + (size_t)t * p.k + j) : 1.0f;
-            }
-            __syncwarp();
             for (int tt = 0; tt < ntok && ok; ++tt) {
                 // lane j owns slot j of the token: its rank among the slots that have a row here (slots
                 // whose expert lives on another rank have row -1 and are skipped)
