@@ -2023,7 +2023,8 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
     }
     __syncthreads();
     if (S.bcast[0]) {
-        for (int i = tid; i < kFine * kMaxEE; i += kThreads) p.fcnt[i] = 0u;
+        if (p.nblk > kLocalBlocks)      // (a batch that every CTA routed for itself left the counts untouched)
+            for (int i = tid; i < kFine * kMaxEE; i += kThreads) p.fcnt[i] = 0u;
         for (int i = tid; i < p.nmb_max; i += kThreads) { p.xe_ready[i] = 0u; p.h_ready[i] = 0u; }
         unsigned *z = reinterpret_cast<unsigned *>(p.ctl);
         if (tid < kCtlZeroWords) z[tid] = 0u;
