@@ -430,81 +430,63 @@ __device__ __forceinline__ void stage_logits_issue(const KParams &p, int b, floa
     }
 }
 
-// Top-k selection of routing block b by k rounds of arg-max.  Thread q of a quad holds the order keys of
-// experts q, q+4, ... in NPT registers and knows its own best (largest key, lowest expert index among
-// equals).  A round: the quad's best of the four bests (two shuffle steps; equal keys go to the lower expert
-// index) is slot j; its owner clears it and rescans its registers.  The scratch arrays come as 32-bit
-// shared-memory addresses.  r_mask[e] (64 bits): bit tl set when token tl of the block selected expert e
-// (an expert hosted here); r_idx[tl][j]: the expert of slot j, -1 when another rank hosts it; r_cnt: local /
-// remote (token, expert) pairs of the block (expert-parallel share only); r_p: [64][16] floats of scratch
-// for the exponentials (the sum is only known after the last round).  write_out: this CTA is the one that
-// writes the block's selections and gates to global memory (every CTA routes a small batch for itself, one
-// of them writes it down).
-// Not inlined: its registers (64 keys per thread at E = 256) stay out of the kernel's own allocation.  What it
-// needs of the kernel's parameters comes by value (a reference would turn every use into a load through
-// the generic window onto the parameter bank), and its shared-memory accesses name the shared space
-// (generic atomics that land in shared memory take a slow path).
+// Top-k selection of routing block b by k rounds of arg-max.  Thread q of a quad owns experts q, q+4, ...
+// of its token.  A first pass turns the staged logits into order keys IN PLACE (shared memory) and finds
+// the thread's best (largest key, lowest expert index among equals).  A round: the quad's best of the four
+// bests (two shuffle steps; equal keys go to the lower expert index) is slot j; its owner writes a zero over
+// that key and rescans its keys.  The keys live in shared memory rather than in registers so that both
+// passes are short ROLLED loops: this code runs once or twice per launch, at the speed of instruction
+// fetch, and a loop body is fetched once (the unrolled register version issued fewer instructions and
+// took twice as long).  The scratch arrays come as 32-bit shared-memory addresses.  r_mask[e] (64 bits):
+// bit tl set when token tl of the block selected expert e (an expert hosted here); r_idx[tl][j]: the
+// expert of slot j, -1 when another rank hosts it; r_cnt: local / remote (token, expert) pairs of the
+// block (expert-parallel share only); r_p: [64][16] floats of scratch for the exponentials (the sum is
+// only known after the last round).  write_out: this CTA is the one that writes the block's selections
+// and gates to global memory (every CTA routes a small batch for itself, one of them writes it down).
+// Not inlined (its registers stay out of the kernel's own allocation); what it needs of the kernel's
+// parameters comes by value, and its shared-memory accesses name the shared space (generic atomics that
+// land in shared memory take a slow path).
 struct RouteArgs {
     int T, E, k, ep_size, ep_rank, ep_tshard;
     int *status;
     int *topk_idx;
     float *gates;
 };
-template <int NPT>
 __device__ __noinline__ void route_block_quads(int T, int E, int k, int ep_size, int ep_rank, int ep_tshard, int *status,
                                                int *topk_idx, float *gates, int b, uint32_t lg_s, uint32_t r_mask,
                                                uint32_t r_idx, uint32_t r_cnt, uint32_t r_p, bool write_out)
 {
-    RouteArgs p;      // (scalars in the call: a structure would travel through local memory)
-    p.T = T; p.E = E; p.k = k; p.ep_size = ep_size; p.ep_rank = ep_rank; p.ep_tshard = ep_tshard;
-    p.status = status; p.topk_idx = topk_idx; p.gates = gates;
     static_assert(kThreads == 4 * kRouteBlock, "four threads per token of a routing block");
     const int tl = threadIdx.x >> 2, q = threadIdx.x & 3;
     const int t = b * kRouteBlock + tl;
-    const bool valid = t < p.T;
-    const int stride = route_row_stride(p.E);
-    const int e_lo = p.ep_size > 1 ? p.ep_rank * (p.E / p.ep_size) : 0;
-    const int e_hi = p.ep_size > 1 ? e_lo + p.E / p.ep_size : p.E;
+    const bool valid = t < T;
+    const int e_lo = ep_size > 1 ? ep_rank * (E / ep_size) : 0;
+    const int e_hi = ep_size > 1 ? e_lo + E / ep_size : E;
+    const uint32_t row = lg_s + 4u * (uint32_t)(tl * route_row_stride(E));      // this token's logits, then keys
 
     // keys: 0 = nothing there; every finite logit maps to a key >= 1 that orders like the float
-    // (rows of tokens past the end and columns past E hold stale values: read, then masked)
-    unsigned key[NPT];
+    // (a token past the end keeps all-zero keys: its quad then selects nothing and writes nothing)
+    unsigned bk = 0u;
+    int be = 0x7fffffff;      // expert of this thread's best key
     bool bad = false;
-#pragma unroll
-    for (int i = 0; i < NPT; ++i) {
-        const int e = q + 4 * i;
-        float x = ld_shared_f32(lg_s + 4u * (uint32_t)(tl * stride + min(e, p.E - 1)));
-        const bool there = valid && e < p.E;
+#pragma unroll 2
+    for (int e = q; e < E; e += 4) {
+        float x = ld_shared_f32(row + 4u * (uint32_t)e);
         const bool nf = !(fabsf(x) <= 3.402823466e38f);      // NaN or +-inf: flag it, keep indices in range
-        bad = bad || (there && nf);
+        bad = bad || (valid && nf);
         x = nf ? -3.402823466e38f : x;
         x = __fadd_rn(x, 0.0f);                              // folds -0 into +0, leaves everything else alone
-        key[i] = there ? float_order_key(x) : 0u;
+        const unsigned c = valid ? float_order_key(x) : 0u;
+        st_shared_u32(row + 4u * (uint32_t)e, c);
+        if (c > bk) { bk = c; be = e; }                      // strict: the lower expert index stays
     }
-    if (__any_sync(0xffffffffu, bad) && (threadIdx.x & 31) == 0) atomicCAS(p.status, 0, kErrNonFinite);
-
-    // this thread's best: two chains over the even and the odd registers, strict '>' keeps the lower index
-    auto rescan = [&](unsigned &bk, int &bi) {
-        unsigned k0 = key[0], k1 = NPT > 1 ? key[1] : 0u;
-        int i0 = 0, i1 = 1;
-#pragma unroll
-        for (int i = 2; i < NPT; i += 2) {
-            if (key[i] > k0) { k0 = key[i]; i0 = i; }
-            if (i + 1 < NPT && key[i + 1] > k1) { k1 = key[i + 1]; i1 = i + 1; }
-        }
-        const bool odd = k1 > k0 || (k1 == k0 && i1 < i0);
-        bk = odd ? k1 : k0;
-        bi = odd ? i1 : i0;
-    };
-    unsigned bk;
-    int bi;
-    rescan(bk, bi);
+    if (__any_sync(0xffffffffu, bad) && (threadIdx.x & 31) == 0) atomicCAS(status, 0, kErrNonFinite);
 
     float vmax = 0.f, sum = 0.f;
     int nloc = 0;
     for (int j = 0; j < k; ++j) {
         unsigned hk = bk;
-        int hi = bk ? q + 4 * bi : 0x7fffffff;
+        int hi = bk ? be : 0x7fffffff;
 #pragma unroll
         for (int o = 1; o <= 2; o <<= 1) {
             const unsigned ok = __shfl_xor_sync(0xffffffffu, hk, o);
@@ -523,26 +505,29 @@ __device__ __noinline__ void route_block_quads(int T, int E, int k, int ep_size,
         if (valid && (j & 3) == q) {
             st_shared_u32(r_p + 4u * (uint32_t)(tl * kMaxTopK + j), __float_as_uint(pj));
             if (write_out) {
-                p.topk_idx[(size_t)t * k + j] = hi;
+                topk_idx[(size_t)t * k + j] = hi;
                 st_shared_u32(r_idx + 4u * (uint32_t)(tl * kMaxTopK + j), (uint32_t)(local ? hi : -1));
             }
             if (local) red_shared_or_u32(r_mask + 8u * (uint32_t)hi + 4u * (uint32_t)(tl >> 5), 1u << (tl & 31));
         }
         // the owner takes its winner out and looks for its next best
         if ((hi & 3) == q && hk != 0u) {
-#pragma unroll
-            for (int i = 0; i < NPT; ++i)
-                if (i == bi) key[i] = 0u;
-            rescan(bk, bi);
+            st_shared_u32(row + 4u * (uint32_t)hi, 0u);
+            bk = 0u; be = 0x7fffffff;
+#pragma unroll 4
+            for (int e = q; e < E; e += 4) {
+                const unsigned c = ld_shared_u32(row + 4u * (uint32_t)e);
+                if (c > bk) { bk = c; be = e; }
+            }
         }
     }
     __syncwarp();
     if (valid) {
         if (write_out)
             for (int j = q; j < k; j += 4)
-                p.gates[(size_t)t * k + j] = __fdiv_rn(__uint_as_float(ld_shared_u32(r_p + 4u * (uint32_t)(tl * kMaxTopK + j))), sum);
-        if (p.ep_size > 1 && q == 0 && nloc) {
-            if (t / p.ep_tshard == p.ep_rank) red_shared_add_u32(r_cnt, (uint32_t)nloc);
+                gates[(size_t)t * k + j] = __fdiv_rn(__uint_as_float(ld_shared_u32(r_p + 4u * (uint32_t)(tl * kMaxTopK + j))), sum);
+        if (ep_size > 1 && q == 0 && nloc) {
+            if (t / ep_tshard == ep_rank) red_shared_add_u32(r_cnt, (uint32_t)nloc);
             else {
                 red_shared_add_u32(r_cnt + 4u, (uint32_t)nloc);
                 red_shared_or_u32(r_mask + 8u * (uint32_t)kMaxEE + 4u * (uint32_t)(tl >> 5), 1u << (tl & 31));
@@ -650,7 +635,8 @@ __device__ __noinline__ PlanPick model_pick(const ModelArgs p, SmemTail &S, int 
         const float t3 = model_t_rejoin(p, cm_bw, cm_tf, cm_bw_n, cm_tf_n, w_comp, w_disp, w_comb);
         if (t3 < t) { t = t3; bi = 3 * kThreads + tid; }
     }
-#pragma unroll
+    // (rolled loops: this code runs once per launch, at the speed of instruction fetch)
+#pragma unroll 1
     for (int o = 16; o > 0; o >>= 1) {
         const float ot = __shfl_xor_sync(0xffffffffu, t, o);
         const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
@@ -659,7 +645,7 @@ __device__ __noinline__ PlanPick model_pick(const ModelArgs p, SmemTail &S, int 
     if (lane == 0) { S.red_f[warp] = t; S.red_i[warp][0] = bi; }
     __syncthreads();
     t = S.red_f[0]; bi = S.red_i[0][0];
-#pragma unroll
+#pragma unroll 1
     for (int w = 1; w < kThreads / 32; ++w) {
         const float ot = S.red_f[w];
         const int oi = S.red_i[w][0];
@@ -1731,10 +1717,7 @@ weave_moe_kernel(const __grid_constant__ KParams p, const __grid_constant__ TmaM
         {
             const uint32_t a0 = smem_u32(lg_s), a1 = smem_u32(r_mask), a2 = smem_u32(idx_b), a3 = smem_u32(r_cnt + 2 * slot),
                            a4 = smem_u32(r_p);
-            if (p.E <= 16) route_block_quads<4>(ra.T, ra.E, ra.k, ra.ep_size, ra.ep_rank, ra.ep_tshard, ra.status, ra.topk_idx, ra.gates, b, a0, a1, a2, a3, a4, writer);
-            else if (p.E <= 64) route_block_quads<16>(ra.T, ra.E, ra.k, ra.ep_size, ra.ep_rank, ra.ep_tshard, ra.status, ra.topk_idx, ra.gates, b, a0, a1, a2, a3, a4, writer);
-            else if (p.E <= 128) route_block_quads<32>(ra.T, ra.E, ra.k, ra.ep_size, ra.ep_rank, ra.ep_tshard, ra.status, ra.topk_idx, ra.gates, b, a0, a1, a2, a3, a4, writer);
-            else route_block_quads<64>(ra.T, ra.E, ra.k, ra.ep_size, ra.ep_rank, ra.ep_tshard, ra.status, ra.topk_idx, ra.gates, b, a0, a1, a2, a3, a4, writer);
+            route_block_quads(ra.T, ra.E, ra.k, ra.ep_size, ra.ep_rank, ra.ep_tshard, ra.status, ra.topk_idx, ra.gates, b, a0, a1, a2, a3, a4, writer);
         }
         __syncthreads();
         if (p.nblk > n_sm) {
