@@ -42,8 +42,8 @@ PER_CONFIG = ["c2_mixtral", "c3_qwen3_30b", "c4_dsv2lite_T64", "c4_dsv2lite_T256
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the megakernel, from the ncu
 # captures summarised under profiles/ (None = not captured).  The Qwen3-235B-shaped layer's figure is
 # the mean of three launches captured whole with the time and DRAM counters only (one pass).
-NCU_DRAM_BYTES_PER_LAUNCH = {"c2_mixtral": 4.156e9, "c3_qwen3_30b": 2.620e9, "c5_qwen3_235b": 11.2e9,
-                             "c5_quarter": 2.983e9}
+NCU_DRAM_BYTES_PER_LAUNCH = {"c2_mixtral": 4.297e9, "c3_qwen3_30b": 2.603e9, "c5_qwen3_235b": 11.2e9,
+                             "c5_quarter": 2.991e9}
 
 
 def load_peaks():
