@@ -441,7 +441,7 @@ __device__ __forceinline__ void stage_logits_issue(const KParams &p, int b, floa
 // bit tl set when token tl of the block selected expert e (an expert hosted here); r_idx[tl][j]: the
 // expert of slot j, -1 when another rank hosts it; r_cnt: local / remote (token, expert) pairs of the
 // block (expert-parallel share only); r_p: [64][16] floats of scratch for the exponentials (the sum is
-// only known after the last round).  write_out: this CTA is the one that writes the block's selections
+// only known once all k slots are chosen).  write_out: this CTA is the one that writes the block's selections
 // and gates to global memory (every CTA routes a small batch for itself, one of them writes it down).
 // Its shared-memory accesses name the shared space, so that it could also be compiled out of line (a function
 // that is not inlined sees generic pointers, and generic atomics that land in shared memory take a slow
