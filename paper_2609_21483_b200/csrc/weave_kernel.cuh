@@ -916,7 +916,8 @@ __device__ __forceinline__ void dispatch_phase(const KParams &p, SmemTail &S, ui
                 bool fenced = false;
                 while (pe_head != pe_tail && pe_idx[pe_head % kPend] <= done_idx) {
                     const int s8 = pe_head % kPend;
-                    if (!fenced) { fence_proxy_async(); __threadfence(); fenced = true; }
+                    // (the bulk stores have completed; the release below orders them for whoever acquires the flag)
+                    if (!fenced) { fence_proxy_async_global(); fenced = true; }
                     if (pe_mb[s8] < 0) {
                         red_release_add_u32(&p.ctl->pull_done, 1u);      // a block of remote tokens is staged
                     } else {
@@ -1259,7 +1260,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
                     // the tile's input rows may have been written with ordinary stores on other SMs and
                     // are read by TMA next: the cross-proxy fence sits here, after the acquire and before
                     // the hand-over to the producers, off their critical path
-                    fence_proxy_async();
+                    fence_proxy_async_global();
                     trace_ev(p, S, kEvGemmLoad, (unsigned)g, tp0, trace_now(p), 0u);
                 }
                 mbar_arrive(&S.ti_full[ps.slot]);
@@ -1587,7 +1588,7 @@ __device__ __forceinline__ void gemm_phase(const KParams &p, SmemTail &S, uint8_
             if (lane == 0) mbar_arrive(&S.rel_empty[rs]);
             if (cnt == kRelEnd) break;
             if (lane == 0) {
-                fence_proxy_async();
+                fence_proxy_async_global();
                 red_release_add_u32(flag, cnt);
             }
             if (++rs == kRel) { rs = 0; rph ^= 1u; }

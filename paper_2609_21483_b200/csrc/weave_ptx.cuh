@@ -50,6 +50,9 @@ __device__ __forceinline__ unsigned atom_acqrel_add_u32(unsigned *p, unsigned v)
 // generic-proxy writes (st.global by any SM, made visible through a flag) -> async-proxy reads
 // (TMA) and back
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+// the same restricted to global memory (about a third of the full fence's ~1900 cycles): for hand-overs of rows in
+// global memory between ordinary stores or bulk stores on one SM and tensor-map loads on another
+__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 
 // ---------------------------------------------------------------- mbarrier
 
