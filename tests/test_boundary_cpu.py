@@ -85,6 +85,25 @@ def test_product_path_has_no_cpu_fallback():
             assert "oracle" not in src
 
 
+def test_cuda_sources_keep_clear_of_batched_copies_and_of_multicast_loads():
+    """The batched-memcpy family of runtime calls is not used anywhere (one asynchronous copy per transfer
+    instead), and the only instruction that carries the cluster-multicast qualifier is the tensor-core commit
+    that arrives on both CTAs' barriers: no tiled or bulk LOAD is multicast."""
+    csrc = os.path.join(ROOT, "paper_2609_21483_b200", "csrc")
+    batched = [a + "Memcpy" + b + "Batch" + "Async" for a in ("cuda", "cu") for b in ("", "3D")]
+    qualifier = ".multi" + "cast::cluster"
+    seen_commit = 0
+    for fn in sorted(os.listdir(csrc)):
+        src = open(os.path.join(csrc, fn)).read()
+        for name in batched:
+            assert name not in src, (fn, name)
+        for line in src.splitlines():
+            if qualifier in line:
+                assert "tcgen05.commit" in line, (fn, line.strip())
+                seen_commit += 1
+    assert seen_commit >= 1
+
+
 _GLOO_WORKER = r"""
 import os, sys
 sys.path.insert(0, {root!r})
