@@ -476,11 +476,12 @@ def test_nonfinite_logits_are_reported():
     moe.close()
 
 
-def test_bounded_wait_gives_up_and_handle_recovers():
+@pytest.mark.parametrize("T", [256, 48])
+def test_bounded_wait_gives_up_and_handle_recovers(T):
     """A producer that never publishes one ready flag: the consumer's wait runs out after the
     configured limit, the kernel returns, the host reads WEAVE_ERR_TIMEOUT, and the next forward
-    on the same handle is correct again."""
-    cfg = wl.CONFIGS["c1_tiny"]
+    on the same handle is correct again.  T = 48 is a batch that every CTA routes for itself."""
+    cfg = wl.CONFIGS["c1_tiny"] if T == 256 else wl.CONFIGS["c1_tiny"].with_T(T)
     inp = wl.make_inputs(cfg)
     dev = to_dev(inp)
     moe = pk.WeaveMoE(dev[2], dev[3], cfg.E, cfg.k, cfg.S, max_tokens=cfg.T)
