@@ -54,6 +54,15 @@ def test_static_scratch_entry_point_matches_the_handle_based_one_twice():
     assert call(x, lg, out4) == 0
     torch.cuda.synchronize()
     assert _same_bits(out3, ref2) and _same_bits(out4, ref)
+    # a batch below the limit at which every CTA routes the batch for itself, then the full one once more
+    x3, lg3 = x[:40].contiguous(), lg[:40].contiguous()
+    ref3 = moe.forward(x3, lg3).clone()
+    moe.check()
+    out5, out6 = torch.zeros_like(x3), torch.zeros_like(x)
+    assert call(x3, lg3, out5) == 0
+    assert call(x, lg, out6) == 0
+    torch.cuda.synchronize()
+    assert _same_bits(out5, ref3) and _same_bits(out6, ref)
     moe.close()
 
 
